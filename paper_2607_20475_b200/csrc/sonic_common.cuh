@@ -1,0 +1,279 @@
+// Shared device-side definitions of the sonic kernels (sm_100a).
+//
+// Vocabulary layout: a row is cut into CTA tiles of 8192 elements (eight warp
+// tiles of 1024); a lane owns 32 elements of its warp tile as 128-bit vectors,
+// vector j of lane l starting at element j*32*VEC + l*VEC (fully coalesced).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <math_constants.h>
+
+namespace sonic {
+
+// mode bits (Section 3.5, indicator table)
+constexpr uint32_t M_GRAMMAR = 0x001, M_REPETITION = 0x002, M_FREQUENCY = 0x004, M_PRESENCE = 0x008,
+                   M_BIAS = 0x010, M_TEMPERATURE = 0x020, M_GREEDY = 0x040, M_TOP_K = 0x080,
+                   M_TOP_P = 0x100, M_MIN_P = 0x200;
+constexpr uint32_t M_PENALTIES = M_REPETITION | M_FREQUENCY | M_PRESENCE;
+
+constexpr uint32_t F_NO_TOKEN = 0x1, F_BADPARAM = 0x2, F_FALLBACK = 0x4;
+constexpr uint32_t F_ACCEPT = 0x100;          // workspace only (per-position verification result)
+
+constexpr int OP_SAMPLE = 0, OP_VERIFY = 1, OP_TOPK = 2;
+
+constexpr int WARP_TILE = 1024;               // elements per warp tile
+constexpr int EPL = 32;                       // elements per lane per warp tile
+constexpr int STREAM_THREADS = 256;
+constexpr int STREAM_WARPS = STREAM_THREADS / 32;
+constexpr int CTA_TILE = WARP_TILE * STREAM_WARPS;   // 8192
+constexpr uint32_t CAND_CAP = 16384;          // candidate slots per row in the workspace
+constexpr int SORT_CAP = 8192;                // keys the merge can sort in shared memory
+constexpr int KFAST_SAMPLE = 2048;            // largest top-k the streaming path finishes for sampling rows
+constexpr int KFAST_TOPK = 4096;              // ... and for sonic_topk rows
+constexpr int MAX_VOCAB = 262144;
+
+constexpr int CLS_GREEDY = 0;                 // streaming path, argmax only
+constexpr int CLS_TOPK = 1;                   // streaming path, candidates + merge
+constexpr int CLS_EXACT = 2;                  // full-vocabulary exact path only
+
+constexpr uint32_t ST_FAILED = 0x1;           // streaming path could not prove the row
+constexpr uint32_t ST_BADID = 0x2;            // a list id was out of range
+
+constexpr uint32_t KEY_NEG_INF = 0x007FFFFFu; // okey(-inf)
+
+struct __align__(16) RowState {
+    unsigned int ticket;                      // tiles of this row that have finished streaming
+    unsigned int ncand;                       // candidate slots reserved
+    unsigned int tkey;                        // largest tile cutoff (ordered key); candidates >= it are complete
+    unsigned int status;                      // ST_*
+    unsigned long long best;                  // greedy: largest (key << 32 | ~index)
+    unsigned long long pad;
+};
+
+struct __align__(16) PosResult {              // per logit row, verification only
+    int token;
+    unsigned int flags;                       // F_* | F_ACCEPT
+    float p;                                  // p_l(d_l)
+    int support;
+};
+
+struct KParams {
+    int op, rows, V, K, ktop, dtype;
+    const void *logits;
+    long long row_stride;
+    const uint32_t *mode;
+    const uint32_t *bitmask;
+    long long bitmask_stride;
+    const float *temperature;
+    const int *top_k;
+    const float *top_p;
+    const float *min_p;
+    const float *rep, *freq, *pres;
+    const int *hist_ids, *hist_counts, *hist_len;
+    int hist_stride;
+    const int *bias_ids;
+    const float *bias_vals;
+    const int *bias_len;
+    int bias_stride;
+    const unsigned long long *seed, *offset;
+    const int *draft_tokens;
+    const float *draft_probs;
+    int *out_token;
+    float *out_prob;
+    uint32_t *out_flags;
+    int *out_support;
+    int *out_tokens;
+    int *out_accept;
+    float *out_pdraft;
+    float *out_vals;
+    int *out_idx;
+    RowState *rs;
+    PosResult *pr;
+    unsigned long long *cand;
+};
+
+// Per-row configuration derived from the request's mode bits and parameters.
+struct RowCfg {
+    uint32_t z;
+    int b, l;              // request, position within the request (0 outside verification)
+    int k;                 // top-k bound, 0 = off
+    float tau, p, theta;
+    float alpha, beta, gamma;
+    int hist_len, bias_len;
+    int cls, G;            // path class; groups per warp tile (0 = keep every finite element)
+    bool bad;              // parameter outside its domain
+    bool temp;             // temperature bit
+    bool div_all;          // streaming path divides every element (greedy with temperature)
+};
+
+// Ordered key of a float: unsigned order == float order, -0 folded into +0.
+__device__ __forceinline__ uint32_t okey(float f) {
+    uint32_t b = __float_as_uint(__fadd_rn(f, 0.0f));
+    return b ^ ((b & 0x80000000u) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float unkey(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+
+// Number of groups per warp tile whose maxima bound the tile cutoff.  With G
+// groups the candidates above the row-wide cutoff number about G * Nw^(1-1/G)
+// for position-independent data (Nw warp tiles per row); pick the smallest
+// power of two that gives 1.5 k.  Returns -1 if no setting up to 64 suffices.
+__device__ __forceinline__ int pick_groups(int k, int V) {
+    if (V <= SORT_CAP) return 0;
+    float nw = (float)((V + WARP_TILE - 1) / WARP_TILE);
+    float lg = __log2f(nw);
+    for (int G = 2; G <= 64; G <<= 1) {
+        float est = (float)G * exp2f(lg * (1.0f - 1.0f / (float)G));
+        if (est >= 1.5f * (float)k) return G;
+    }
+    return -1;
+}
+
+__device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) {
+    RowCfg c;
+    c.b = row; c.l = 0;
+    if (P.op == OP_VERIFY) { c.b = row / (P.K + 1); c.l = row - c.b * (P.K + 1); }
+    c.z = (P.op == OP_TOPK) ? M_TOP_K : P.mode[c.b];
+    uint32_t z = c.z;
+    c.bad = false;
+    // a set bit whose parameter array is missing cannot be honoured
+    if ((z & M_TEMPERATURE) && !P.temperature) { c.bad = true; z &= ~M_TEMPERATURE; }
+    if (P.op != OP_TOPK && (z & M_TOP_K) && !P.top_k) { c.bad = true; z &= ~M_TOP_K; }
+    if ((z & M_TOP_P) && !P.top_p) { c.bad = true; z &= ~M_TOP_P; }
+    if ((z & M_MIN_P) && !P.min_p) { c.bad = true; z &= ~M_MIN_P; }
+    if ((z & M_REPETITION) && !P.rep) { c.bad = true; z &= ~M_REPETITION; }
+    if ((z & M_FREQUENCY) && !P.freq) { c.bad = true; z &= ~M_FREQUENCY; }
+    if ((z & M_PRESENCE) && !P.pres) { c.bad = true; z &= ~M_PRESENCE; }
+    if ((z & M_PENALTIES) && !(P.hist_ids && P.hist_counts && P.hist_len)) { c.bad = true; z &= ~M_PENALTIES; }
+    if ((z & M_BIAS) && !(P.bias_ids && P.bias_vals && P.bias_len)) { c.bad = true; z &= ~M_BIAS; }
+    if ((z & M_GRAMMAR) && !P.bitmask) { c.bad = true; z &= ~M_GRAMMAR; }
+    c.z = z;
+    c.temp = (z & M_TEMPERATURE) != 0;
+    c.tau = c.temp ? P.temperature[c.b] : 1.0f;
+    c.k = (P.op == OP_TOPK) ? P.ktop : ((z & M_TOP_K) ? P.top_k[c.b] : 0);
+    c.p = (z & M_TOP_P) ? P.top_p[c.b] : 1.0f;
+    c.theta = (z & M_MIN_P) ? P.min_p[c.b] : 0.0f;
+    c.alpha = (z & M_REPETITION) ? P.rep[c.b] : 1.0f;
+    c.beta = (z & M_FREQUENCY) ? P.freq[c.b] : 0.0f;
+    c.gamma = (z & M_PRESENCE) ? P.pres[c.b] : 0.0f;
+    c.hist_len = (z & M_PENALTIES) ? P.hist_len[c.b] : 0;
+    c.bias_len = (z & M_BIAS) ? P.bias_len[c.b] : 0;
+    bool greedy = (z & M_GREEDY) != 0;
+    if (c.temp && !(c.tau > 0.0f && c.tau < CUDART_INF_F)) c.bad = true;
+    if (!greedy) {
+        if ((z & M_TOP_K) && c.k < 0) c.bad = true;
+        if ((z & M_TOP_P) && !(c.p > 0.0f && c.p <= 1.0f)) c.bad = true;
+        if ((z & M_MIN_P) && !(c.theta > 0.0f && c.theta <= 1.0f)) c.bad = true;
+    }
+    if (c.k < 0) c.k = 0;
+    c.div_all = false;
+    c.G = 0;
+    if (greedy || (P.op == OP_TOPK && c.k == 1)) {
+        c.cls = CLS_GREEDY;
+        c.div_all = c.temp;
+    } else {
+        int kfast = (P.op == OP_TOPK) ? KFAST_TOPK : KFAST_SAMPLE;
+        c.cls = CLS_EXACT;
+        if (c.k > 0 && c.k <= kfast) {
+            int G = pick_groups(c.k, P.V);
+            if (G >= 0) { c.cls = CLS_TOPK; c.G = G; }
+        }
+    }
+    return c;
+}
+
+// ---------------------------------------------------------------- Philox4x32-10
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// 24-bit cell index of the two uniforms of (seed, position, request):
+// u = (a + 1/2) / 2^24, word 0 for the accept test, word 1 for the draw.
+__device__ __forceinline__ void draw_cells(const KParams &P, const RowCfg &c, uint32_t &a_accept, uint32_t &a_draw) {
+    unsigned long long seed = P.seed ? P.seed[c.b] : 0ull;
+    unsigned long long pos = (P.offset ? P.offset[c.b] : 0ull) + (unsigned long long)c.l;
+    uint32_t r[4];
+    philox4x32_10((uint32_t)pos, (uint32_t)(pos >> 32), (uint32_t)c.b, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), r);
+    a_accept = r[0] >> 8;
+    a_draw = r[1] >> 8;
+}
+__device__ __forceinline__ double cell_to_u(uint32_t a) { return ((double)a + 0.5) * (1.0 / 16777216.0); }
+
+// Penalties of one history token, in the paper's order, one rounding per operator.
+__device__ __forceinline__ float apply_penalties(float v, int count, const RowCfg &c) {
+    if (count <= 0) return v;
+    if (c.z & M_REPETITION) v = (v > 0.0f) ? __fdiv_rn(v, c.alpha) : __fmul_rn(v, c.alpha);
+    if (c.z & M_FREQUENCY) v = __fsub_rn(v, __fmul_rn(c.beta, (float)count));
+    if (c.z & M_PRESENCE) v = __fsub_rn(v, c.gamma);
+    return v;
+}
+
+__device__ __forceinline__ unsigned long long ldcg_u64(const unsigned long long *p) {
+    return __ldcg(p);
+}
+
+// Descending bitonic sort of m (power of two) 64-bit keys in shared memory.
+template <int THREADS>
+__device__ __forceinline__ void bitonic_sort_desc(unsigned long long *a, int m, int tid) {
+    for (int k2 = 2; k2 <= m; k2 <<= 1) {
+        for (int j = k2 >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < (m >> 1); i += THREADS) {
+                int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
+                int hi = lo | j;
+                unsigned long long x = a[lo], y = a[hi];
+                bool desc = ((lo & k2) == 0);
+                if ((x < y) == desc) { a[lo] = y; a[hi] = x; }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__device__ __forceinline__ int next_pow2(int n) {
+    int m = 2;
+    while (m < n) m <<= 1;
+    return m;
+}
+
+// Inclusive scan of n doubles in shared memory (in place), THREADS threads,
+// fixed evaluation order (deterministic).  `scratch` holds THREADS doubles.
+template <int THREADS>
+__device__ __forceinline__ void block_inclusive_scan(double *v, int n, double *scratch, int tid) {
+    int chunk = (n + THREADS - 1) / THREADS;
+    int lo = tid * chunk, hi = min(lo + chunk, n);
+    double s = 0.0;
+    for (int i = lo; i < hi; ++i) { s += v[i]; v[i] = s; }
+    scratch[tid] = s;
+    __syncthreads();
+    if (tid < 32) {
+        // serial over 32 segments of THREADS/32 partials each: short and order-fixed
+        constexpr int PER = THREADS / 32;
+        double loc = 0.0;
+        for (int i = 0; i < PER; ++i) { double t = scratch[tid * PER + i]; scratch[tid * PER + i] = loc; loc += t; }
+        double incl = loc;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            double o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (tid >= off) incl += o;
+        }
+        double excl = incl - loc;
+        for (int i = 0; i < PER; ++i) scratch[tid * PER + i] += excl;
+    }
+    __syncthreads();
+    double off = scratch[tid];
+    for (int i = lo; i < hi; ++i) v[i] += off;
+    __syncthreads();
+}
+
+}  // namespace sonic

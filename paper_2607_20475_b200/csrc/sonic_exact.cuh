@@ -1,0 +1,543 @@
+// Exact full-vocabulary kernel: one thread-block cluster of 8 CTAs per row keeps
+// the whole processed row resident in distributed shared memory (ordered 32-bit
+// keys, 32768 per CTA) and answers any truncation exactly with radix descents
+// over count / probability-mass histograms, cluster-wide reductions going
+// through DSMEM and hardware cluster barriers (no flags, no spinning).
+//
+// It serves (a) rows whose answer needs the whole vocabulary by construction
+// (top-k off, or k beyond what the streaming path sorts) and (b) rows the
+// streaming path could not prove.  The paper bounds k at 128 and is lossy
+// beyond it (Section 3.3); this path removes that bound.
+//
+// Probability mass is accumulated as 64-bit fixed point (2^-40 units of the
+// largest weight), so sums are order-independent and replays are bit-identical.
+#pragma once
+#include <cooperative_groups.h>
+#include "sonic_common.cuh"
+#include "sonic_stream.cuh"
+
+namespace sonic {
+namespace cg = cooperative_groups;
+
+constexpr int EX_THREADS = 1024;
+constexpr int EX_WARPS = EX_THREADS / 32;
+constexpr int CL = 8;                         // CTAs per cluster
+constexpr int SLICE_MAX = MAX_VOCAB / CL;     // 32768 keys per CTA
+constexpr int HBINS = 2048;
+constexpr int XV = 4;                         // 64-bit values per exchange
+
+struct Cut {                                  // member: key > v || (key == v && index <= idx)
+    uint32_t v;
+    int idx;
+};
+__device__ __forceinline__ bool member(const Cut &c, uint32_t key, int gidx) {
+    return key > c.v || (key == c.v && gidx <= c.idx);
+}
+__device__ __forceinline__ bool tighter(const Cut &a, const Cut &b) {   // a keeps fewer elements than b
+    return a.v > b.v || (a.v == b.v && a.idx < b.idx);
+}
+
+struct ExactShared {
+    unsigned long long xch[2][CL][XV];
+    unsigned long long vals[XV];
+    unsigned long long wtot[EX_WARPS];
+    unsigned long long red_mass[HBINS / CL];
+    unsigned int red_cnt[HBINS / CL];
+    unsigned int ucount;
+    int flag;
+};
+
+struct ExactCtx {
+    ExactShared *sh;
+    uint32_t *keys;
+    unsigned int *hcnt;
+    unsigned long long *hmass;
+    int rank, lo, len, per, tid, lane, warp;
+    int phase;
+    float Mf;                                  // largest processed logit
+};
+
+// All CTAs contribute XV values; afterwards every CTA holds all of them.
+__device__ __forceinline__ void allgather(ExactCtx &x, const unsigned long long (&v)[XV],
+                                          unsigned long long (&out)[CL][XV]) {
+    __syncthreads();
+    if (x.tid == 0) {
+#pragma unroll
+        for (int i = 0; i < XV; ++i) x.sh->vals[i] = v[i];
+    }
+    __syncthreads();
+    if (x.tid < CL * XV) {
+        int r = x.tid / XV, i = x.tid % XV;
+        ExactShared *remote = cg::this_cluster().map_shared_rank(x.sh, r);
+        remote->xch[x.phase][x.rank][i] = x.sh->vals[i];
+    }
+    cg::this_cluster().sync();
+#pragma unroll
+    for (int r = 0; r < CL; ++r)
+#pragma unroll
+        for (int i = 0; i < XV; ++i) out[r][i] = x.sh->xch[x.phase][r][i];
+    x.phase ^= 1;
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    return v;
+}
+
+// Sum over the block of one 64-bit value per thread; result valid in every thread.
+__device__ __forceinline__ unsigned long long block_sum_u64(ExactCtx &x, unsigned long long v) {
+    v = warp_sum_u64(v);
+    __syncthreads();
+    if (x.lane == 0) x.sh->wtot[x.warp] = v;
+    __syncthreads();
+    unsigned long long t = 0;
+#pragma unroll
+    for (int w = 0; w < EX_WARPS; ++w) t += x.sh->wtot[w];
+    return t;
+}
+
+// Fixed-point softmax weight of a key relative to the row maximum: 2^40 * exp(y - M).
+__device__ __forceinline__ unsigned long long qweight(uint32_t key, float Mf) {
+    float d = __fsub_rn(unkey(key), Mf);
+    const float L1 = 1.44269502162933349609375f;        // fp32(log2 e)
+    const float L2 = 1.925963033500011e-08f;            // log2 e - L1
+    float t = fmaf(d, L1, d * L2);
+    float w;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w) : "f"(t));
+    return __float2ull_rn(w * 1099511627776.0f);
+}
+
+// Ordered crossing: elements are visited in vocabulary-index order (warp w owns a
+// contiguous run of the slice, lanes interleaved), each with weight wf(local index).
+// Computes the row total and, if want_cross, the first element whose inclusive
+// running sum exceeds `target` over the whole row (its global index, -1 if
+// none).  Results are identical in every CTA.  T is a 64-bit type.
+template <typename T, typename WF>
+__device__ int ordered_cross(ExactCtx &x, T target, bool want_cross, WF wf, T &total_out) {
+    const int wch = x.per / EX_WARPS;                    // elements per warp (multiple of 32)
+    const int wlo = x.warp * wch;
+    T wt = T(0);
+    for (int i = wlo + x.lane; i < wlo + wch; i += 32) wt += wf(i);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) wt += __shfl_xor_sync(0xFFFFFFFFu, wt, off);
+    __syncthreads();
+    if (x.lane == 0) x.sh->wtot[x.warp] = *reinterpret_cast<unsigned long long *>(&wt);
+    __syncthreads();
+    T cta_total = T(0), my_woff = T(0);
+    for (int w = 0; w < EX_WARPS; ++w) {
+        T v = *reinterpret_cast<T *>(&x.sh->wtot[w]);
+        if (w == x.warp) my_woff = cta_total;
+        cta_total += v;
+    }
+    unsigned long long v[XV] = {*reinterpret_cast<unsigned long long *>(&cta_total), 0, 0, 0};
+    unsigned long long all[CL][XV];
+    allgather(x, v, all);
+    T off = T(0), total = T(0);
+    int cross_rank = -1;
+    for (int r = 0; r < CL; ++r) {
+        T t = *reinterpret_cast<T *>(&all[r][0]);
+        if (r == x.rank) off = total;
+        if (cross_rank < 0 && total + t > target) cross_rank = r;
+        total += t;
+    }
+    total_out = total;
+    if (!want_cross) return -1;
+    if (cross_rank == x.rank) {
+        int cross_warp = -1;
+        T acc = off;
+        for (int w = 0; w < EX_WARPS; ++w) {
+            T v2 = *reinterpret_cast<T *>(&x.sh->wtot[w]);
+            if (cross_warp < 0 && acc + v2 > target) cross_warp = w;
+            acc += v2;
+        }
+        if (cross_warp < 0) cross_warp = EX_WARPS - 1;    // rounding between levels
+        if (x.warp == cross_warp) {
+            T run = off + my_woff;
+            int found = -1, last_member = -1;
+            for (int i = wlo; i < wlo + wch; i += 32) {
+                T wv = wf(i + x.lane);
+                T incl = wv;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (x.lane >= o) incl += up;
+                }
+                unsigned int hit = __ballot_sync(0xFFFFFFFFu, (run + incl > target) && (wv > T(0)));
+                unsigned int pos = __ballot_sync(0xFFFFFFFFu, wv > T(0));
+                if (hit) { found = x.lo + i + (__ffs(hit) - 1); break; }
+                if (pos) last_member = x.lo + i + (31 - __clz(pos));
+                run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+            if (found < 0) found = last_member;            // rounding between levels: last positive element
+            if (x.lane == 0) x.sh->flag = found;
+        }
+    }
+    __syncthreads();
+    unsigned long long v2[XV] = {0, 0, 0, 0};
+    if (cross_rank == x.rank) v2[0] = (unsigned long long)(long long)x.sh->flag;
+    allgather(x, v2, all);
+    if (cross_rank < 0) return -1;
+    return (int)(long long)all[cross_rank][0];
+}
+
+// Radix descent (11 + 11 + 10 bits) over the keys inside `base`.
+//   by_mass == false: the cut of the `need`-th largest element (need >= 1, need <= count inside base)
+//   by_mass == true : the cut of the smallest ranking prefix whose mass reaches p * (mass inside base)
+__device__ Cut radix_select(ExactCtx &x, const Cut &base, bool by_mass, unsigned long long need, float p) {
+    uint32_t prefix = 0;
+    int pbits = 0;
+    unsigned long long target = need;
+    unsigned long long ties = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+        const int nb = (pass < 2) ? 11 : 10;
+        const int nbins = 1 << nb;
+        const int shift = 32 - pbits - nb;
+        for (int i = x.tid; i < HBINS; i += EX_THREADS) { x.hcnt[i] = 0; x.hmass[i] = 0ull; }
+        __syncthreads();
+        for (int i = x.tid; i < x.len; i += EX_THREADS) {
+            uint32_t key = x.keys[i];
+            if (pbits && (key >> (32 - pbits)) != prefix) continue;
+            if (!member(base, key, x.lo + i)) continue;
+            uint32_t bin = (key >> shift) & (nbins - 1);
+            atomicAdd(&x.hcnt[bin], 1u);
+            if (by_mass) atomicAdd(&x.hmass[bin], qweight(key, x.Mf));
+        }
+        cg::this_cluster().sync();
+        // CTA r reduces bins [r*bpr, (r+1)*bpr) over the cluster
+        const int bpr = nbins / CL;
+        unsigned long long sc = 0, sm = 0;
+        if (x.tid < bpr) {
+            int bin = x.rank * bpr + x.tid;
+            unsigned int cc = 0;
+            unsigned long long mm = 0;
+            for (int r = 0; r < CL; ++r) {
+                cc += *cg::this_cluster().map_shared_rank(&x.hcnt[bin], r);
+                if (by_mass) mm += *cg::this_cluster().map_shared_rank(&x.hmass[bin], r);
+            }
+            x.sh->red_cnt[x.tid] = cc;
+            x.sh->red_mass[x.tid] = mm;
+            sc = cc; sm = mm;
+        }
+        sc = block_sum_u64(x, sc);
+        sm = block_sum_u64(x, sm);
+        unsigned long long v[XV] = {sc, sm, 0, 0};
+        unsigned long long all[CL][XV];
+        allgather(x, v, all);                 // every remote histogram read precedes this barrier
+        if (by_mass && pass == 0) {
+            unsigned long long Zq = 0;
+            for (int r = 0; r < CL; ++r) Zq += all[r][1];
+            double t = ceil((double)p * (double)Zq);
+            target = (unsigned long long)t;
+            if (target > Zq) target = Zq;
+            if (target < 1) target = 1;
+        }
+        // segment (CTA) holding the crossing, scanning from the largest keys
+        int seg = -1;
+        unsigned long long cum = 0;
+        for (int r = CL - 1; r >= 0; --r) {
+            unsigned long long s = by_mass ? all[r][1] : all[r][0];
+            if (cum + s >= target) { seg = r; break; }
+            cum += s;
+        }
+        if (seg < 0) {                             // target beyond the total: cannot happen for valid calls
+            seg = 0;
+            cum -= by_mass ? all[0][1] : all[0][0];
+            target = cum + (by_mass ? all[0][1] : all[0][0]);
+        }
+        unsigned long long v2[XV] = {0, 0, 0, 0};
+        if (x.rank == seg && x.tid == 0) {
+            unsigned long long c2 = cum;
+            int b = 0;
+            for (int t = bpr - 1; t >= 0; --t) {
+                unsigned long long s = by_mass ? x.sh->red_mass[t] : (unsigned long long)x.sh->red_cnt[t];
+                if (c2 + s >= target) { b = t; break; }
+                c2 += s;
+            }
+            x.sh->vals[0] = (unsigned long long)(seg * bpr + b);
+            x.sh->vals[1] = target > c2 ? target - c2 : 1ull;   // still needed inside the bin
+            x.sh->vals[2] = x.sh->red_cnt[b];
+        }
+        __syncthreads();
+        if (x.rank == seg) { v2[0] = x.sh->vals[0]; v2[1] = x.sh->vals[1]; v2[2] = x.sh->vals[2]; }
+        allgather(x, v2, all);
+        prefix = (prefix << nb) | (uint32_t)all[seg][0];
+        target = all[seg][1];
+        ties = all[seg][2];
+        pbits += nb;
+    }
+    // prefix is the boundary value; `target` of its ties (by count) or enough of them to reach the mass
+    unsigned long long r = target;
+    if (by_mass) {
+        unsigned long long qw = qweight(prefix, x.Mf);
+        r = qw ? (target + qw - 1) / qw : 1;
+    }
+    if (r < 1) r = 1;
+    if (r > ties) r = ties;
+    const uint32_t v = prefix;
+    unsigned long long tot;
+    int idx = ordered_cross<unsigned long long>(
+        x, r - 1, true,
+        [&](int i) -> unsigned long long {
+            return (i < x.len && x.keys[i] == v && member(base, v, x.lo + i)) ? 1ull : 0ull;
+        },
+        tot);
+    Cut c;
+    c.v = v;
+    c.idx = idx;
+    return c;
+}
+
+template <int DT>
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
+sonic_exact_kernel(const KParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ExactCtx x;
+    x.rank = (int)cg::this_cluster().block_rank();
+    const int row = blockIdx.x / CL;
+    x.tid = threadIdx.x; x.lane = x.tid & 31; x.warp = x.tid >> 5;
+    x.phase = 0;
+    const RowCfg c = load_cfg(P, row);
+    RowState *rs = P.rs + row;
+    const unsigned int status = __ldcg(&rs->status);
+    if (c.cls != CLS_EXACT && !(status & ST_FAILED)) return;          // uniform over the cluster
+
+    x.keys = reinterpret_cast<uint32_t *>(smem_raw);
+    x.hmass = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4);
+    x.hcnt = reinterpret_cast<unsigned int *>(smem_raw + SLICE_MAX * 4 + HBINS * 8);
+    x.sh = reinterpret_cast<ExactShared *>(smem_raw + SLICE_MAX * 4 + HBINS * 12);
+    unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 12 + 8192);
+
+    const int V = P.V;
+    x.per = (((V + CL - 1) / CL) + 1023) & ~1023;
+    x.lo = x.rank * x.per;
+    x.len = max(0, min(V - x.lo, x.per));
+    cg::this_cluster().sync();                               // every CTA of the cluster is resident before DSMEM traffic
+
+    // ---- load the slice, mask, sparse patches, temperature, keys
+    constexpr int VEC = VecTraits<DT>::VEC;
+    float *zf = reinterpret_cast<float *>(x.keys);
+    const bool masked = (c.z & M_GRAMMAR) != 0;
+    const uint32_t *mrow = masked ? P.bitmask + (long long)row * P.bitmask_stride : nullptr;
+    const int nwords = (V + 31) >> 5;
+#pragma unroll 4
+    for (int li = x.tid * VEC; li < x.per; li += EX_THREADS * VEC) {
+        const int first = x.lo + li;
+        float vals[VEC];
+        if (first < V) {
+            uint4 raw;
+            if (DT == 0) raw = __ldcs(reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(P.logits) + (long long)row * P.row_stride + first));
+            else raw = __ldcs(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(P.logits) + (long long)row * P.row_stride + first));
+            uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+            uint32_t mw = 0xFFFFFFFFu;
+            if (masked) { int w = first >> 5; mw = (w < nwords ? __ldg(mrow + w) : 0u) >> (first & 31); }
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) {
+                float v;
+                if (DT == 0) v = __uint_as_float(r[q]);
+                else v = __uint_as_float((q & 1) ? (r[q >> 1] & 0xFFFF0000u) : (r[q >> 1] << 16));
+                if (first + q >= V || !((mw >> q) & 1u)) v = -CUDART_INF_F;
+                vals[q] = v;
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) vals[q] = -CUDART_INF_F;
+        }
+#pragma unroll
+        for (int q = 0; q < VEC; q += 4)
+            *reinterpret_cast<float4 *>(zf + li + q) = make_float4(vals[q], vals[q + 1], vals[q + 2], vals[q + 3]);
+    }
+    __syncthreads();
+    int bad = c.bad ? 1 : 0;
+    if (c.hist_len > 0) {
+        const int *hid = P.hist_ids + (long long)c.b * P.hist_stride;
+        const int *hct = P.hist_counts + (long long)c.b * P.hist_stride;
+        for (int t = x.tid; t < c.hist_len; t += EX_THREADS) {
+            int id = __ldg(hid + t), ct = __ldg(hct + t);
+            if (id < 0 || id >= V) { bad = 1; continue; }
+            int li = id - x.lo;
+            if (li >= 0 && li < x.len) zf[li] = apply_penalties(zf[li], ct, c);
+        }
+    }
+    __syncthreads();
+    if (c.bias_len > 0) {
+        const int *bid = P.bias_ids + (long long)c.b * P.bias_stride;
+        const float *bvl = P.bias_vals + (long long)c.b * P.bias_stride;
+        for (int t = x.tid; t < c.bias_len; t += EX_THREADS) {
+            int id = __ldg(bid + t);
+            if (id < 0 || id >= V) { bad = 1; continue; }
+            int li = id - x.lo;
+            if (li >= 0 && li < x.len) zf[li] = __fadd_rn(zf[li], __ldg(bvl + t));
+        }
+    }
+    bad = __syncthreads_or(bad);
+    uint32_t kmax = 0;
+    unsigned long long nfin = 0;
+    for (int li = x.tid; li < x.per; li += EX_THREADS) {
+        float z = zf[li];
+        float y = c.temp ? __fdiv_rn(z, c.tau) : z;
+        uint32_t k = okey(y);
+        x.keys[li] = k;
+        kmax = max(kmax, k);
+        nfin += (k > KEY_NEG_INF && li < x.len) ? 1 : 0;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, off));
+    nfin = block_sum_u64(x, nfin);
+    __syncthreads();
+    if (x.lane == 0) x.sh->wtot[x.warp] = kmax;
+    __syncthreads();
+    for (int w = 0; w < EX_WARPS; ++w) kmax = max(kmax, (uint32_t)x.sh->wtot[w]);
+    unsigned long long all[CL][XV];
+    {
+        unsigned long long v[XV] = {kmax, nfin, 0, 0};
+        allgather(x, v, all);
+    }
+    uint32_t Mkey = 0;
+    unsigned long long Nf = 0;
+    for (int r = 0; r < CL; ++r) { Mkey = max(Mkey, (uint32_t)all[r][0]); Nf += all[r][1]; }
+    x.Mf = unkey(Mkey);
+    const bool leader = (x.rank == 0 && x.tid == 0);
+
+    if (bad) {
+        if (leader) { emit_row(P, c, row, -1, 0.0f, F_BADPARAM | F_FALLBACK, 0, 0.0f); rs->status = 0; }
+        cg::this_cluster().sync();
+        return;
+    }
+
+    // ---------------------------------------------------------------- sonic_topk rows
+    if (P.op == OP_TOPK) {
+        Cut all_cut; all_cut.v = 0; all_cut.idx = -1;
+        Cut cut = all_cut;
+        if (c.k < V) cut = radix_select(x, all_cut, false, (unsigned long long)c.k, 1.0f);
+        // compact the members into CTA 0's sort buffer
+        if (x.tid == 0) x.sh->ucount = 0;
+        __syncthreads();
+        unsigned long long cnt = 0;
+        for (int i = x.tid; i < x.len; i += EX_THREADS) cnt += member(cut, x.keys[i], x.lo + i) ? 1 : 0;
+        cnt = block_sum_u64(x, cnt);
+        unsigned long long v[XV] = {cnt, 0, 0, 0};
+        allgather(x, v, all);
+        unsigned int off = 0;
+        for (int r = 0; r < x.rank; ++r) off += (unsigned int)all[r][0];
+        unsigned long long *dst = cg::this_cluster().map_shared_rank(sortbuf, 0);
+        for (int i = x.tid; i < x.len; i += EX_THREADS) {
+            uint32_t key = x.keys[i];
+            if (member(cut, key, x.lo + i)) {
+                unsigned int pos = off + atomicAdd(&x.sh->ucount, 1u);
+                if (pos < (unsigned int)KFAST_TOPK) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+            }
+        }
+        cg::this_cluster().sync();
+        if (x.rank == 0) {
+            const int n = min(c.k, KFAST_TOPK);
+            const int m = next_pow2(n);
+            for (int i = n + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
+            __syncthreads();
+            bitonic_sort_desc<EX_THREADS>(sortbuf, m, x.tid);
+            for (int j = x.tid; j < n; j += EX_THREADS) {
+                unsigned long long kv = sortbuf[j];
+                P.out_vals[(size_t)row * P.ktop + j] = unkey((uint32_t)(kv >> 32));
+                P.out_idx[(size_t)row * P.ktop + j] = (int)(~(uint32_t)kv);
+            }
+            if (x.tid == 0) rs->status = 0;
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- sampling / verification rows
+    if (Nf == 0) {
+        if (leader) { emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN | F_FALLBACK, 0, 0.0f); rs->status = 0; }
+        cg::this_cluster().sync();
+        return;
+    }
+    Cut cut; cut.v = KEY_NEG_INF; cut.idx = -1;            // every finite element
+    if (c.k > 0 && (unsigned long long)c.k < Nf) cut = radix_select(x, cut, false, (unsigned long long)c.k, 1.0f);
+    const Cut cut_k = cut;
+    if (c.z & M_TOP_P) {
+        Cut cp = radix_select(x, cut_k, true, 0ull, c.p);
+        if (tighter(cp, cut)) cut = cp;
+    }
+    if (c.z & M_MIN_P) {
+        double thr = (double)x.Mf + log((double)c.theta);
+        float tf = (float)thr;
+        if ((double)tf < thr) tf = nextafterf(tf, CUDART_INF_F);
+        uint32_t tk = okey(tf);
+        Cut cm; cm.v = tk - 1; cm.idx = -1;                // key >= tk
+        if (tighter(cm, cut)) cut = cm;
+    }
+    // final support: size, mass, draw in index order
+    unsigned long long cnt = 0;
+    for (int i = x.tid; i < x.len; i += EX_THREADS) cnt += member(cut, x.keys[i], x.lo + i) ? 1 : 0;
+    cnt = block_sum_u64(x, cnt);
+    {
+        unsigned long long v[XV] = {cnt, 0, 0, 0};
+        allgather(x, v, all);
+    }
+    unsigned long long nS = 0;
+    for (int r = 0; r < CL; ++r) nS += all[r][0];
+
+    uint32_t a_acc, a_draw;
+    draw_cells(P, c, a_acc, a_draw);
+    auto wq = [&](int i) -> unsigned long long {
+        return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? qweight(x.keys[i], x.Mf) : 0ull;
+    };
+    // total mass first (target depends on it): a crossing search with an unreachable target
+    unsigned long long Wq;
+    ordered_cross<unsigned long long>(x, ~0ull, false, wq, Wq);
+    const unsigned long long mul = 2ull * a_draw + 1ull;               // u = mul / 2^25
+    const unsigned long long T = (__umul64hi(Wq, mul) << 39) | ((Wq * mul) >> 25);
+    unsigned long long dummy;
+    int token = ordered_cross<unsigned long long>(x, T, true, wq, dummy);
+
+    uint32_t flags = F_FALLBACK;
+    float p_draft = 0.0f;
+    if (P.op == OP_VERIFY && c.l < P.K) {
+        const int d = P.draft_tokens[(size_t)c.b * P.K + c.l];
+        const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)V;
+        unsigned long long v[XV] = {0, 0, 0, 0};
+        if (d >= x.lo && d < x.lo + x.len) v[0] = wq(d - x.lo) + 1ull;   // +1 marks the owner
+        allgather(x, v, all);
+        unsigned long long qd = 0;
+        for (int r = 0; r < CL; ++r) if (all[r][0]) qd = all[r][0] - 1ull;
+        double Pd = (double)qd / (double)Wq;
+        double Q = (d >= 0 && d < V) ? (double)__ldg(q + d) : 0.0;
+        bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);
+        p_draft = (float)Pd;
+        if (accept) flags |= F_ACCEPT;
+        // residual max(0, p - q) over the support, weights in fp64
+        const double Md = (double)x.Mf;
+        auto wd = [&](int i) -> double {
+            return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? exp((double)unkey(x.keys[i]) - Md) : 0.0;
+        };
+        double Wd;
+        ordered_cross<double>(x, CUDART_INF, false, wd, Wd);
+        auto rd = [&](int i) -> double {
+            if (!(i < x.len && member(cut, x.keys[i], x.lo + i))) return 0.0;
+            double r = exp((double)unkey(x.keys[i]) - Md) / Wd - (double)__ldg(q + x.lo + i);
+            return r > 0.0 ? r : 0.0;
+        };
+        double R;
+        ordered_cross<double>(x, CUDART_INF, false, rd, R);
+        if (R > 0.0) {
+            double dummy2;
+            int t2 = ordered_cross<double>(x, cell_to_u(a_draw) * R, true, rd, dummy2);
+            if (t2 >= 0) token = t2;
+        }
+    }
+    // probability of the chosen token under the final distribution
+    {
+        unsigned long long v[XV] = {0, 0, 0, 0};
+        if (token >= x.lo && token < x.lo + x.len) v[0] = wq(token - x.lo) + 1ull;
+        allgather(x, v, all);
+        unsigned long long qt = 0;
+        for (int r = 0; r < CL; ++r) if (all[r][0]) qt = all[r][0] - 1ull;
+        if (leader) {
+            emit_row(P, c, row, token, (float)((double)qt / (double)Wq), flags, (int)nS, p_draft);
+            rs->status = 0;
+        }
+    }
+    cg::this_cluster().sync();
+}
+
+}  // namespace sonic
