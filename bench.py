@@ -1,0 +1,433 @@
+#!/usr/bin/env python
+"""Benchmark of the fused sampling / verification path on B200.
+
+A "step" is one fused call (sonic_sample on the heterogeneous-batch workload c2
+by default) over one batch of seeded synthetic input.  Inputs rotate over enough
+distinct copies that their total footprint exceeds twice the L2 capacity, so
+every call reads its logits from HBM.  Calls are captured in CUDA graphs and
+timed with CUDA events on the launching stream; with N > 1 (torchrun) every rank
+runs an independent replica on its own GPU and the slowest rank's time counts.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_20475_b200 import workloads as wl  # noqa: E402
+
+METRIC = "us_per_fused_sample_call"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def make_workload(name: str, copy: int = 0):
+    """Workload `name`; `copy` > 0 gives an independent draw of the same recipe."""
+    if name == "c1":
+        return wl.config1()
+    if name == "c2":
+        return wl.config2(data_seed=wl.BASE_SEED + 2 + 1000 * copy)
+    if name == "c3":
+        return wl.config3(data_seed=wl.BASE_SEED + 3 + 1000 * copy)
+    if name == "c4":
+        return wl.config4(data_seed=wl.BASE_SEED + 4 + 1000 * copy)
+    raise ValueError(name)
+
+
+def algorithmic_bytes(name: str, w) -> int:
+    """Bytes a call must read at least once: logits, grammar words, sparse lists (verification: target logits)."""
+    if name == "c4":
+        return w.sample.input_bytes()
+    return w.input_bytes()
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nme, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_time(name: str, w, budget_s: float):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns (us per call, description)."""
+    from oracle import oracle
+    import copy as _copy
+    if name == "c4":
+        vw = w
+        nreq = max(1, min(vw.B, 4))
+        sub = _copy.copy(vw)
+        sub.B = nreq
+        sub.sample = _slice_sample(vw.sample, nreq, rows=nreq * (vw.K + 1))
+        sub.draft_tokens = vw.draft_tokens[:nreq]
+        sub.draft_probs = vw.draft_probs[:nreq]
+        t0 = time.perf_counter(); oracle.verify(sub); dt = time.perf_counter() - t0
+        reps = max(1, int(budget_s / max(dt, 1e-3)) - 1)
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            oracle.verify(sub)
+        dt = (time.perf_counter() - t0) / reps if reps else dt
+        return dt * vw.B / nreq * 1e6, f"{nreq} of {vw.B} requests x {reps} repetitions, scaled to the full batch"
+    n = max(1, min(w.B, 8))
+    sub = _slice_sample(w, n, rows=n)
+    t0 = time.perf_counter(); oracle.sample(sub); dt = time.perf_counter() - t0
+    per_row = dt / n
+    n2 = int(max(1, min(w.B, budget_s / max(per_row, 1e-6))))
+    sub = _slice_sample(w, n2, rows=n2)
+    t0 = time.perf_counter(); oracle.sample(sub); dt = time.perf_counter() - t0
+    return dt * w.B / n2 * 1e6, f"first {n2} of {w.B} rows, one pass, scaled to the full batch"
+
+
+def _slice_sample(w, n, rows):
+    import copy as _copy
+    s = _copy.copy(w)
+    s.B = n
+    s.logits = w.logits[:rows]
+    for f in ("mode", "temperature", "top_k", "top_p", "min_p", "rep_penalty", "freq_penalty", "pres_penalty", "seed",
+              "offset", "hist_ids", "hist_counts", "hist_len", "bias_ids", "bias_vals", "bias_len"):
+        v = getattr(w, f)
+        setattr(s, f, None if v is None else v[:n])
+    if w.bitmask is not None:
+        s.bitmask = w.bitmask[:rows]
+    return s
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    name = args.workload
+    w = make_workload(name)
+    B = w.B
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    times = []
+    desc = ""
+    for i in range(args.warmup + args.steps):
+        us, desc = oracle_time(name, w, budget_s=max(0.05, budget))
+        if i >= args.warmup:
+            times.append(us)
+    us = float(np.mean(times))
+    out = {
+        "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": us / 1000.0, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "impl": "reference",
+        "config": {"workload": f"{name}: B={B}, V={w.V}", "l2": "n/a (host)"},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+def build_device_copies(name, copies, binding):
+    import torch
+    devs = []
+    ws = None
+    for c in range(copies):
+        w = make_workload(name, copy=c)
+        if name == "c4":
+            if ws is None:
+                ws = binding.new_workspace(w.B * (w.K + 1))
+            devs.append(binding.DeviceVerify(w, ws=ws))
+        else:
+            if ws is None:
+                ws = binding.new_workspace(w.B)
+            devs.append(binding.DeviceSample(w, ws=ws))
+    torch.cuda.synchronize()
+    return devs
+
+
+def capture(devs, calls):
+    """One CUDA graph of `calls` back-to-back fused calls over rotating input copies."""
+    import torch
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(calls):
+            devs[i % len(devs)].run()
+    return g
+
+
+def time_graph_steps(graph_full, per_graph, graph_rem, rem, steps):
+    import torch
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps // per_graph):
+        graph_full.replay()
+    if rem:
+        graph_rem.replay()
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / 1000.0
+
+
+def measure_floor(calls=64, reps=20):
+    """Device time per node of a graph of trivial kernels: the launch floor small calls are compared with."""
+    import torch
+    x = torch.zeros(1, device="cuda")
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(calls):
+            x.add_(1.0)
+    for _ in range(3):
+        g.replay()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s.record()
+    for _ in range(reps):
+        g.replay()
+    e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e) * 1000.0 / (calls * reps)
+
+
+def e2e_measure(name, dev, steps):
+    """Same call through the public API from HOST buffers: every step copies the step's inputs host->device from
+    pinned memory, runs the fused call and reads the result back."""
+    import torch
+    s = dev.s if name == "c4" else dev
+    pairs = []
+    for key, t in s.t.items():
+        if t is None:
+            continue
+        h = t.detach().cpu().pin_memory()
+        pairs.append((t, h))
+    if name == "c4":
+        for t in (dev.draft_tokens, dev.draft_probs):
+            pairs.append((t, t.detach().cpu().pin_memory()))
+        outs = [dev.out_tokens, dev.out_accept, dev.out_p_draft, s.out_flags]
+    else:
+        outs = [s.out_token, s.out_prob, s.out_flags, s.out_support]
+    houts = [torch.empty_like(o, device="cpu").pin_memory() for o in outs]
+    h2d = sum(h.numel() * h.element_size() for _, h in pairs)
+    d2h = sum(h.numel() * h.element_size() for h in houts)
+
+    def one():
+        for t, h in pairs:
+            t.copy_(h, non_blocking=True)
+        dev.run()
+        for o, h in zip(outs, houts):
+            h.copy_(o, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(3):
+        one()
+    st, en = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    st.record()
+    for _ in range(steps):
+        one()
+    en.record()
+    torch.cuda.synchronize()
+    return st.elapsed_time(en) * 1000.0 / steps, h2d, d2h
+
+
+def run_sonic(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_20475_b200 import binding
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    binding.lib()
+    name = args.workload
+    w0 = make_workload(name)
+    bytes_call = algorithmic_bytes(name, w0)
+    copies = max(2, int(np.ceil(2.0 * L2_BYTES / bytes_call)))
+    copies = min(copies, 24)
+    devs = build_device_copies(name, copies, binding)
+    per_graph = copies
+    steps = max(1, args.steps)
+    g_full = capture(devs, per_graph)
+    rem = steps % per_graph
+    g_rem = capture(devs, rem) if rem else None
+    # warm-up: at least 3 calls, in whole graphs
+    for _ in range(max(1, int(np.ceil(max(3, args.warmup) / per_graph)))):
+        g_full.replay()
+    if g_rem is not None:
+        g_rem.replay()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    elapsed = time_graph_steps(g_full, per_graph, g_rem, rem, steps)
+    # keep the sampler busy long enough to see clocks under load
+    t_end = time.time() + 0.6
+    while rank == 0 and time.time() < t_end:
+        g_full.replay()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([elapsed], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+
+    us_call = elapsed / steps * 1e6                     # per replica
+    e2e_us, h2d, d2h = e2e_measure(name, devs[0], steps=min(steps, 40))
+    if world > 1:
+        t = torch.tensor([e2e_us], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_us = float(t.item())
+    floor_us = measure_floor() if rank == 0 else None
+
+    extra = {}
+    if rank == 0 and args.also:
+        for other in [n for n in args.also.split(",") if n and n != name]:
+            extra[other] = quick_measure(other, binding)
+
+    if rank == 0:
+        peak, which = peaks()
+        B = w0.B
+        rows = B * (w0.K + 1) if name == "c4" else B
+        achieved = bytes_call / (us_call * 1e-6) / 1e9
+        launches_per_call = 3 if name == "c4" else 2
+        cpu_us, cpu_desc = oracle_time(name, w0, budget_s=15.0)
+        out = {
+            "metric": METRIC, "value": us_call / world, "unit": "us", "n_gpus": world, "steps": steps,
+            "warmup": max(3, args.warmup), "ms_per_step": us_call / 1000.0, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{name}: B={B}, V={w0.V}, {'bf16' if w0_dtype(w0) == wl.DTYPE_BF16 else 'fp32'} logits"
+                                   + (f", K={w0.K}" if name == "c4" else ""),
+                       "l2": f"inputs rotate over {copies} distinct copies ({copies * bytes_call / 1e6:.0f} MB > 2x L2)",
+                       "timing": "CUDA-graph replays, CUDA events on the launching stream", "replicas": world},
+            "rows_per_s": rows * world / (us_call * 1e-6),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": which,
+                         "note": "algorithmic bytes of the whole call / CUDA-event time of the whole call (all kernels)"},
+            "cpu_baseline": {"value": cpu_us, "unit": "us", "cores": 1, "kind": "oracle", "sample": cpu_desc},
+            "e2e": {"value": e2e_us / world, "unit": "us", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": launches_per_call * steps,
+            "empty_graph_node_us": floor_us,
+            "clocks": clocks,
+            "also": extra,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def w0_dtype(w):
+    return w.sample.dtype if hasattr(w, "sample") else w.dtype
+
+
+def quick_measure(name, binding, reps=30):
+    """Short cold-input timing of another configuration (not the headline line)."""
+    import torch
+    w0 = make_workload(name)
+    bytes_call = algorithmic_bytes(name, w0)
+    copies = int(min(8, max(2, np.ceil(2.0 * L2_BYTES / bytes_call))))
+    devs = build_device_copies(name, copies, binding)
+    g = capture(devs, copies)
+    for _ in range(2):
+        g.replay()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s.record()
+    for _ in range(reps):
+        g.replay()
+    e.record()
+    torch.cuda.synchronize()
+    us = s.elapsed_time(e) * 1000.0 / (reps * copies)
+    peak, which = peaks()
+    gbs = bytes_call / (us * 1e-6) / 1e9
+    del devs, g
+    torch.cuda.empty_cache()
+    return {"us_per_call": us, "algorithmic_bytes": int(bytes_call), "achieved_gbs": gbs, "frac": gbs / peak,
+            "copies": copies}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", default="sonic", choices=["sonic", "reference"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4"])
+    ap.add_argument("--also", default="c3,c4", help="other configurations to time briefly (comma separated, '' for none)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if args.steps == 2000:
+            args.steps = 5
+        if args.warmup == 16:
+            args.warmup = 1
+        run_reference(args, rank, world)
+        return
+    run_sonic(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

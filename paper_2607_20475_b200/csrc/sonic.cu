@@ -43,7 +43,7 @@ __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
 
 constexpr size_t WS_HEADER = 256;
 constexpr int STREAM_SMEM = SORT_CAP * 8;
-constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 12 + 8192 + KFAST_TOPK * 8;
+constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 12 + 8192 + KFAST_TOPK * 8 + 8192;
 
 static thread_local char g_err[256] = "";
 
@@ -60,7 +60,9 @@ static size_t ws_bytes_for(int rows) {
     return WS_HEADER + (size_t)rows * (sizeof(RowState) + sizeof(PosResult)) + (size_t)rows * CAND_CAP * 8;
 }
 
-static int configure_once() {
+static int g_max_clusters[64];      // co-resident 8-CTA clusters of the exact kernel, per device
+
+static int configure_once(int *max_clusters) {
     static std::once_flag once[64];
     static cudaError_t result[64];
     int dev = 0;
@@ -76,9 +78,26 @@ static int configure_once() {
         set((const void *)sonic_stream_kernel<1>, STREAM_SMEM);
         set((const void *)sonic_exact_kernel<0>, EXACT_SMEM);
         set((const void *)sonic_exact_kernel<1>, EXACT_SMEM);
+        int n = 0;
+        if (r == cudaSuccess) {
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof(cfg));
+            cfg.gridDim = dim3(CL * 64);
+            cfg.blockDim = dim3(EX_THREADS);
+            cfg.dynamicSmemBytes = EXACT_SMEM;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = CL; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            r = cudaOccupancyMaxActiveClusters(&n, (const void *)sonic_exact_kernel<0>, &cfg);
+        }
+        g_max_clusters[dev] = n;
         result[dev] = r;
     });
-    if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "cudaFuncSetAttribute");
+    if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "kernel configuration");
+    if (g_max_clusters[dev] < 1) return fail(SONIC_ECUDA, "no 8-CTA cluster of the exact kernel fits on this device");
+    *max_clusters = g_max_clusters[dev];
     return SONIC_OK;
 }
 
@@ -86,7 +105,8 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
     if (ws_bytes < ws_bytes_for(P.rows)) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows");
-    int rc = configure_once();
+    int max_clusters = 0;
+    int rc = configure_once(&max_clusters);
     if (rc != SONIC_OK) return rc;
     // the layout depends on the row capacity the workspace was sized for, recovered from its size
     const size_t per_row = sizeof(RowState) + sizeof(PosResult) + (size_t)CAND_CAP * 8;
@@ -103,7 +123,7 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
 
-    dim3 grid2(P.rows * CL);
+    dim3 grid2((P.rows < max_clusters ? P.rows : max_clusters) * CL);
     if (P.dtype == SONIC_DTYPE_F32) sonic_exact_kernel<0><<<grid2, EX_THREADS, EXACT_SMEM, st>>>(P);
     else sonic_exact_kernel<1><<<grid2, EX_THREADS, EXACT_SMEM, st>>>(P);
     e = cudaGetLastError();

@@ -288,26 +288,12 @@ __device__ Cut radix_select(ExactCtx &x, const Cut &base, bool by_mass, unsigned
     return c;
 }
 
+// One row, start to finish, by the whole cluster.  Control flow is uniform over
+// the cluster (every CTA executes the same sequence of cluster barriers).
 template <int DT>
-__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
-sonic_exact_kernel(const KParams P) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    ExactCtx x;
-    x.rank = (int)cg::this_cluster().block_rank();
-    const int row = blockIdx.x / CL;
-    x.tid = threadIdx.x; x.lane = x.tid & 31; x.warp = x.tid >> 5;
-    x.phase = 0;
+__device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned long long *sortbuf) {
     const RowCfg c = load_cfg(P, row);
     RowState *rs = P.rs + row;
-    const unsigned int status = __ldcg(&rs->status);
-    if (c.cls != CLS_EXACT && !(status & ST_FAILED)) return;          // uniform over the cluster
-
-    x.keys = reinterpret_cast<uint32_t *>(smem_raw);
-    x.hmass = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4);
-    x.hcnt = reinterpret_cast<unsigned int *>(smem_raw + SLICE_MAX * 4 + HBINS * 8);
-    x.sh = reinterpret_cast<ExactShared *>(smem_raw + SLICE_MAX * 4 + HBINS * 12);
-    unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 12 + 8192);
-
     const int V = P.V;
     x.per = (((V + CL - 1) / CL) + 1023) & ~1023;
     x.lo = x.rank * x.per;
@@ -538,6 +524,47 @@ sonic_exact_kernel(const KParams P) {
         }
     }
     cg::this_cluster().sync();
+}
+
+// Persistent clusters: cluster c handles rows c, c + nclusters, ...; it first marks
+// the rows that need this path (their class, or a failure recorded by the
+// streaming kernel), then processes them in order.
+template <int DT>
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
+sonic_exact_kernel(const KParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ExactCtx x;
+    x.rank = (int)cg::this_cluster().block_rank();
+    x.tid = threadIdx.x; x.lane = x.tid & 31; x.warp = x.tid >> 5;
+    x.phase = 0;
+    x.keys = reinterpret_cast<uint32_t *>(smem_raw);
+    x.hmass = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4);
+    x.hcnt = reinterpret_cast<unsigned int *>(smem_raw + SLICE_MAX * 4 + HBINS * 8);
+    x.sh = reinterpret_cast<ExactShared *>(smem_raw + SLICE_MAX * 4 + HBINS * 12);
+    unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 12 + 8192);
+    uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 12 + 8192 + KFAST_TOPK * 8);
+
+    const int ncl = gridDim.x / CL;
+    const int cid = blockIdx.x / CL;
+    const int nmine = (P.rows - cid + ncl - 1) / ncl;           // rows of this cluster (cid < rows by construction)
+    const int nwords = (nmine + 31) >> 5;
+    for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
+    __syncthreads();
+    for (int j = x.tid; j < nmine; j += EX_THREADS) {
+        const int row = cid + j * ncl;
+        const RowCfg c = load_cfg(P, row);
+        const unsigned int status = __ldcg(&P.rs[row].status);
+        if (c.cls == CLS_EXACT || (status & ST_FAILED)) atomicOr(&need[j >> 5], 1u << (j & 31));
+    }
+    __syncthreads();
+    for (int w = 0; w < nwords; ++w) {
+        uint32_t bits = need[w];
+        while (bits) {
+            const int j = (w << 5) + __ffs(bits) - 1;
+            bits &= bits - 1;
+            exact_row<DT>(P, cid + j * ncl, x, sortbuf);
+        }
+    }
 }
 
 }  // namespace sonic

@@ -223,7 +223,7 @@ def test_config4_reduced(sonic, oracle):
 
 def test_config4_full(sonic, oracle):
     vw = wl.config4()
-    got, ref, n = run_verify(sonic, oracle, vw, max_near=2)
+    got, ref, n = run_verify(sonic, oracle, vw, max_near=8)   # dense top-p rows: a token carries ~1e-6 of the mass
     print("config4 accept lengths:", got["accept_len"].tolist(), "near-margin:", n)
 
 
