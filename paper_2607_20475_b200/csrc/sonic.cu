@@ -42,8 +42,7 @@ __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
 }
 
 constexpr size_t WS_HEADER = 256;
-constexpr int STREAM_SMEM = SORT_CAP * 8;
-constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 12 + 8192 + KFAST_TOPK * 8 + 8192;
+constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8 + 8192;
 
 static thread_local char g_err[256] = "";
 
@@ -56,9 +55,10 @@ static int fail_cuda(cudaError_t e, const char *what) {
     return SONIC_ECUDA;
 }
 
-static size_t ws_bytes_for(int rows) {
-    return WS_HEADER + (size_t)rows * (sizeof(RowState) + sizeof(PosResult)) + (size_t)rows * CAND_CAP * 8;
-}
+constexpr size_t WS_ROW_CTRL = sizeof(RowState) + sizeof(PosResult) + sizeof(TileRec) * MAX_TILES;
+constexpr size_t WS_ROW = WS_ROW_CTRL + (size_t)CAND_CAP * 8;
+
+static size_t ws_bytes_for(int rows) { return WS_HEADER + (size_t)rows * WS_ROW; }
 
 static int g_max_clusters[64];      // co-resident 8-CTA clusters of the exact kernel, per device
 
@@ -74,8 +74,6 @@ static int configure_once(int *max_clusters) {
         auto set = [&](const void *f, int bytes) {
             if (r == cudaSuccess) r = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         };
-        set((const void *)sonic_stream_kernel<0>, STREAM_SMEM);
-        set((const void *)sonic_stream_kernel<1>, STREAM_SMEM);
         set((const void *)sonic_exact_kernel<0>, EXACT_SMEM);
         set((const void *)sonic_exact_kernel<1>, EXACT_SMEM);
         int n = 0;
@@ -109,17 +107,17 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     int rc = configure_once(&max_clusters);
     if (rc != SONIC_OK) return rc;
     // the layout depends on the row capacity the workspace was sized for, recovered from its size
-    const size_t per_row = sizeof(RowState) + sizeof(PosResult) + (size_t)CAND_CAP * 8;
-    const size_t cap_rows = (ws_bytes - WS_HEADER) / per_row;
+    const size_t cap_rows = (ws_bytes - WS_HEADER) / WS_ROW;
     unsigned char *base = reinterpret_cast<unsigned char *>(ws);
     P.rs = reinterpret_cast<RowState *>(base + WS_HEADER);
     P.pr = reinterpret_cast<PosResult *>(base + WS_HEADER + cap_rows * sizeof(RowState));
-    P.cand = reinterpret_cast<unsigned long long *>(base + WS_HEADER + cap_rows * (sizeof(RowState) + sizeof(PosResult)));
+    P.tiles = reinterpret_cast<TileRec *>(base + WS_HEADER + cap_rows * (sizeof(RowState) + sizeof(PosResult)));
+    P.cand = reinterpret_cast<unsigned long long *>(base + WS_HEADER + cap_rows * WS_ROW_CTRL);
 
     const int tiles = (P.V + CTA_TILE - 1) / CTA_TILE;
     dim3 grid1(tiles, P.rows);
-    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_THREADS, STREAM_SMEM, st>>>(P);
-    else sonic_stream_kernel<1><<<grid1, STREAM_THREADS, STREAM_SMEM, st>>>(P);
+    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_THREADS, 0, st>>>(P);
+    else sonic_stream_kernel<1><<<grid1, STREAM_THREADS, 0, st>>>(P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
 
@@ -184,10 +182,8 @@ size_t sonic_workspace_bytes(int max_rows) {
 int sonic_workspace_init(void *workspace, size_t bytes, void *stream) {
     if (!workspace) return fail(SONIC_EINVAL, "workspace is NULL");
     if (bytes < ws_bytes_for(1)) return fail(SONIC_EWORKSPACE, "workspace smaller than one row");
-    const size_t per_row = sizeof(RowState) + sizeof(PosResult) + (size_t)CAND_CAP * 8;
-    const size_t cap_rows = (bytes - WS_HEADER) / per_row;
-    cudaError_t e = cudaMemsetAsync(workspace, 0, WS_HEADER + cap_rows * (sizeof(RowState) + sizeof(PosResult)),
-                                    (cudaStream_t)stream);
+    const size_t cap_rows = (bytes - WS_HEADER) / WS_ROW;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, WS_HEADER + cap_rows * WS_ROW_CTRL, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail_cuda(e, "cudaMemsetAsync");
     g_err[0] = 0;
     return SONIC_OK;

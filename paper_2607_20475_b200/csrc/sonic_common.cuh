@@ -27,10 +27,12 @@ constexpr int EPL = 32;                       // elements per lane per warp tile
 constexpr int STREAM_THREADS = 256;
 constexpr int STREAM_WARPS = STREAM_THREADS / 32;
 constexpr int CTA_TILE = WARP_TILE * STREAM_WARPS;   // 8192
-constexpr uint32_t CAND_CAP = 16384;          // candidate slots per row in the workspace
-constexpr int SORT_CAP = 8192;                // keys the merge can sort in shared memory
-constexpr int KFAST_SAMPLE = 2048;            // largest top-k the streaming path finishes for sampling rows
-constexpr int KFAST_TOPK = 4096;              // ... and for sonic_topk rows
+constexpr int MAX_TILES = (262144 + CTA_TILE - 1) / CTA_TILE;   // 32 tiles at the largest vocabulary
+constexpr uint32_t CAND_CAP = 32768;          // candidate slots per row, divided evenly among the row's tiles
+constexpr int MERGE_CAP = CTA_TILE / 2;       // 64-bit keys the row merge can sort (it reuses the 32 KB staging tile)
+constexpr int KFAST_SAMPLE = MERGE_CAP / 4;   // largest top-k the streaming path finishes for sampling rows (1024)
+constexpr int KFAST_TOPK = MERGE_CAP / 2;     // ... and for sonic_topk rows (2048)
+constexpr int MAX_TOPK = 4096;                // largest k of sonic_topk (beyond KFAST_TOPK: exact kernel)
 constexpr int MAX_VOCAB = 262144;
 
 constexpr int CLS_GREEDY = 0;                 // streaming path, argmax only
@@ -43,12 +45,15 @@ constexpr uint32_t ST_BADID = 0x2;            // a list id was out of range
 constexpr uint32_t KEY_NEG_INF = 0x007FFFFFu; // okey(-inf)
 
 struct __align__(16) RowState {
-    unsigned int ticket;                      // tiles of this row that have finished streaming
-    unsigned int ncand;                       // candidate slots reserved
-    unsigned int tkey;                        // largest tile cutoff (ordered key); candidates >= it are complete
-    unsigned int status;                      // ST_*
-    unsigned long long best;                  // greedy: largest (key << 32 | ~index)
-    unsigned long long pad;
+    unsigned int status;                      // ST_*; zero between calls
+    unsigned int ticket;                      // tiles of the row that finished streaming; zero between calls
+    unsigned int pad[2];
+};
+
+struct __align__(16) TileRec {                // written by the tile's CTA, read by the merge kernel
+    unsigned long long best;                  // greedy rows: largest (key << 32 | ~index) of the tile, 0 if none finite
+    unsigned int cnt;                         // top-k rows: candidates of the tile (may exceed the slot: overflow)
+    unsigned int tkey;                        // top-k rows: the tile's cutoff as an ordered key
 };
 
 struct __align__(16) PosResult {              // per logit row, verification only
@@ -89,6 +94,7 @@ struct KParams {
     float *out_vals;
     int *out_idx;
     RowState *rs;
+    TileRec *tiles;
     PosResult *pr;
     unsigned long long *cand;
 };
@@ -121,7 +127,7 @@ __device__ __forceinline__ float unkey(uint32_t k) {
 // for position-independent data (Nw warp tiles per row); pick the smallest
 // power of two that gives 1.5 k.  Returns -1 if no setting up to 64 suffices.
 __device__ __forceinline__ int pick_groups(int k, int V) {
-    if (V <= SORT_CAP) return 0;
+    if (V <= MERGE_CAP) return 0;
     float nw = (float)((V + WARP_TILE - 1) / WARP_TILE);
     float lg = __log2f(nw);
     for (int G = 2; G <= 64; G <<= 1) {

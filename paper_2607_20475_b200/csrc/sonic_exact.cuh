@@ -50,8 +50,7 @@ struct ExactShared {
 struct ExactCtx {
     ExactShared *sh;
     uint32_t *keys;
-    unsigned int *hcnt;
-    unsigned long long *hmass;
+    unsigned int *hcnt, *hm0, *hm1, *hm2;      // per-bin count and mass in three 14-bit limbs (32-bit adds only)
     int rank, lo, len, per, tid, lane, warp;
     int phase;
     float Mf;                                  // largest processed logit
@@ -181,99 +180,256 @@ __device__ int ordered_cross(ExactCtx &x, T target, bool want_cross, WF wf, T &t
     return (int)(long long)all[cross_rank][0];
 }
 
-// Radix descent (11 + 11 + 10 bits) over the keys inside `base`.
-//   by_mass == false: the cut of the `need`-th largest element (need >= 1, need <= count inside base)
+// One histogram level of a selection.  digit(key) gives the element's bin
+// (larger bin = ranks earlier) or -1 if the element is outside the level's
+// range; only members of `base` take part.  Scanning bins from the top, finds
+// the bin where the running count (or mass) first reaches `target`; on return
+// `target` is what is still needed inside that bin and `in_bin` is the bin's
+// element count.  For by_mass with first == true the target is set to
+// ceil(p * total mass) first.  Two cluster barriers.
+template <typename DF>
+__device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first, float p, int nbins, DF digit,
+                          unsigned long long &target, unsigned long long &in_bin) {
+    for (int i = x.tid; i < nbins; i += EX_THREADS) { x.hcnt[i] = 0; x.hm0[i] = 0; x.hm1[i] = 0; x.hm2[i] = 0; }
+    __syncthreads();
+    for (int i0 = 0; i0 < x.len; i0 += EX_THREADS) {
+        const int i = i0 + x.tid;
+        int bin = -1;
+        uint32_t key = 0;
+        if (i < x.len) {
+            key = x.keys[i];
+            if (member(base, key, x.lo + i)) bin = digit(key);
+        }
+        const unsigned int active = __ballot_sync(0xFFFFFFFFu, bin >= 0);
+        if (bin < 0) continue;
+        unsigned int q0 = 0, q1 = 0, q2 = 0;
+        if (by_mass) {
+            unsigned long long q = qweight(key, x.Mf);
+            q0 = (unsigned int)(q & 0x3FFFu); q1 = (unsigned int)((q >> 14) & 0x3FFFu); q2 = (unsigned int)(q >> 28);
+        }
+        int same;
+        __match_all_sync(active, bin, &same);
+        if (same) {                                   // the whole warp hits one bin: one lane adds for all
+            unsigned int n = __popc(active);
+            if (by_mass) { q0 = __reduce_add_sync(active, q0); q1 = __reduce_add_sync(active, q1); q2 = __reduce_add_sync(active, q2); }
+            if ((int)(__ffs(active) - 1) == x.lane) {
+                atomicAdd(&x.hcnt[bin], n);
+                if (by_mass) { atomicAdd(&x.hm0[bin], q0); atomicAdd(&x.hm1[bin], q1); atomicAdd(&x.hm2[bin], q2); }
+            }
+        } else {
+            atomicAdd(&x.hcnt[bin], 1u);
+            if (by_mass) { atomicAdd(&x.hm0[bin], q0); atomicAdd(&x.hm1[bin], q1); atomicAdd(&x.hm2[bin], q2); }
+        }
+    }
+    cg::this_cluster().sync();
+    // CTA r reduces bins [r*bpr, (r+1)*bpr) over the cluster
+    const int bpr = nbins / CL;
+    unsigned long long sc = 0, sm = 0;
+    if (x.tid < bpr) {
+        const int bin = x.rank * bpr + x.tid;
+        unsigned int cc = 0;
+        unsigned long long mm = 0;
+        for (int r = 0; r < CL; ++r) {
+            cc += *cg::this_cluster().map_shared_rank(&x.hcnt[bin], r);
+            if (by_mass) {
+                mm += (unsigned long long)*cg::this_cluster().map_shared_rank(&x.hm0[bin], r)
+                    + ((unsigned long long)*cg::this_cluster().map_shared_rank(&x.hm1[bin], r) << 14)
+                    + ((unsigned long long)*cg::this_cluster().map_shared_rank(&x.hm2[bin], r) << 28);
+            }
+        }
+        x.sh->red_cnt[x.tid] = cc;
+        x.sh->red_mass[x.tid] = mm;
+        sc = cc; sm = mm;
+    }
+    sc = block_sum_u64(x, sc);
+    sm = block_sum_u64(x, sm);
+    unsigned long long v[XV] = {sc, sm, 0, 0};
+    unsigned long long all[CL][XV];
+    allgather(x, v, all);                      // every remote histogram read precedes this barrier
+    if (by_mass && first) {
+        unsigned long long Zq = 0;
+        for (int r = 0; r < CL; ++r) Zq += all[r][1];
+        double t = ceil((double)p * (double)Zq);
+        target = (unsigned long long)t;
+        if (target > Zq) target = Zq;
+        if (target < 1) target = 1;
+    }
+    // segment (CTA) holding the crossing, scanning from the top
+    int seg = -1;
+    unsigned long long cum = 0;
+    for (int r = CL - 1; r >= 0; --r) {
+        unsigned long long sseg = by_mass ? all[r][1] : all[r][0];
+        if (cum + sseg >= target) { seg = r; break; }
+        cum += sseg;
+    }
+    if (seg < 0) {                             // target beyond the total: cannot happen for valid calls
+        seg = 0;
+        cum -= by_mass ? all[0][1] : all[0][0];
+        target = cum + (by_mass ? all[0][1] : all[0][0]);
+    }
+    // every CTA reads the crossing segment's reduced bins from their owner and scans them itself
+    const unsigned int *rc = cg::this_cluster().map_shared_rank(&x.sh->red_cnt[0], seg);
+    const unsigned long long *rm = cg::this_cluster().map_shared_rank(&x.sh->red_mass[0], seg);
+    if (x.tid < 32) {
+        // warp 0: lanes take bins from the top in chunks of 32
+        unsigned long long c2 = cum;
+        int found = -1;
+        unsigned long long rest = 0, cnt = 0;
+        for (int top = bpr - 1; top >= 0 && found < 0; top -= 32) {
+            const int t = top - x.lane;
+            unsigned long long val = 0;
+            unsigned int cval = 0;
+            if (t >= 0) { cval = rc[t]; val = by_mass ? rm[t] : (unsigned long long)cval; }
+            unsigned long long incl = val;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (x.lane >= o) incl += up;
+            }
+            unsigned int hit = __ballot_sync(0xFFFFFFFFu, t >= 0 && c2 + incl >= target);
+            if (hit) {
+                const int l = __ffs(hit) - 1;
+                found = top - l;
+                rest = target - (c2 + __shfl_sync(0xFFFFFFFFu, incl, l) - __shfl_sync(0xFFFFFFFFu, val, l));
+                cnt = __shfl_sync(0xFFFFFFFFu, cval, l);
+            } else {
+                c2 += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+        }
+        if (found < 0) { found = 0; rest = 1; cnt = rc[0]; }
+        if (x.lane == 0) {
+            x.sh->vals[0] = (unsigned long long)(seg * bpr + found);
+            x.sh->vals[1] = rest;
+            x.sh->vals[2] = cnt;
+        }
+    }
+    __syncthreads();
+    const int bin = (int)x.sh->vals[0];
+    target = x.sh->vals[1];
+    in_bin = x.sh->vals[2];
+    // red_* of this level stay untouched until after the next cluster barrier (start of the next level / gather)
+    return bin;
+}
+
+constexpr int GATHER_CAP = MAX_TOPK;          // elements CTA 0 can sort
+
+// Selection inside `base`:
+//   by_mass == false: the cut of the `need`-th largest element (1 <= need <= count inside base)
 //   by_mass == true : the cut of the smallest ranking prefix whose mass reaches p * (mass inside base)
-__device__ Cut radix_select(ExactCtx &x, const Cut &base, bool by_mass, unsigned long long need, float p) {
-    uint32_t prefix = 0;
-    int pbits = 0;
-    unsigned long long target = need;
-    unsigned long long ties = 0;
-    for (int pass = 0; pass < 3; ++pass) {
-        const int nb = (pass < 2) ? 11 : 10;
-        const int nbins = 1 << nb;
-        const int shift = 32 - pbits - nb;
-        for (int i = x.tid; i < HBINS; i += EX_THREADS) { x.hcnt[i] = 0; x.hmass[i] = 0ull; }
+// Levels: two histograms uniform in (M - y) (1/32 then 2^-16 wide), which spread any
+// smooth logit distribution over many bins; then the few elements of the crossing bin
+// are gathered into CTA 0 and sorted.  Bins too crowded for that (massive ties) are
+// resolved by three more levels over the key bits and an ordered tie count.
+__device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned long long need, float p,
+                          unsigned long long *sortbuf) {
+    unsigned long long target = need, in_bin = 0;
+    const float Mf = x.Mf;
+    auto dig_a = [&](uint32_t key) -> int {
+        float t = fminf(__fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f), 2047.0f);
+        return 2047 - (int)t;
+    };
+    const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin);
+    auto dig_b = [&](uint32_t key) -> int {
+        float t = __fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f);
+        int aa = (int)fminf(t, 2047.0f);
+        if (2047 - aa != a) return -1;
+        float f = fminf(__fmul_rn(__fsub_rn(t, (float)aa), 2048.0f), 2047.0f);
+        return 2047 - (int)f;
+    };
+    int b = -1;
+    if (in_bin > (unsigned long long)GATHER_CAP) b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin);
+    auto in_range = [&](uint32_t key) -> bool {
+        if (dig_a(key) != a) return false;
+        return b < 0 || dig_b(key) == b;
+    };
+    if (in_bin <= (unsigned long long)GATHER_CAP) {
+        // gather the bin into CTA 0, sort it there, pick the element that completes the target
+        if (x.tid == 0) x.sh->ucount = 0;
         __syncthreads();
+        unsigned long long cnt = 0;
         for (int i = x.tid; i < x.len; i += EX_THREADS) {
             uint32_t key = x.keys[i];
-            if (pbits && (key >> (32 - pbits)) != prefix) continue;
-            if (!member(base, key, x.lo + i)) continue;
-            uint32_t bin = (key >> shift) & (nbins - 1);
-            atomicAdd(&x.hcnt[bin], 1u);
-            if (by_mass) atomicAdd(&x.hmass[bin], qweight(key, x.Mf));
+            cnt += (member(base, key, x.lo + i) && in_range(key)) ? 1 : 0;
+        }
+        cnt = block_sum_u64(x, cnt);
+        unsigned long long v[XV] = {cnt, 0, 0, 0};
+        unsigned long long all[CL][XV];
+        allgather(x, v, all);
+        unsigned int off = 0, n = 0;
+        for (int r = 0; r < CL; ++r) { if (r < x.rank) off += (unsigned int)all[r][0]; n += (unsigned int)all[r][0]; }
+        unsigned long long *dst = cg::this_cluster().map_shared_rank(sortbuf, 0);
+        for (int i = x.tid; i < x.len; i += EX_THREADS) {
+            uint32_t key = x.keys[i];
+            if (member(base, key, x.lo + i) && in_range(key)) {
+                unsigned int pos = off + atomicAdd(&x.sh->ucount, 1u);
+                if (pos < (unsigned int)GATHER_CAP) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+            }
         }
         cg::this_cluster().sync();
-        // CTA r reduces bins [r*bpr, (r+1)*bpr) over the cluster
-        const int bpr = nbins / CL;
-        unsigned long long sc = 0, sm = 0;
-        if (x.tid < bpr) {
-            int bin = x.rank * bpr + x.tid;
-            unsigned int cc = 0;
-            unsigned long long mm = 0;
-            for (int r = 0; r < CL; ++r) {
-                cc += *cg::this_cluster().map_shared_rank(&x.hcnt[bin], r);
-                if (by_mass) mm += *cg::this_cluster().map_shared_rank(&x.hmass[bin], r);
-            }
-            x.sh->red_cnt[x.tid] = cc;
-            x.sh->red_mass[x.tid] = mm;
-            sc = cc; sm = mm;
-        }
-        sc = block_sum_u64(x, sc);
-        sm = block_sum_u64(x, sm);
-        unsigned long long v[XV] = {sc, sm, 0, 0};
-        unsigned long long all[CL][XV];
-        allgather(x, v, all);                 // every remote histogram read precedes this barrier
-        if (by_mass && pass == 0) {
-            unsigned long long Zq = 0;
-            for (int r = 0; r < CL; ++r) Zq += all[r][1];
-            double t = ceil((double)p * (double)Zq);
-            target = (unsigned long long)t;
-            if (target > Zq) target = Zq;
-            if (target < 1) target = 1;
-        }
-        // segment (CTA) holding the crossing, scanning from the largest keys
-        int seg = -1;
-        unsigned long long cum = 0;
-        for (int r = CL - 1; r >= 0; --r) {
-            unsigned long long s = by_mass ? all[r][1] : all[r][0];
-            if (cum + s >= target) { seg = r; break; }
-            cum += s;
-        }
-        if (seg < 0) {                             // target beyond the total: cannot happen for valid calls
-            seg = 0;
-            cum -= by_mass ? all[0][1] : all[0][0];
-            target = cum + (by_mass ? all[0][1] : all[0][0]);
-        }
         unsigned long long v2[XV] = {0, 0, 0, 0};
-        if (x.rank == seg && x.tid == 0) {
-            unsigned long long c2 = cum;
-            int b = 0;
-            for (int t = bpr - 1; t >= 0; --t) {
-                unsigned long long s = by_mass ? x.sh->red_mass[t] : (unsigned long long)x.sh->red_cnt[t];
-                if (c2 + s >= target) { b = t; break; }
-                c2 += s;
+        if (x.rank == 0) {
+            const int nn = (int)min(n, (unsigned int)GATHER_CAP);
+            const int m = next_pow2(nn);
+            for (int i = nn + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
+            __syncthreads();
+            bitonic_sort_desc<EX_THREADS>(sortbuf, m, x.tid);
+            // running count / mass in ranking order; each thread owns a contiguous chunk of the sorted list
+            const int chunk = (nn + EX_THREADS - 1) / EX_THREADS;
+            const int lo = min(nn, x.tid * chunk), hi = min(nn, lo + chunk);
+            unsigned long long mine = 0;
+            for (int j = lo; j < hi; ++j) mine += by_mass ? qweight((uint32_t)(sortbuf[j] >> 32), Mf) : 1ull;
+            // exclusive prefix over threads (warp scan, then warp totals)
+            unsigned long long incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (x.lane >= o) incl += up;
             }
-            x.sh->vals[0] = (unsigned long long)(seg * bpr + b);
-            x.sh->vals[1] = target > c2 ? target - c2 : 1ull;   // still needed inside the bin
-            x.sh->vals[2] = x.sh->red_cnt[b];
+            __syncthreads();
+            if (x.lane == 31) x.sh->wtot[x.warp] = incl;
+            __syncthreads();
+            unsigned long long woff = 0;
+            for (int w = 0; w < x.warp; ++w) woff += x.sh->wtot[w];
+            unsigned long long run = woff + incl - mine;
+            if (x.tid == 0) x.sh->flag = nn - 1;
+            __syncthreads();
+            for (int j = lo; j < hi; ++j) {
+                unsigned long long wj = by_mass ? qweight((uint32_t)(sortbuf[j] >> 32), Mf) : 1ull;
+                if (run < target && run + wj >= target) x.sh->flag = j;
+                run += wj;
+            }
+            __syncthreads();
+            v2[0] = sortbuf[max(0, x.sh->flag)];
         }
-        __syncthreads();
-        if (x.rank == seg) { v2[0] = x.sh->vals[0]; v2[1] = x.sh->vals[1]; v2[2] = x.sh->vals[2]; }
         allgather(x, v2, all);
-        prefix = (prefix << nb) | (uint32_t)all[seg][0];
-        target = all[seg][1];
-        ties = all[seg][2];
+        Cut c;
+        c.v = (uint32_t)(all[0][0] >> 32);
+        c.idx = (int)(~(uint32_t)all[0][0]);
+        return c;
+    }
+    // crowded bin: descend over the key bits of the elements in range
+    uint32_t prefix = 0;
+    int pbits = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+        const int nb = (pass < 2) ? 11 : 10;
+        const int shift = 32 - pbits - nb;
+        auto dig_k = [&](uint32_t key) -> int {
+            if (pbits && (key >> (32 - pbits)) != prefix) return -1;
+            if (!in_range(key)) return -1;
+            return (int)((key >> shift) & ((1u << nb) - 1u));
+        };
+        const int d = hist_level(x, base, by_mass, false, p, 1 << nb, dig_k, target, in_bin);
+        prefix = (prefix << nb) | (uint32_t)d;
         pbits += nb;
     }
     // prefix is the boundary value; `target` of its ties (by count) or enough of them to reach the mass
     unsigned long long r = target;
     if (by_mass) {
-        unsigned long long qw = qweight(prefix, x.Mf);
+        unsigned long long qw = qweight(prefix, Mf);
         r = qw ? (target + qw - 1) / qw : 1;
     }
     if (r < 1) r = 1;
-    if (r > ties) r = ties;
+    if (r > in_bin) r = in_bin;
     const uint32_t v = prefix;
     unsigned long long tot;
     int idx = ordered_cross<unsigned long long>(
@@ -395,7 +551,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     if (P.op == OP_TOPK) {
         Cut all_cut; all_cut.v = 0; all_cut.idx = -1;
         Cut cut = all_cut;
-        if (c.k < V) cut = radix_select(x, all_cut, false, (unsigned long long)c.k, 1.0f);
+        if (c.k < V) cut = select_cut(x, all_cut, false, (unsigned long long)c.k, 1.0f, sortbuf);
         // compact the members into CTA 0's sort buffer
         if (x.tid == 0) x.sh->ucount = 0;
         __syncthreads();
@@ -411,12 +567,12 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
             uint32_t key = x.keys[i];
             if (member(cut, key, x.lo + i)) {
                 unsigned int pos = off + atomicAdd(&x.sh->ucount, 1u);
-                if (pos < (unsigned int)KFAST_TOPK) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+                if (pos < (unsigned int)MAX_TOPK) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
             }
         }
         cg::this_cluster().sync();
         if (x.rank == 0) {
-            const int n = min(c.k, KFAST_TOPK);
+            const int n = min(c.k, MAX_TOPK);
             const int m = next_pow2(n);
             for (int i = n + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
             __syncthreads();
@@ -438,10 +594,10 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         return;
     }
     Cut cut; cut.v = KEY_NEG_INF; cut.idx = -1;            // every finite element
-    if (c.k > 0 && (unsigned long long)c.k < Nf) cut = radix_select(x, cut, false, (unsigned long long)c.k, 1.0f);
+    if (c.k > 0 && (unsigned long long)c.k < Nf) cut = select_cut(x, cut, false, (unsigned long long)c.k, 1.0f, sortbuf);
     const Cut cut_k = cut;
     if (c.z & M_TOP_P) {
-        Cut cp = radix_select(x, cut_k, true, 0ull, c.p);
+        Cut cp = select_cut(x, cut_k, true, 0ull, c.p, sortbuf);
         if (tighter(cp, cut)) cut = cp;
     }
     if (c.z & M_MIN_P) {
@@ -538,11 +694,11 @@ sonic_exact_kernel(const KParams P) {
     x.tid = threadIdx.x; x.lane = x.tid & 31; x.warp = x.tid >> 5;
     x.phase = 0;
     x.keys = reinterpret_cast<uint32_t *>(smem_raw);
-    x.hmass = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4);
-    x.hcnt = reinterpret_cast<unsigned int *>(smem_raw + SLICE_MAX * 4 + HBINS * 8);
-    x.sh = reinterpret_cast<ExactShared *>(smem_raw + SLICE_MAX * 4 + HBINS * 12);
-    unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 12 + 8192);
-    uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 12 + 8192 + KFAST_TOPK * 8);
+    x.hcnt = reinterpret_cast<unsigned int *>(smem_raw + SLICE_MAX * 4);
+    x.hm0 = x.hcnt + HBINS; x.hm1 = x.hcnt + 2 * HBINS; x.hm2 = x.hcnt + 3 * HBINS;
+    x.sh = reinterpret_cast<ExactShared *>(smem_raw + SLICE_MAX * 4 + HBINS * 16);
+    unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192);
+    uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8);
 
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;

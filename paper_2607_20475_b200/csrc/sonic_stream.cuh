@@ -1,11 +1,11 @@
 // Streaming kernel: reads every logit of the rows it owns exactly once, applies
 // the logit-processing prologue, and reduces each 8192-element tile either to
 // an argmax (greedy rows) or to the complete set of elements above a tile
-// cutoff (top-k rows).  The CTA that finishes a row's last tile merges the row
-// (global top-k, truncation epilogue, token selection) while other CTAs keep
-// streaming.  Corresponds to the paper's Stage 1 and Stage 2 (Algorithms
-// "Stage 1: Tile-Local Reduction Kernel" and "Stage 2: Cross-Tile Merge and
-// Selection Kernel") fused into one launch; the selection itself is ours.
+// cutoff (top-k rows), written to the tile's own slot of the workspace without
+// atomics.  The merge kernel (one CTA per row) then finishes the row: global
+// top-k, truncation epilogue, token selection.  The two correspond to the
+// paper's Algorithms "Stage 1: Tile-Local Reduction Kernel" and "Stage 2:
+// Cross-Tile Merge and Selection Kernel"; the selection itself is ours.
 //
 // Exactness: a tile's cutoff t is the minimum of G group maxima, so at least G
 // of its elements are >= t, and the tile emits EVERY finite element >= t.  With
@@ -142,6 +142,8 @@ __device__ __forceinline__ void patch_tile(const KParams &P, const RowCfg &c, in
 
 struct MergeShared {
     int count;
+    int tcnt[MAX_TILES + 1];                   // exclusive prefix of the tiles' candidate counts
+    unsigned int tkey;
     int n_p, n_m, pick;
     int found;
     double scratch[STREAM_THREADS];
@@ -162,33 +164,49 @@ __device__ __forceinline__ void emit_row(const KParams &P, const RowCfg &c, int 
     }
 }
 
-// Row merge for top-k class rows, executed by the CTA that finished the row's
-// last tile.  buf is SORT_CAP 64-bit words of shared memory.  Returns false if
-// the candidates cannot prove the row's answer.
-__device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, RowState *rs, unsigned long long *buf,
-                               MergeShared &sh, int tid) {
-    const unsigned int ncand = __ldcg(&rs->ncand);
-    const unsigned int tkey = __ldcg(&rs->tkey);
-    if (ncand > CAND_CAP) return false;
+// Row merge for top-k class rows, run by the CTA that finished the row's last
+// tile.  buf is MERGE_CAP 64-bit words of shared memory (the staging tile,
+// free by then).  Returns false if the candidates cannot prove the row's answer.
+__device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int tiles,
+                               unsigned long long *buf, MergeShared &sh, int tid) {
+    const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
+    const TileRec *rec = P.tiles + (size_t)row * MAX_TILES;
+    // tile records: one thread per tile, then a serial prefix over at most 32 entries
+    if (tid == 0) { sh.count = 0; sh.tkey = 0; sh.found = 0; }
+    __syncthreads();
+    if (tid < tiles) {
+        const unsigned int cnt = __ldcg(&rec[tid].cnt);
+        sh.tcnt[tid + 1] = (int)cnt;
+        atomicMax(&sh.tkey, __ldcg(&rec[tid].tkey));
+        if (cnt > (unsigned int)cap_t) sh.found = 1;     // a tile overflowed its slot
+    }
+    __syncthreads();
+    if (sh.found) return false;
+    if (tid == 0) {
+        sh.tcnt[0] = 0;
+        for (int t = 0; t < tiles; ++t) sh.tcnt[t + 1] += sh.tcnt[t];
+    }
+    __syncthreads();
+    const unsigned int tkey = sh.tkey;
     const bool complete = (tkey == KEY_NEG_INF);
     const bool strict = c.temp && !complete;            // keys are compared after the temperature division
     const uint32_t tykey = c.temp ? okey(__fdiv_rn(unkey(tkey), c.tau)) : tkey;
-    if (tid == 0) sh.count = 0;
-    __syncthreads();
-    const unsigned long long *cand = P.cand + (size_t)row * CAND_CAP;
-    for (unsigned int i = tid; i < ncand; i += STREAM_THREADS) {
-        unsigned long long cd = __ldcg(cand + i);
+    const int total = sh.tcnt[tiles];
+    for (int j = tid; j < total; j += STREAM_THREADS) {
+        int t = 0;
+        while (sh.tcnt[t + 1] <= j) ++t;
+        unsigned long long cd = __ldcg(P.cand + (size_t)row * CAND_CAP + (size_t)t * cap_t + (j - sh.tcnt[t]));
         uint32_t zk = (uint32_t)(cd >> 32);
         if (zk < tkey) continue;
         uint32_t yk = zk;
         if (c.temp) yk = okey(__fdiv_rn(unkey(zk), c.tau));
         if (strict && yk <= tykey) continue;
         int pos = atomicAdd(&sh.count, 1);
-        if (pos < SORT_CAP) buf[pos] = ((unsigned long long)yk << 32) | (uint32_t)cd;
+        if (pos < MERGE_CAP) buf[pos] = ((unsigned long long)yk << 32) | (uint32_t)cd;
     }
     __syncthreads();
     const int Pn = sh.count;
-    if (Pn > SORT_CAP) return false;
+    if (Pn > MERGE_CAP) return false;
     int n;
     if (Pn >= c.k) n = c.k;
     else if (complete && P.op != OP_TOPK) n = Pn;
@@ -210,14 +228,14 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, RowSt
         if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN, 0, 0.0f);
         return true;
     }
-    // shared-memory layout after the sort (n <= 2048):
-    //   buf[0, 2048)      sorted keys (value key << 32 | ~index)
-    //   w  [2048, 4096)   weights exp(y - M) in ranking order
-    //   cs [4096, 6144)   cumulative sums (ranking order), later residual / CDF in index order
-    //   ik [6144, 8192)   (~index << 32 | ranking position), sorted descending = index ascending
-    double *w = reinterpret_cast<double *>(buf + 2048);
-    double *cs = reinterpret_cast<double *>(buf + 4096);
-    unsigned long long *ik = buf + 6144;
+    // shared-memory layout after the sort (n <= KFAST_SAMPLE = MERGE_CAP / 4):
+    //   buf[0, n)     sorted keys (value key << 32 | ~index)
+    //   w             weights exp(y - M) in ranking order
+    //   cs            cumulative sums (ranking order), later residual / CDF in index order
+    //   ik            (~index << 32 | ranking position), sorted descending = index ascending
+    double *w = reinterpret_cast<double *>(buf + KFAST_SAMPLE);
+    double *cs = reinterpret_cast<double *>(buf + 2 * KFAST_SAMPLE);
+    unsigned long long *ik = buf + 3 * KFAST_SAMPLE;
     const double M = (double)unkey((uint32_t)(buf[0] >> 32));
     for (int j = tid; j < n; j += STREAM_THREADS) {
         double y = (double)unkey((uint32_t)(buf[j] >> 32));
@@ -306,10 +324,12 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, RowSt
 }
 
 template <int DT>
-__global__ void __launch_bounds__(STREAM_THREADS)
+__global__ void __launch_bounds__(STREAM_THREADS, 4)
 sonic_stream_kernel(const KParams P) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ __align__(16) float s_tile[CTA_TILE];
     __shared__ float s_tw[STREAM_WARPS];
+    __shared__ int s_wcnt[STREAM_WARPS];
+    __shared__ unsigned long long s_best[STREAM_WARPS];
     __shared__ int s_last;
     __shared__ MergeShared s_merge;
 
@@ -317,15 +337,16 @@ sonic_stream_kernel(const KParams P) {
     const int tile = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const RowCfg c = load_cfg(P, row);
-    if (c.cls == CLS_EXACT) return;
     RowState *rs = P.rs + row;
+    if (c.cls == CLS_EXACT) return;
+    TileRec *rec = P.tiles + (size_t)row * MAX_TILES + tile;
     const int tile_base = tile * CTA_TILE;
     const int wbase = tile_base + warp * WARP_TILE;
 
     float e[EPL];
     load_warp_tile<DT>(P, c, row, wbase, lane, e);
     if (c.hist_len > 0 || c.bias_len > 0)
-        patch_tile<DT>(P, c, tile_base, reinterpret_cast<float *>(smem_raw), warp, lane, tid, tile == 0, rs, e);
+        patch_tile<DT>(P, c, tile_base, s_tile, warp, lane, tid, tile == 0, rs, e);
     if (c.div_all) {
 #pragma unroll
         for (int s = 0; s < EPL; ++s) e[s] = __fdiv_rn(e[s], c.tau);
@@ -350,6 +371,7 @@ sonic_stream_kernel(const KParams P) {
         float wm = lm;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xFFFFFFFFu, wm, off));
+        unsigned long long key = 0ull;
         if (wm > -CUDART_INF_F) {
             int best = 0x7FFFFFFF;
             if (lm == wm) {
@@ -359,111 +381,129 @@ sonic_stream_kernel(const KParams P) {
             }
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) best = min(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
-            if (lane == 0)
-                atomicMax(&rs->best, ((unsigned long long)okey(wm) << 32) | (uint32_t)(~(uint32_t)best));
+            key = ((unsigned long long)okey(wm) << 32) | (uint32_t)(~(uint32_t)best);
+        }
+        if (lane == 0) s_best[warp] = key;
+        __syncthreads();
+        if (tid == 0) {
+            unsigned long long b = s_best[0];
+#pragma unroll
+            for (int w = 1; w < STREAM_WARPS; ++w) b = max(b, s_best[w]);
+            rec->best = b;
         }
     } else {
-        // tile cutoff: minimum over G groups of the group maximum
-        float g;
-        const int G = c.G;
-        if (G == 0) {
-            g = -CUDART_INF_F;
-        } else {
-            const int L = (G >= 32) ? 1 : (32 / G);           // lanes per group
-            g = (G == 64) ? fminf(h0, h1) : lm;
+    // tile cutoff: minimum over G groups of the group maximum, then the largest over the CTA's warp tiles
+    float g;
+    const int G = c.G;
+    if (G == 0) {
+        g = -CUDART_INF_F;
+    } else {
+        const int L = (G >= 32) ? 1 : (32 / G);           // lanes per group
+        g = (G == 64) ? fminf(h0, h1) : lm;
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                float o = __shfl_xor_sync(0xFFFFFFFFu, g, off);
-                g = (off < L) ? fmaxf(g, o) : fminf(g, o);
-            }
+        for (int off = 1; off < 32; off <<= 1) {
+            float o = __shfl_xor_sync(0xFFFFFFFFu, g, off);
+            g = (off < L) ? fmaxf(g, o) : fminf(g, o);
         }
-        if (lane == 0) s_tw[warp] = g;
-        __syncthreads();
-        float t = s_tw[0];
+    }
+    if (lane == 0) s_tw[warp] = g;
+    __syncthreads();
+    float t = s_tw[0];
 #pragma unroll
-        for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, s_tw[w]);
-        // emit every finite element >= t
-        int cnt = 0;
+    for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, s_tw[w]);
+    // every finite element >= t goes to the tile's candidate slot
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+        if (mv[j] >= t) {
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) cnt += (e[j * VEC + q] >= t && e[j * VEC + q] > -CUDART_INF_F) ? 1 : 0;
+        }
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += o;
+    }
+    if (lane == 31) s_wcnt[warp] = incl;
+    __syncthreads();
+    int base = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < STREAM_WARPS; ++w) {
+        if (w == warp) base = total;
+        total += s_wcnt[w];
+    }
+    const int cap_t = (int)(CAND_CAP / gridDim.x);
+    if (cnt > 0 && total <= cap_t) {
+        unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + (size_t)tile * cap_t + base + (incl - cnt);
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
             if (mv[j] >= t) {
 #pragma unroll
-                for (int q = 0; q < VEC; ++q) cnt += (e[j * VEC + q] >= t && e[j * VEC + q] > -CUDART_INF_F) ? 1 : 0;
-            }
-        }
-        int incl = cnt;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-            if (lane >= off) incl += o;
-        }
-        const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-        unsigned int base = 0;
-        if (lane == 0 && total > 0) base = atomicAdd(&rs->ncand, (unsigned int)total);
-        base = __shfl_sync(0xFFFFFFFFu, base, 0);
-        if (cnt > 0 && base + (unsigned int)total <= CAND_CAP) {
-            unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + base + (incl - cnt);
-#pragma unroll
-            for (int j = 0; j < NV; ++j) {
-                if (mv[j] >= t) {
-#pragma unroll
-                    for (int q = 0; q < VEC; ++q) {
-                        float v = e[j * VEC + q];
-                        if (v >= t && v > -CUDART_INF_F) {
-                            int idx = slot_index<DT>(wbase, lane, j * VEC + q);
-                            *dst++ = ((unsigned long long)okey(v) << 32) | (uint32_t)(~(uint32_t)idx);
-                        }
+                for (int q = 0; q < VEC; ++q) {
+                    float v = e[j * VEC + q];
+                    if (v >= t && v > -CUDART_INF_F) {
+                        int idx = slot_index<DT>(wbase, lane, j * VEC + q);
+                        *dst++ = ((unsigned long long)okey(v) << 32) | (uint32_t)(~(uint32_t)idx);
                     }
                 }
             }
         }
-        if (tid == 0) atomicMax(&rs->tkey, okey(t));
+    }
+    if (tid == 0) { rec->cnt = (unsigned int)total; rec->tkey = okey(t); }
     }
 
-    // ---- last tile of the row merges it
+    // ---- the CTA that finishes the row's last tile merges the row while others keep streaming
     __threadfence();
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        unsigned int done = atomicAdd(&rs->ticket, 1u);
+        const unsigned int done = atomicAdd(&rs->ticket, 1u);
         s_last = (done == gridDim.x - 1) ? 1 : 0;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-
+    const int tiles = gridDim.x;
+    const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
     const unsigned int status = __ldcg(&rs->status);
     bool ok = true;
     if (c.bad || (status & ST_BADID)) {
         if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_BADPARAM, 0, 0.0f);
     } else if (c.cls == CLS_GREEDY) {
-        if (tid == 0) {
-            unsigned long long best = __ldcg(&rs->best);
-            if (P.op == OP_TOPK) {
-                // k == 1: a row of nothing but -inf still has a first element
-                P.out_vals[row] = best ? unkey((uint32_t)(best >> 32)) : -CUDART_INF_F;
-                P.out_idx[row] = best ? (int)(~(uint32_t)best) : 0;
-            } else if (best == 0ull) {
-                emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN, 0, 0.0f);
-            } else {
-                int token = (int)(~(uint32_t)best);
-                uint32_t flags = 0;
-                float pd = 0.0f;
-                if (P.op == OP_VERIFY && c.l < P.K) {
-                    bool acc = P.draft_tokens[(size_t)c.b * P.K + c.l] == token;
-                    if (acc) { flags |= F_ACCEPT; pd = 1.0f; }
+        if (tid < 32) {
+            unsigned long long best = (tid < tiles) ? __ldcg(&recs[tid].best) : 0ull;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
+            if (tid == 0) {
+                if (P.op == OP_TOPK) {
+                    // k == 1: a row of nothing but -inf still has a first element
+                    P.out_vals[row] = best ? unkey((uint32_t)(best >> 32)) : -CUDART_INF_F;
+                    P.out_idx[row] = best ? (int)(~(uint32_t)best) : 0;
+                } else if (best == 0ull) {
+                    emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN, 0, 0.0f);
+                } else {
+                    int token = (int)(~(uint32_t)best);
+                    uint32_t flags = 0;
+                    float pd = 0.0f;
+                    if (P.op == OP_VERIFY && c.l < P.K) {
+                        bool acc = P.draft_tokens[(size_t)c.b * P.K + c.l] == token;
+                        if (acc) { flags |= F_ACCEPT; pd = 1.0f; }
+                    }
+                    emit_row(P, c, row, token, 1.0f, flags, 1, pd);
                 }
-                emit_row(P, c, row, token, 1.0f, flags, 1, pd);
             }
         }
     } else {
-        ok = merge_topk_row(P, c, row, rs, reinterpret_cast<unsigned long long *>(smem_raw), s_merge, tid);
+        ok = merge_topk_row(P, c, row, tiles, reinterpret_cast<unsigned long long *>(s_tile), s_merge, tid);
     }
     __syncthreads();
     if (tid == 0) {
-        rs->ticket = 0; rs->ncand = 0; rs->tkey = 0; rs->best = 0ull;
+        rs->ticket = 0;
         rs->status = ok ? 0u : ST_FAILED;
     }
 }
 
 }  // namespace sonic
+
