@@ -133,6 +133,30 @@ int sonic_verify(const sonic_verify_args *args, void *workspace, size_t workspac
 int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, int k,
                float *out_vals, int32_t *out_idx, void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * sonic_topk without a caller-provided workspace and without any allocation.
+ * (The paper has no counterpart: this entry point exists for callers of this library
+ * that are not allowed to allocate device memory -- plugins handed a fixed memory
+ * budget by their host engine, processes whose device memory pool was sized once at
+ * start-up, and latency-critical serving loops in which a cudaMalloc would synchronise
+ * the whole device.)
+ *
+ * Same inputs, outputs and results as sonic_topk, for at most SONIC_STATIC_MAX_ROWS rows
+ * per call; larger B is rejected with SONIC_ESHAPE.  The scratch memory is a fixed array
+ * of about 2.1 MB inside the library image (SONIC_STATIC_MAX_ROWS rows of candidate
+ * slots and control words); every GPU that loads the library holds it until the process
+ * exits.  The function calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * The first call on each device resolves the array's device address and configures the
+ * kernels; that first call should come before any stream capture is begun.  All calls on a device share
+ * the one array, which keeps the contents of the previous call: each call first clears
+ * the control words it needs at zero (a memset enqueued on `stream`), and two calls that
+ * overlap on the device (different streams, or graphs replayed concurrently) race on it.
+ */
+#define SONIC_STATIC_MAX_ROWS 8
+int sonic_topk_static(const void *logits, int dtype, int B, int V, int64_t row_stride, int k,
+                      float *out_vals, int32_t *out_idx, void *stream);
+
 /* Text of the calling thread's last error ("" if none).  Never NULL. */
 const char *sonic_last_error(void);
 

@@ -71,6 +71,9 @@ def lib():
         L.sonic_topk.restype = C.c_int
         L.sonic_topk.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_size_t, C.c_void_p]
+        L.sonic_topk_static.restype = C.c_int
+        L.sonic_topk_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_void_p,
+                                        C.c_void_p, C.c_void_p]
         L.sonic_last_error.restype = C.c_char_p
         _lib = L
     return _lib
@@ -122,6 +125,17 @@ def sonic_topk(logits: torch.Tensor, dtype: int, B: int, V: int, row_stride: int
                out_vals: torch.Tensor, out_idx: torch.Tensor, ws: torch.Tensor):
     _check(lib().sonic_topk(logits.data_ptr(), dtype, B, V, row_stride, k, out_vals.data_ptr(), out_idx.data_ptr(),
                             ws.data_ptr(), ws.numel(), _stream()))
+
+
+STATIC_MAX_ROWS = 8
+
+
+def sonic_topk_static(logits: torch.Tensor, dtype: int, B: int, V: int, row_stride: int, k: int,
+                      out_vals: torch.Tensor, out_idx: torch.Tensor):
+    """sonic_topk for callers that cannot allocate: no workspace argument, at most STATIC_MAX_ROWS rows.
+    The scratch is a fixed array inside the library; calls on one device must not overlap."""
+    _check(lib().sonic_topk_static(logits.data_ptr(), dtype, B, V, row_stride, k, out_vals.data_ptr(),
+                                   out_idx.data_ptr(), _stream()))
 
 
 # --------------------------------------------------------------------------- device-side holders

@@ -242,6 +242,52 @@ int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, 
     return launch_all(P, workspace, workspace_bytes, (cudaStream_t)stream, B);
 }
 
+// ---------------------------------------------------------------- no-allocation variant
+// Scratch of sonic_topk_static: a workspace for SONIC_STATIC_MAX_ROWS rows that lives in
+// the library image.  In host code this name is only a stand-in for the symbol; the device
+// address the kernels need comes from cudaGetSymbolAddress (below), never from `&`.
+static __device__ __align__(256) unsigned char g_static_workspace[WS_HEADER + (size_t)SONIC_STATIC_MAX_ROWS * WS_ROW];
+
+static int static_workspace_address(void **out) {
+    static std::once_flag once[64];
+    static cudaError_t result[64];
+    static void *address[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return fail(SONIC_EINVAL, "device ordinal out of range");
+    std::call_once(once[dev], [&] {          // once per device, with that device current
+        void *p = nullptr;
+        result[dev] = cudaGetSymbolAddress(&p, g_static_workspace);
+        address[dev] = p;
+    });
+    if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "cudaGetSymbolAddress");
+    *out = address[dev];
+    return SONIC_OK;
+}
+
+int sonic_topk_static(const void *logits, int dtype, int B, int V, int64_t row_stride, int k,
+                      float *out_vals, int32_t *out_idx, void *stream) {
+    int rc = check_logits(logits, dtype, B, V, row_stride);
+    if (rc != SONIC_OK) return rc;
+    if (B > SONIC_STATIC_MAX_ROWS) return fail(SONIC_ESHAPE, "sonic_topk_static handles at most SONIC_STATIC_MAX_ROWS rows per call");
+    if (k < 1 || k > V || k > SONIC_MAX_TOPK) return fail(SONIC_ESHAPE, "k outside 1..min(V, SONIC_MAX_TOPK)");
+    if (!out_vals || !out_idx) return fail(SONIC_EINVAL, "an output pointer is NULL");
+    void *ws = nullptr;
+    rc = static_workspace_address(&ws);
+    if (rc != SONIC_OK) return rc;
+    const size_t bytes = WS_HEADER + (size_t)SONIC_STATIC_MAX_ROWS * WS_ROW;
+    // the array keeps whatever the previous call left: the control words must start at zero
+    cudaError_t e = cudaMemsetAsync(ws, 0, WS_HEADER + (size_t)SONIC_STATIC_MAX_ROWS * WS_ROW_CTRL, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaMemsetAsync");
+    KParams P;
+    memset(&P, 0, sizeof(P));
+    P.op = OP_TOPK;
+    P.rows = B; P.V = V; P.dtype = dtype; P.logits = logits; P.row_stride = row_stride; P.ktop = k;
+    P.out_vals = out_vals; P.out_idx = out_idx;
+    return launch_all(P, ws, bytes, (cudaStream_t)stream, B);
+}
+
 const char *sonic_last_error(void) { return g_err; }
 
 }  // extern "C"
