@@ -42,6 +42,8 @@ __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
 }
 
 constexpr size_t WS_HEADER = 256;
+constexpr int STREAM_SMEM_F32 = VecTraits<0>::NSTAGE * CTA_TILE * 4 + (int)sizeof(StreamShared<0>);
+constexpr int STREAM_SMEM_BF16 = VecTraits<1>::NSTAGE * CTA_TILE * 2 + CTA_TILE * 4 + (int)sizeof(StreamShared<1>);
 constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8 + 8192;
 
 static thread_local char g_err[256] = "";
@@ -61,8 +63,9 @@ constexpr size_t WS_ROW = WS_ROW_CTRL + (size_t)CAND_CAP * 8;
 static size_t ws_bytes_for(int rows) { return WS_HEADER + (size_t)rows * WS_ROW; }
 
 static int g_max_clusters[64];      // co-resident 8-CTA clusters of the exact kernel, per device
+static int g_sm_count[64];
 
-static int configure_once(int *max_clusters) {
+static int configure_once(int *max_clusters, int *sm_count) {
     static std::once_flag once[64];
     static cudaError_t result[64];
     int dev = 0;
@@ -74,6 +77,9 @@ static int configure_once(int *max_clusters) {
         auto set = [&](const void *f, int bytes) {
             if (r == cudaSuccess) r = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         };
+        set((const void *)sonic_stream_kernel<0>, STREAM_SMEM_F32);
+        set((const void *)sonic_stream_kernel<1>, STREAM_SMEM_BF16);
+        if (r == cudaSuccess) r = cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
         set((const void *)sonic_exact_kernel<0>, EXACT_SMEM);
         set((const void *)sonic_exact_kernel<1>, EXACT_SMEM);
         int n = 0;
@@ -96,6 +102,7 @@ static int configure_once(int *max_clusters) {
     if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "kernel configuration");
     if (g_max_clusters[dev] < 1) return fail(SONIC_ECUDA, "no 8-CTA cluster of the exact kernel fits on this device");
     *max_clusters = g_max_clusters[dev];
+    *sm_count = g_sm_count[dev] > 0 ? g_sm_count[dev] : 1;
     return SONIC_OK;
 }
 
@@ -103,21 +110,25 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
     if (ws_bytes < ws_bytes_for(P.rows)) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows");
-    int max_clusters = 0;
-    int rc = configure_once(&max_clusters);
+    int max_clusters = 0, sm_count = 1;
+    int rc = configure_once(&max_clusters, &sm_count);
     if (rc != SONIC_OK) return rc;
     // the layout depends on the row capacity the workspace was sized for, recovered from its size
     const size_t cap_rows = (ws_bytes - WS_HEADER) / WS_ROW;
     unsigned char *base = reinterpret_cast<unsigned char *>(ws);
+    P.error = reinterpret_cast<unsigned int *>(base);
     P.rs = reinterpret_cast<RowState *>(base + WS_HEADER);
     P.pr = reinterpret_cast<PosResult *>(base + WS_HEADER + cap_rows * sizeof(RowState));
     P.tiles = reinterpret_cast<TileRec *>(base + WS_HEADER + cap_rows * (sizeof(RowState) + sizeof(PosResult)));
     P.cand = reinterpret_cast<unsigned long long *>(base + WS_HEADER + cap_rows * WS_ROW_CTRL);
 
     const int tiles = (P.V + CTA_TILE - 1) / CTA_TILE;
-    dim3 grid1(tiles, P.rows);
-    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_THREADS, 0, st>>>(P);
-    else sonic_stream_kernel<1><<<grid1, STREAM_THREADS, 0, st>>>(P);
+    const long long nitems_ll = (long long)tiles * P.rows;
+    if (nitems_ll > 0x7FFFFFFF) return fail(SONIC_ESHAPE, "rows x tiles too large");
+    const int nitems = (int)nitems_ll;
+    const int grid1 = nitems < sm_count * 2 ? nitems : sm_count * 2;       // persistent: two CTAs per SM
+    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems);
+    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
 

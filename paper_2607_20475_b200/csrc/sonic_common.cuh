@@ -41,6 +41,7 @@ constexpr int CLS_EXACT = 2;                  // full-vocabulary exact path only
 
 constexpr uint32_t ST_FAILED = 0x1;           // streaming path could not prove the row
 constexpr uint32_t ST_BADID = 0x2;            // a list id was out of range
+constexpr unsigned int ERR_TIMEOUT = 0x1;     // workspace header: a bounded mbarrier wait expired
 
 constexpr uint32_t KEY_NEG_INF = 0x007FFFFFu; // okey(-inf)
 
@@ -93,6 +94,7 @@ struct KParams {
     float *out_pdraft;
     float *out_vals;
     int *out_idx;
+    unsigned int *error;                      // workspace header word: ERR_* (sticky)
     RowState *rs;
     TileRec *tiles;
     PosResult *pr;
@@ -229,9 +231,17 @@ __device__ __forceinline__ unsigned long long ldcg_u64(const unsigned long long 
     return __ldcg(p);
 }
 
+// Block-level barriers: the whole CTA, or only the 256 consumer threads of the
+// streaming kernel (named barrier 1; its producer warp never joins).
+struct BlockSync { __device__ __forceinline__ void operator()() const { __syncthreads(); } };
+struct ConsumerSync {
+    __device__ __forceinline__ void operator()() const { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+};
+
 // Descending bitonic sort of m (power of two) 64-bit keys in shared memory.
-template <int THREADS>
+template <int THREADS, typename Sync = BlockSync>
 __device__ __forceinline__ void bitonic_sort_desc(unsigned long long *a, int m, int tid) {
+    Sync sync;
     for (int k2 = 2; k2 <= m; k2 <<= 1) {
         for (int j = k2 >> 1; j > 0; j >>= 1) {
             for (int i = tid; i < (m >> 1); i += THREADS) {
@@ -241,7 +251,7 @@ __device__ __forceinline__ void bitonic_sort_desc(unsigned long long *a, int m, 
                 bool desc = ((lo & k2) == 0);
                 if ((x < y) == desc) { a[lo] = y; a[hi] = x; }
             }
-            __syncthreads();
+            sync();
         }
     }
 }
@@ -254,14 +264,15 @@ __device__ __forceinline__ int next_pow2(int n) {
 
 // Inclusive scan of n doubles in shared memory (in place), THREADS threads,
 // fixed evaluation order (deterministic).  `scratch` holds THREADS doubles.
-template <int THREADS>
+template <int THREADS, typename Sync = BlockSync>
 __device__ __forceinline__ void block_inclusive_scan(double *v, int n, double *scratch, int tid) {
+    Sync sync;
     int chunk = (n + THREADS - 1) / THREADS;
     int lo = tid * chunk, hi = min(lo + chunk, n);
     double s = 0.0;
     for (int i = lo; i < hi; ++i) { s += v[i]; v[i] = s; }
     scratch[tid] = s;
-    __syncthreads();
+    sync();
     if (tid < 32) {
         // serial over 32 segments of THREADS/32 partials each: short and order-fixed
         constexpr int PER = THREADS / 32;
@@ -276,10 +287,10 @@ __device__ __forceinline__ void block_inclusive_scan(double *v, int n, double *s
         double excl = incl - loc;
         for (int i = 0; i < PER; ++i) scratch[tid * PER + i] += excl;
     }
-    __syncthreads();
+    sync();
     double off = scratch[tid];
     for (int i = lo; i < hi; ++i) v[i] += off;
-    __syncthreads();
+    sync();
 }
 
 }  // namespace sonic

@@ -688,7 +688,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
 template <int DT>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
 sonic_exact_kernel(const KParams P) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     ExactCtx x;
     x.rank = (int)cg::this_cluster().block_rank();
     x.tid = threadIdx.x; x.lane = x.tid & 31; x.warp = x.tid >> 5;
