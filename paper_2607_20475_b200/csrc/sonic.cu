@@ -42,6 +42,7 @@ __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
 }
 
 constexpr size_t WS_HEADER = 256;
+constexpr int MERGE_SMEM = MERGE_CAP * 8;
 constexpr int STREAM_SMEM_F32 = VecTraits<0>::NSTAGE * CTA_TILE * 4 + (int)sizeof(StreamShared<0>);
 constexpr int STREAM_SMEM_BF16 = VecTraits<1>::NSTAGE * CTA_TILE * 2 + CTA_TILE * 4 + (int)sizeof(StreamShared<1>);
 constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8 + 8192;
@@ -77,6 +78,7 @@ static int configure_once(int *max_clusters, int *sm_count) {
         auto set = [&](const void *f, int bytes) {
             if (r == cudaSuccess) r = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         };
+        set((const void *)sonic_merge_kernel, MERGE_SMEM);
         set((const void *)sonic_stream_kernel<0>, STREAM_SMEM_F32);
         set((const void *)sonic_stream_kernel<1>, STREAM_SMEM_BF16);
         if (r == cudaSuccess) r = cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
@@ -131,6 +133,9 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
+    sonic_merge_kernel<<<P.rows, MERGE_THREADS, MERGE_SMEM, st>>>(P, tiles);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
 
     dim3 grid2((P.rows < max_clusters ? P.rows : max_clusters) * CL);
     if (P.dtype == SONIC_DTYPE_F32) sonic_exact_kernel<0><<<grid2, EX_THREADS, EXACT_SMEM, st>>>(P);

@@ -29,10 +29,11 @@ constexpr int STREAM_WARPS = STREAM_THREADS / 32;
 constexpr int CTA_TILE = WARP_TILE * STREAM_WARPS;   // 8192
 constexpr int MAX_TILES = (262144 + CTA_TILE - 1) / CTA_TILE;   // 32 tiles at the largest vocabulary
 constexpr uint32_t CAND_CAP = 32768;          // candidate slots per row, divided evenly among the row's tiles
-constexpr int MERGE_CAP = CTA_TILE / 2;       // 64-bit keys the row merge can sort (it reuses the 32 KB staging tile)
-constexpr int KFAST_SAMPLE = MERGE_CAP / 4;   // largest top-k the streaming path finishes for sampling rows (1024)
-constexpr int KFAST_TOPK = MERGE_CAP / 2;     // ... and for sonic_topk rows (2048)
-constexpr int MAX_TOPK = 4096;                // largest k of sonic_topk (beyond KFAST_TOPK: exact kernel)
+constexpr int MERGE_THREADS = 512;
+constexpr int MERGE_CAP = 8192;               // 64-bit keys the row merge can sort (64 KB of shared memory)
+constexpr int KFAST_SAMPLE = MERGE_CAP / 4;   // largest top-k the streaming path finishes for sampling rows (2048)
+constexpr int KFAST_TOPK = MERGE_CAP / 2;     // ... and for sonic_topk rows (4096)
+constexpr int MAX_TOPK = 4096;                // largest k of sonic_topk
 constexpr int MAX_VOCAB = 262144;
 
 constexpr int CLS_GREEDY = 0;                 // streaming path, argmax only
@@ -47,8 +48,7 @@ constexpr uint32_t KEY_NEG_INF = 0x007FFFFFu; // okey(-inf)
 
 struct __align__(16) RowState {
     unsigned int status;                      // ST_*; zero between calls
-    unsigned int ticket;                      // tiles of the row that finished streaming; zero between calls
-    unsigned int pad[2];
+    unsigned int pad[3];
 };
 
 struct __align__(16) TileRec {                // written by the tile's CTA, read by the merge kernel
@@ -124,17 +124,24 @@ __device__ __forceinline__ float unkey(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
 }
 
-// Number of groups per warp tile whose maxima bound the tile cutoff.  With G
-// groups the candidates above the row-wide cutoff number about G * Nw^(1-1/G)
-// for position-independent data (Nw warp tiles per row); pick the smallest
-// power of two that gives 1.5 k.  Returns -1 if no setting up to 64 suffices.
+// Number of groups G per warp tile whose maxima bound the tile cutoff (a power of two,
+// 2..32, or 64 with half-lane groups).  For position-independent data a warp tile's
+// cutoff exceeds t with probability (1 - exp(-x))^G, x = (elements above t per group),
+// so the row-wide cutoff T (the largest over Nw warp tiles) sits where
+// 1 - exp(-x) = Nw^(-1/G), and the proven prefix holds about
+//     P(G) = V * (G / 1024) * -ln(1 - Nw^(-1/G))
+// elements.  Pick the smallest G whose P(G) clears k with a margin that covers the
+// spread of T, and give up (-1: exact kernel) if that needs more than the merge can sort.
+// G = 0 means "keep every finite element" (vocabularies the merge can sort whole).
 __device__ __forceinline__ int pick_groups(int k, int V) {
     if (V <= MERGE_CAP) return 0;
-    float nw = (float)((V + WARP_TILE - 1) / WARP_TILE);
-    float lg = __log2f(nw);
+    const float nw = (float)((V + WARP_TILE - 1) / WARP_TILE);
+    const float lg = __log2f(nw);
     for (int G = 2; G <= 64; G <<= 1) {
-        float est = (float)G * exp2f(lg * (1.0f - 1.0f / (float)G));
-        if (est >= 1.5f * (float)k) return G;
+        const float r = exp2f(-lg / (float)G);                       // Nw^(-1/G)
+        const float est = (float)V * ((float)G / (float)WARP_TILE) * -__logf(1.0f - r);
+        const float need = (float)k * (1.0f + 4.0f * rsqrtf((float)G)) + 30.0f;
+        if (est >= need) return (est <= 0.7f * (float)MERGE_CAP) ? G : -1;
     }
     return -1;
 }

@@ -19,7 +19,14 @@
 namespace sonic {
 namespace cg = cooperative_groups;
 
-constexpr int EX_THREADS = 1024;
+#ifdef SONIC_TRACE
+// debug builds: rank 0 / thread 0 of the cluster handling the traced row stamps the clock into the workspace header
+#define SONIC_STAMP(i) do { if (x.rank == 0 && x.tid == 0 && x.trace) x.tracep[8 + (i)] = (unsigned int)clock64(); } while (0)
+#else
+#define SONIC_STAMP(i) do { } while (0)
+#endif
+
+constexpr int EX_THREADS = 512;
 constexpr int EX_WARPS = EX_THREADS / 32;
 constexpr int CL = 8;                         // CTAs per cluster
 constexpr int SLICE_MAX = MAX_VOCAB / CL;     // 32768 keys per CTA
@@ -53,6 +60,8 @@ struct ExactCtx {
     unsigned int *hcnt, *hm0, *hm1, *hm2;      // per-bin count and mass in three 14-bit limbs (32-bit adds only)
     int rank, lo, len, per, tid, lane, warp;
     int phase;
+    int trace;
+    unsigned int *tracep;
     float Mf;                                  // largest processed logit
 };
 
@@ -94,6 +103,16 @@ __device__ __forceinline__ unsigned long long block_sum_u64(ExactCtx &x, unsigne
 #pragma unroll
     for (int w = 0; w < EX_WARPS; ++w) t += x.sh->wtot[w];
     return t;
+}
+
+// Position for an element a lane wants to append to a list whose length lives in shared
+// memory: one atomic per warp.  Every lane of the warp must call it (want = false to skip).
+__device__ __forceinline__ unsigned int warp_append(unsigned int *counter, bool want, int lane) {
+    const unsigned int m = __ballot_sync(0xFFFFFFFFu, want);
+    unsigned int base = 0;
+    if (lane == 0 && m) base = atomicAdd(counter, (unsigned int)__popc(m));
+    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+    return base + __popc(m & ((1u << lane) - 1u));
 }
 
 // Fixed-point softmax weight of a key relative to the row maximum: 2^40 * exp(y - M).
@@ -329,6 +348,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         return 2047 - (int)t;
     };
     const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin);
+    SONIC_STAMP(4);
     auto dig_b = [&](uint32_t key) -> int {
         float t = __fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f);
         int aa = (int)fminf(t, 2047.0f);
@@ -338,6 +358,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     };
     int b = -1;
     if (in_bin > (unsigned long long)GATHER_CAP) b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin);
+    SONIC_STAMP(5);
     auto in_range = [&](uint32_t key) -> bool {
         if (dig_a(key) != a) return false;
         return b < 0 || dig_b(key) == b;
@@ -358,14 +379,15 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         unsigned int off = 0, n = 0;
         for (int r = 0; r < CL; ++r) { if (r < x.rank) off += (unsigned int)all[r][0]; n += (unsigned int)all[r][0]; }
         unsigned long long *dst = cg::this_cluster().map_shared_rank(sortbuf, 0);
-        for (int i = x.tid; i < x.len; i += EX_THREADS) {
-            uint32_t key = x.keys[i];
-            if (member(base, key, x.lo + i) && in_range(key)) {
-                unsigned int pos = off + atomicAdd(&x.sh->ucount, 1u);
-                if (pos < (unsigned int)GATHER_CAP) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
-            }
+        for (int i0 = 0; i0 < x.len; i0 += EX_THREADS) {
+            const int i = i0 + x.tid;
+            const uint32_t key = (i < x.len) ? x.keys[i] : 0u;
+            const bool want = (i < x.len) && member(base, key, x.lo + i) && in_range(key);
+            const unsigned int pos = off + warp_append(&x.sh->ucount, want, x.lane);
+            if (want && pos < (unsigned int)GATHER_CAP) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
         }
         cg::this_cluster().sync();
+        SONIC_STAMP(6);
         unsigned long long v2[XV] = {0, 0, 0, 0};
         if (x.rank == 0) {
             const int nn = (int)min(n, (unsigned int)GATHER_CAP);
@@ -373,6 +395,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
             for (int i = nn + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
             __syncthreads();
             bitonic_sort_desc<EX_THREADS>(sortbuf, m, x.tid);
+            SONIC_STAMP(7);
             // running count / mass in ranking order; each thread owns a contiguous chunk of the sorted list
             const int chunk = (nn + EX_THREADS - 1) / EX_THREADS;
             const int lo = min(nn, x.tid * chunk), hi = min(nn, lo + chunk);
@@ -402,6 +425,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
             v2[0] = sortbuf[max(0, x.sh->flag)];
         }
         allgather(x, v2, all);
+        SONIC_STAMP(8);
         Cut c;
         c.v = (uint32_t)(all[0][0] >> 32);
         c.idx = (int)(~(uint32_t)all[0][0]);
@@ -450,11 +474,27 @@ template <int DT>
 __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned long long *sortbuf) {
     const RowCfg c = load_cfg(P, row);
     RowState *rs = P.rs + row;
+#ifdef SONIC_TRACE
+    x.tracep = P.error;
+    x.trace = (row == (int)P.error[4]);
+#endif
     const int V = P.V;
     x.per = (((V + CL - 1) / CL) + 1023) & ~1023;
     x.lo = x.rank * x.per;
     x.len = max(0, min(V - x.lo, x.per));
     cg::this_cluster().sync();                               // every CTA of the cluster is resident before DSMEM traffic
+    SONIC_STAMP(0);
+#ifdef SONIC_TRACE
+    SONIC_STAMP(12);
+    cg::this_cluster().sync();
+    SONIC_STAMP(13);
+    cg::this_cluster().sync();
+    SONIC_STAMP(14);
+    { unsigned long long tv[XV] = {1, 2, 3, 4}; unsigned long long ta[CL][XV]; allgather(x, tv, ta); if (ta[0][0] == 77) x.trace = 0; }
+    SONIC_STAMP(15);
+    __syncthreads();
+    SONIC_STAMP(16);
+#endif
 
     // ---- load the slice, mask, sparse patches, temperature, keys
     constexpr int VEC = VecTraits<DT>::VEC;
@@ -513,6 +553,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         }
     }
     bad = __syncthreads_or(bad);
+    SONIC_STAMP(1);
     uint32_t kmax = 0;
     unsigned long long nfin = 0;
     for (int li = x.tid; li < x.per; li += EX_THREADS) {
@@ -539,6 +580,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     unsigned long long Nf = 0;
     for (int r = 0; r < CL; ++r) { Mkey = max(Mkey, (uint32_t)all[r][0]); Nf += all[r][1]; }
     x.Mf = unkey(Mkey);
+    SONIC_STAMP(2);
     const bool leader = (x.rank == 0 && x.tid == 0);
 
     if (bad) {
@@ -563,12 +605,12 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         unsigned int off = 0;
         for (int r = 0; r < x.rank; ++r) off += (unsigned int)all[r][0];
         unsigned long long *dst = cg::this_cluster().map_shared_rank(sortbuf, 0);
-        for (int i = x.tid; i < x.len; i += EX_THREADS) {
-            uint32_t key = x.keys[i];
-            if (member(cut, key, x.lo + i)) {
-                unsigned int pos = off + atomicAdd(&x.sh->ucount, 1u);
-                if (pos < (unsigned int)MAX_TOPK) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
-            }
+        for (int i0 = 0; i0 < x.len; i0 += EX_THREADS) {
+            const int i = i0 + x.tid;
+            const uint32_t key = (i < x.len) ? x.keys[i] : 0u;
+            const bool want = (i < x.len) && member(cut, key, x.lo + i);
+            const unsigned int pos = off + warp_append(&x.sh->ucount, want, x.lane);
+            if (want && pos < (unsigned int)MAX_TOPK) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
         }
         cg::this_cluster().sync();
         if (x.rank == 0) {
@@ -597,7 +639,9 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     if (c.k > 0 && (unsigned long long)c.k < Nf) cut = select_cut(x, cut, false, (unsigned long long)c.k, 1.0f, sortbuf);
     const Cut cut_k = cut;
     if (c.z & M_TOP_P) {
+        SONIC_STAMP(3);
         Cut cp = select_cut(x, cut_k, true, 0ull, c.p, sortbuf);
+        SONIC_STAMP(9);
         if (tighter(cp, cut)) cut = cp;
     }
     if (c.z & M_MIN_P) {
@@ -627,10 +671,12 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     // total mass first (target depends on it): a crossing search with an unreachable target
     unsigned long long Wq;
     ordered_cross<unsigned long long>(x, ~0ull, false, wq, Wq);
+    SONIC_STAMP(10);
     const unsigned long long mul = 2ull * a_draw + 1ull;               // u = mul / 2^25
     const unsigned long long T = (__umul64hi(Wq, mul) << 39) | ((Wq * mul) >> 25);
     unsigned long long dummy;
     int token = ordered_cross<unsigned long long>(x, T, true, wq, dummy);
+    SONIC_STAMP(11);
 
     uint32_t flags = F_FALLBACK;
     float p_draft = 0.0f;
@@ -682,9 +728,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     cg::this_cluster().sync();
 }
 
-// Persistent clusters: cluster c handles rows c, c + nclusters, ...; it first marks
-// the rows that need this path (their class, or a failure recorded by the
-// streaming kernel), then processes them in order.
+// Persistent clusters over the rows that need this path.
 template <int DT>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
 sonic_exact_kernel(const KParams P) {
@@ -700,25 +744,28 @@ sonic_exact_kernel(const KParams P) {
     unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192);
     uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8);
 
+    // Every CTA marks, for ALL rows, which ones need this path (their class, or a failure recorded
+    // by the merge kernel); the marked rows are then dealt round-robin to the clusters, so the
+    // work is balanced whatever the rows' positions.  All CTAs derive the same list.
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;
-    const int nmine = (P.rows - cid + ncl - 1) / ncl;           // rows of this cluster (cid < rows by construction)
-    const int nwords = (nmine + 31) >> 5;
+    const int nwords = (P.rows + 31) >> 5;
     for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
     __syncthreads();
-    for (int j = x.tid; j < nmine; j += EX_THREADS) {
-        const int row = cid + j * ncl;
+    for (int row = x.tid; row < P.rows; row += EX_THREADS) {
         const RowCfg c = load_cfg(P, row);
         const unsigned int status = __ldcg(&P.rs[row].status);
-        if (c.cls == CLS_EXACT || (status & ST_FAILED)) atomicOr(&need[j >> 5], 1u << (j & 31));
+        if (c.cls == CLS_EXACT || (status & ST_FAILED)) atomicOr(&need[row >> 5], 1u << (row & 31));
     }
     __syncthreads();
+    int ordinal = 0;
     for (int w = 0; w < nwords; ++w) {
         uint32_t bits = need[w];
         while (bits) {
-            const int j = (w << 5) + __ffs(bits) - 1;
+            const int row = (w << 5) + __ffs(bits) - 1;
             bits &= bits - 1;
-            exact_row<DT>(P, cid + j * ncl, x, sortbuf);
+            if (ordinal % ncl == cid) exact_row<DT>(P, row, x, sortbuf);
+            ++ordinal;
         }
     }
 }

@@ -72,13 +72,14 @@ __device__ __forceinline__ int slot_index(int wbase, int lane, int s) {
     return wbase + (s / VEC) * 32 * VEC + lane * VEC + (s % VEC);
 }
 
+template <int THREADS>
 struct MergeShared {
     int count;
     int tcnt[MAX_TILES + 1];                   // exclusive prefix of the tiles' candidate counts
     unsigned int tkey;
     int n_p, n_m, pick;
     int found;
-    double scratch[STREAM_THREADS];
+    double scratch[THREADS];
 };
 
 // Writes the per-row outputs of the sample / verify operations.
@@ -96,12 +97,27 @@ __device__ __forceinline__ void emit_row(const KParams &P, const RowCfg &c, int 
     }
 }
 
-// Row merge for top-k class rows, run by the 256 consumer threads of the CTA
-// that finished the row's last tile.  buf is MERGE_CAP 64-bit words of shared
-// memory.  Returns false if the candidates cannot prove the row's answer.
+#ifdef SONIC_TRACE
+#define MERGE_STAMP(i) do { if (tid == 0 && row == (int)P.error[4]) P.error[8 + (i)] = (unsigned int)clock64(); } while (0)
+#else
+#define MERGE_STAMP(i) do { } while (0)
+#endif
+
+constexpr int RANK_SORT_MAX = 1024;           // at most this many candidates: sort by rank counting
+constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
+struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
+
+template <int NT, typename Sync, typename SH>
+__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid);
+
+// Row merge for top-k class rows (one CTA per row).  buf is MERGE_CAP 64-bit
+// words of shared memory.  Returns false if the candidates cannot prove the
+// row's answer.
+template <int THREADS, typename Sync>
 __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int tiles,
-                               unsigned long long *buf, MergeShared &sh, int tid) {
-    ConsumerSync csync;
+                               unsigned long long *buf, MergeShared<THREADS> &sh, int tid) {
+    Sync csync;
+    MERGE_STAMP(0);
     const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
     const TileRec *rec = P.tiles + (size_t)row * MAX_TILES;
     // tile records: one thread per tile, then a serial prefix over at most 32 entries
@@ -120,37 +136,71 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         for (int t = 0; t < tiles; ++t) sh.tcnt[t + 1] += sh.tcnt[t];
     }
     csync();
+    MERGE_STAMP(1);
     const unsigned int tkey = sh.tkey;
     const bool complete = (tkey == KEY_NEG_INF);
     const bool strict = c.temp && !complete;            // keys are compared after the temperature division
     const uint32_t tykey = c.temp ? okey(__fdiv_rn(unkey(tkey), c.tau)) : tkey;
     const int total = sh.tcnt[tiles];
-    for (int j = tid; j < total; j += STREAM_THREADS) {
-        int t = 0;
-        while (sh.tcnt[t + 1] <= j) ++t;
-        unsigned long long cd = __ldcg(P.cand + (size_t)row * CAND_CAP + (size_t)t * cap_t + (j - sh.tcnt[t]));
-        uint32_t zk = (uint32_t)(cd >> 32);
-        if (zk < tkey) continue;
-        uint32_t yk = zk;
-        if (c.temp) yk = okey(__fdiv_rn(unkey(zk), c.tau));
-        if (strict && yk <= tykey) continue;
-        int pos = atomicAdd(&sh.count, 1);
-        if (pos < MERGE_CAP) buf[pos] = ((unsigned long long)yk << 32) | (uint32_t)cd;
+    for (int j0 = 0; j0 < total; j0 += THREADS) {
+        const int j = j0 + tid;
+        bool keep = false;
+        unsigned long long out = 0ull;
+        if (j < total) {
+            int t = 0;
+            while (sh.tcnt[t + 1] <= j) ++t;
+            const unsigned long long cd = __ldcg(P.cand + (size_t)row * CAND_CAP + (size_t)t * cap_t + (j - sh.tcnt[t]));
+            const uint32_t zk = (uint32_t)(cd >> 32);
+            uint32_t yk = zk;
+            if (c.temp) yk = okey(__fdiv_rn(unkey(zk), c.tau));
+            keep = (zk >= tkey) && !(strict && yk <= tykey);
+            out = ((unsigned long long)yk << 32) | (uint32_t)cd;
+        }
+        // one shared-memory atomic per warp, not per candidate
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, keep);
+        int base = 0;
+        if ((tid & 31) == 0 && m) base = atomicAdd(&sh.count, __popc(m));
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if (keep) {
+            const int pos = base + __popc(m & ((1u << (tid & 31)) - 1u));
+            if (pos < MERGE_CAP) buf[pos] = out;
+        }
     }
     csync();
     const int Pn = sh.count;
+    MERGE_STAMP(2);
     if (Pn > MERGE_CAP) return false;
     int n;
     if (Pn >= c.k) n = c.k;
     else if (complete && P.op != OP_TOPK) n = Pn;
     else return false;
-    const int m = next_pow2(Pn);
-    for (int i = Pn + tid; i < m; i += STREAM_THREADS) buf[i] = 0ull;
-    csync();
-    bitonic_sort_desc<STREAM_THREADS, ConsumerSync>(buf, m, tid);
+    unsigned long long *sorted = buf;
+    if (Pn <= RANK_SORT_MAX) {
+        // few candidates: each key counts the keys above it (keys are distinct) and lands at its rank
+        unsigned long long *dst = buf + MERGE_CAP / 2;
+        for (int i = tid; i < Pn; i += THREADS) {
+            const unsigned long long key = buf[i];
+            int rank = 0;
+            for (int j = 0; j < Pn; ++j) rank += (buf[j] > key) ? 1 : 0;
+            dst[rank] = key;
+        }
+        csync();
+        for (int i = tid; i < Pn; i += THREADS) buf[i] = dst[i];
+        csync();
+    } else {
+        const int m = next_pow2(Pn);
+        for (int i = Pn + tid; i < m; i += THREADS) buf[i] = 0ull;
+        csync();
+        bitonic_sort_desc<THREADS, Sync>(buf, m, tid);
+    }
+    (void)sorted;
+    MERGE_STAMP(3);
+#ifdef SONIC_TRACE
+    if (tid == 0 && row == (int)P.error[4]) { P.error[30] = Pn; P.error[31] = n; }
+#endif
 
     if (P.op == OP_TOPK) {
-        for (int j = tid; j < n; j += STREAM_THREADS) {
+        for (int j = tid; j < n; j += THREADS) {
             unsigned long long kv = buf[j];
             P.out_vals[(size_t)row * P.ktop + j] = unkey((uint32_t)(kv >> 32));
             P.out_idx[(size_t)row * P.ktop + j] = (int)(~(uint32_t)kv);
@@ -161,6 +211,23 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN, 0, 0.0f);
         return true;
     }
+    // small supports are finished by one warp without block barriers
+    if (n <= WARP_EPILOGUE_MAX) {
+        if (tid < 32) merge_epilogue<32, WarpSync>(P, c, row, n, buf, sh, tid);
+    } else {
+        merge_epilogue<THREADS, Sync>(P, c, row, n, buf, sh, tid);
+    }
+    return true;
+}
+
+// Truncation epilogue and token selection over the n best candidates, sorted in
+// buf[0, n) (TopK already applied): TopP, MinP, index-order CDF, Philox draw,
+// and for verification rows the accept test and the residual.  Run by NT
+// threads that synchronise with Sync (a whole CTA, or one warp).
+template <int NT, typename Sync, typename SH>
+__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+    Sync csync;
+    constexpr int THREADS = NT;
     // shared-memory layout after the sort (n <= KFAST_SAMPLE = MERGE_CAP / 4):
     //   buf[0, n)     sorted keys (value key << 32 | ~index)
     //   w             weights exp(y - M) in ranking order
@@ -170,23 +237,25 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     double *cs = reinterpret_cast<double *>(buf + 2 * KFAST_SAMPLE);
     unsigned long long *ik = buf + 3 * KFAST_SAMPLE;
     const double M = (double)unkey((uint32_t)(buf[0] >> 32));
-    for (int j = tid; j < n; j += STREAM_THREADS) {
+    for (int j = tid; j < n; j += THREADS) {
         double y = (double)unkey((uint32_t)(buf[j] >> 32));
         double wj = exp(y - M);
         w[j] = wj; cs[j] = wj;
     }
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
     csync();
-    block_inclusive_scan<STREAM_THREADS, ConsumerSync>(cs, n, sh.scratch, tid);
+    MERGE_STAMP(4);
+    block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
+    MERGE_STAMP(5);
     const double Z = cs[n - 1];
     if (c.z & M_TOP_P) {
         const double target = (double)c.p * Z;
-        for (int j = tid; j < n; j += STREAM_THREADS)
+        for (int j = tid; j < n; j += THREADS)
             if (cs[j] >= target && (j == 0 || cs[j - 1] < target)) sh.n_p = j + 1;
     }
     if (c.z & M_MIN_P) {
         const double thr = M + log((double)c.theta);
-        for (int j = tid; j < n; j += STREAM_THREADS) {
+        for (int j = tid; j < n; j += THREADS) {
             bool in = (double)unkey((uint32_t)(buf[j] >> 32)) >= thr;
             bool prev_in = (j == 0) || ((double)unkey((uint32_t)(buf[j - 1] >> 32)) >= thr);
             if (!in && prev_in) sh.n_m = j;
@@ -198,10 +267,12 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     csync();
     // survivors in vocabulary-index order
     const int m2 = next_pow2(n);
-    for (int j = tid; j < m2; j += STREAM_THREADS)
+    for (int j = tid; j < m2; j += THREADS)
         ik[j] = (j < n) ? ((buf[j] << 32) | (unsigned long long)j) : 0ull;
     csync();
-    bitonic_sort_desc<STREAM_THREADS, ConsumerSync>(ik, m2, tid);
+    MERGE_STAMP(6);
+    bitonic_sort_desc<THREADS, Sync>(ik, m2, tid);
+    MERGE_STAMP(7);
 
     uint32_t a_acc, a_draw;
     draw_cells(P, c, a_acc, a_draw);
@@ -214,7 +285,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)P.V;
         if (tid == 0) sh.pick = -1;
         csync();
-        for (int j = tid; j < n; j += STREAM_THREADS)
+        for (int j = tid; j < n; j += THREADS)
             if ((int)(~(uint32_t)(ik[j] >> 32)) == d) sh.pick = j;
         csync();
         double Pd = 0.0;
@@ -225,26 +296,27 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         if (accept) flags |= F_ACCEPT;
         csync();
         // residual max(0, p - q) over the support, in index order
-        for (int j = tid; j < n; j += STREAM_THREADS) {
+        for (int j = tid; j < n; j += THREADS) {
             int idx = (int)(~(uint32_t)(ik[j] >> 32));
             double r = w[(uint32_t)ik[j]] / W - (double)__ldg(q + idx);
             cs[j] = r > 0.0 ? r : 0.0;
         }
         csync();
-        block_inclusive_scan<STREAM_THREADS, ConsumerSync>(cs, n, sh.scratch, tid);
+        block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
         use_residual = cs[n - 1] > 0.0;
         csync();
     }
     if (!use_residual) {
-        for (int j = tid; j < n; j += STREAM_THREADS) cs[j] = w[(uint32_t)ik[j]];
+        for (int j = tid; j < n; j += THREADS) cs[j] = w[(uint32_t)ik[j]];
         csync();
-        block_inclusive_scan<STREAM_THREADS, ConsumerSync>(cs, n, sh.scratch, tid);
+        block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
     }
+    MERGE_STAMP(8);
     const double R = cs[n - 1];
     const double target = u_draw * R;
     if (tid == 0) sh.pick = n - 1;
     csync();
-    for (int j = tid; j < n; j += STREAM_THREADS)
+    for (int j = tid; j < n; j += THREADS)
         if (cs[j] > target && (j == 0 || !(cs[j - 1] > target))) sh.pick = j;
     csync();
     if (tid == 0) {
@@ -253,7 +325,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         float prob = (float)(w[(uint32_t)ik[j]] / W);
         emit_row(P, c, row, token, prob, flags, n, p_draft);
     }
-    return true;
+    MERGE_STAMP(9);
 }
 
 // What the producer hands to the consumers with each stage.
@@ -272,8 +344,6 @@ struct StreamShared {
     float tw[STREAM_WARPS];
     int wcnt[STREAM_WARPS];
     unsigned long long best[STREAM_WARPS];
-    int last;
-    MergeShared merge;
 };
 
 template <int DT>
@@ -348,6 +418,19 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                 mw[j] = ((w < nwords) ? __ldg(mrow + w) : 0u) >> (first & 31);
             }
         }
+        // the first entries of the row's sparse lists as well (lengths are checked once the configuration is known)
+        const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
+        int h_id0 = -1, h_ct0 = 0, h_id1 = -1, h_ct1 = 0, b_id0 = -1;
+        float b_v0 = 0.0f;
+        const int *hid = P.hist_ids ? P.hist_ids + (size_t)req * P.hist_stride : nullptr;
+        const int *hct = P.hist_counts ? P.hist_counts + (size_t)req * P.hist_stride : nullptr;
+        const int *bid = P.bias_ids ? P.bias_ids + (size_t)req * P.bias_stride : nullptr;
+        const float *bvl = P.bias_vals ? P.bias_vals + (size_t)req * P.bias_stride : nullptr;
+        if (hid && hct) {
+            if (tid < P.hist_stride) { h_id0 = __ldg(hid + tid); h_ct0 = __ldg(hct + tid); }
+            if (tid + STREAM_THREADS < P.hist_stride) { h_id1 = __ldg(hid + tid + STREAM_THREADS); h_ct1 = __ldg(hct + tid + STREAM_THREADS); }
+        }
+        if (bid && bvl && tid < P.bias_stride) { b_id0 = __ldg(bid + tid); b_v0 = __ldg(bvl + tid); }
         if (!mbar_wait(&sh.full[s], (n / NSTAGE) & 1)) {
             if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
             return;
@@ -362,17 +445,6 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
             const bool tail = tile_base + CTA_TILE > P.V;
             const bool patched = (c.hist_len > 0 || c.bias_len > 0);
             float *ptile = (DT == 0) ? reinterpret_cast<float *>(stage) : conv;    // fp32 view the sparse lists patch
-
-            // list entries of this thread (issued early; applied after the tile is staged as fp32)
-            int h_id0 = -1, h_ct0 = 0, h_id1 = -1, h_ct1 = 0, b_id0 = -1;
-            float b_v0 = 0.0f;
-            const int *hid = P.hist_ids + (size_t)c.b * P.hist_stride;
-            const int *hct = P.hist_counts + (size_t)c.b * P.hist_stride;
-            const int *bid = P.bias_ids + (size_t)c.b * P.bias_stride;
-            const float *bvl = P.bias_vals + (size_t)c.b * P.bias_stride;
-            if (tid < c.hist_len) { h_id0 = __ldg(hid + tid); h_ct0 = __ldg(hct + tid); }
-            if (tid + STREAM_THREADS < c.hist_len) { h_id1 = __ldg(hid + tid + STREAM_THREADS); h_ct1 = __ldg(hct + tid + STREAM_THREADS); }
-            if (tid < c.bias_len) { b_id0 = __ldg(bid + tid); b_v0 = __ldg(bvl + tid); }
 
             float e[EPL];
             auto read_raw = [&]() {
@@ -554,62 +626,61 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                 if (tid == 0) { rec->cnt = (unsigned int)total; rec->tkey = okey(t); }
             }
 
-            // ---- the CTA that finishes the row's last tile merges the row while others keep streaming
-            __threadfence();
-            csync();
-            if (tid == 0) {
-                __threadfence();
-                const unsigned int done = atomicAdd(&rs->ticket, 1u);
-                sh.last = (done == (unsigned int)tiles - 1) ? 1 : 0;
-            }
-            csync();
-            if (sh.last) {
-                __threadfence();
-                const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
-                const unsigned int status = __ldcg(&rs->status);
-                bool ok = true;
-                if (c.bad || (status & ST_BADID)) {
-                    if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_BADPARAM, 0, 0.0f);
-                } else if (c.cls == CLS_GREEDY) {
-                    if (tid < 32) {
-                        unsigned long long best = (tid < tiles) ? __ldcg(&recs[tid].best) : 0ull;
-#pragma unroll
-                        for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
-                        if (tid == 0) {
-                            if (P.op == OP_TOPK) {
-                                // k == 1: a row of nothing but -inf still has a first element
-                                P.out_vals[row] = best ? unkey((uint32_t)(best >> 32)) : -CUDART_INF_F;
-                                P.out_idx[row] = best ? (int)(~(uint32_t)best) : 0;
-                            } else if (best == 0ull) {
-                                emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN, 0, 0.0f);
-                            } else {
-                                const int token = (int)(~(uint32_t)best);
-                                uint32_t flags = 0;
-                                float pd = 0.0f;
-                                if (P.op == OP_VERIFY && c.l < P.K) {
-                                    const bool acc = P.draft_tokens[(size_t)c.b * P.K + c.l] == token;
-                                    if (acc) { flags |= F_ACCEPT; pd = 1.0f; }
-                                }
-                                emit_row(P, c, row, token, 1.0f, flags, 1, pd);
-                            }
-                        }
-                    }
-                } else {
-                    // the merge sorts in the fp32 tile of this stage (fp32 logits) or in the conversion tile (bf16)
-                    ok = merge_topk_row(P, c, row, tiles, reinterpret_cast<unsigned long long *>(ptile), sh.merge, tid);
-                }
-                csync();
-                if (tid == 0) {
-                    rs->ticket = 0;
-                    rs->status = ok ? 0u : ST_FAILED;
-                }
-            }
-            // generic-proxy writes into the stage (patches, merge scratch) precede the next bulk copy into it
-            if (DT == 0) fence_async_proxy();
+            // generic-proxy writes into the stage (in-place patches) precede the next bulk copy into it
+            if (DT == 0 && patched) fence_async_proxy();
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.empty[s]);
     }
+}
+
+// One CTA per row of the streaming classes: combines the tile records and
+// finishes the row (global top-k, truncation epilogue, token selection, or the
+// per-position verification result).  Rows it cannot prove are flagged for the
+// exact kernel.
+__global__ void __launch_bounds__(MERGE_THREADS)
+sonic_merge_kernel(const KParams P, const int tiles) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ MergeShared<MERGE_THREADS> s_merge;
+    const int row = blockIdx.x;
+    const int tid = threadIdx.x;
+    const RowCfg c = load_cfg(P, row);
+    if (c.cls == CLS_EXACT) return;
+    RowState *rs = P.rs + row;
+    const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
+    const unsigned int status = rs->status;
+    if (c.bad || (status & ST_BADID)) {
+        if (tid == 0) { emit_row(P, c, row, -1, 0.0f, F_BADPARAM, 0, 0.0f); rs->status = 0; }
+        return;
+    }
+    if (c.cls == CLS_GREEDY) {
+        if (tid < 32) {
+            unsigned long long best = (tid < tiles) ? recs[tid].best : 0ull;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
+            if (tid == 0) {
+                if (P.op == OP_TOPK) {
+                    // k == 1: a row of nothing but -inf still has a first element
+                    P.out_vals[row] = best ? unkey((uint32_t)(best >> 32)) : -CUDART_INF_F;
+                    P.out_idx[row] = best ? (int)(~(uint32_t)best) : 0;
+                } else if (best == 0ull) {
+                    emit_row(P, c, row, -1, 0.0f, F_NO_TOKEN, 0, 0.0f);
+                } else {
+                    const int token = (int)(~(uint32_t)best);
+                    uint32_t flags = 0;
+                    float pd = 0.0f;
+                    if (P.op == OP_VERIFY && c.l < P.K) {
+                        const bool acc = P.draft_tokens[(size_t)c.b * P.K + c.l] == token;
+                        if (acc) { flags |= F_ACCEPT; pd = 1.0f; }
+                    }
+                    emit_row(P, c, row, token, 1.0f, flags, 1, pd);
+                }
+            }
+        }
+        return;
+    }
+    const bool ok = merge_topk_row<MERGE_THREADS, BlockSync>(P, c, row, tiles, reinterpret_cast<unsigned long long *>(smem_raw), s_merge, tid);
+    if (tid == 0 && !ok) rs->status = ST_FAILED;
 }
 
 }  // namespace sonic
