@@ -128,19 +128,32 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     const long long nitems_ll = (long long)tiles * P.rows;
     if (nitems_ll > 0x7FFFFFFF) return fail(SONIC_ESHAPE, "rows x tiles too large");
     const int nitems = (int)nitems_ll;
-    const int grid1 = nitems < sm_count * 2 ? nitems : sm_count * 2;       // persistent: two CTAs per SM
+    const int grid1 = nitems < sm_count * 3 ? nitems : sm_count * 3;       // persistent: three CTAs per SM
     if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems);
     else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
-    sonic_merge_kernel<<<P.rows, MERGE_THREADS, MERGE_SMEM, st>>>(P, tiles);
-    e = cudaGetLastError();
+    // merge and exact kernels are programmatic dependents: they may begin launching while their
+    // predecessor still runs and synchronise on it inside the kernel
+    cudaLaunchAttribute pdl;
+    pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.stream = st;
+    cfg.attrs = &pdl;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(P.rows);
+    cfg.blockDim = dim3(MERGE_THREADS);
+    cfg.dynamicSmemBytes = MERGE_SMEM;
+    e = cudaLaunchKernelEx(&cfg, sonic_merge_kernel, P, tiles);
     if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
 
-    dim3 grid2((P.rows < max_clusters ? P.rows : max_clusters) * CL);
-    if (P.dtype == SONIC_DTYPE_F32) sonic_exact_kernel<0><<<grid2, EX_THREADS, EXACT_SMEM, st>>>(P);
-    else sonic_exact_kernel<1><<<grid2, EX_THREADS, EXACT_SMEM, st>>>(P);
-    e = cudaGetLastError();
+    cfg.gridDim = dim3((P.rows < max_clusters ? P.rows : max_clusters) * CL);
+    cfg.blockDim = dim3(EX_THREADS);
+    cfg.dynamicSmemBytes = EXACT_SMEM;
+    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P);
+    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P);
     if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch");
 
     if (P.op == OP_VERIFY) {

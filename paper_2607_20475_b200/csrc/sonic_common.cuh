@@ -238,6 +238,12 @@ __device__ __forceinline__ unsigned long long ldcg_u64(const unsigned long long 
     return __ldcg(p);
 }
 
+// Programmatic dependent launch (the paper overlaps its two stages the same way, Section 3.5):
+// a kernel lets the next kernel of the stream start launching early, and that kernel waits
+// here until the previous one has completed and its writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Block-level barriers: the whole CTA, or only the 256 consumer threads of the
 // streaming kernel (named barrier 1; its producer warp never joins).
 struct BlockSync { __device__ __forceinline__ void operator()() const { __syncthreads(); } };
@@ -246,6 +252,9 @@ struct ConsumerSync {
 };
 
 // Descending bitonic sort of m (power of two) 64-bit keys in shared memory.
+// The 32 lanes of a warp always work on one aligned block of 64 keys when the
+// partner distance j is at most 32, so those stages only need a warp barrier;
+// the block barrier is kept around the stages with j >= 64.
 template <int THREADS, typename Sync = BlockSync>
 __device__ __forceinline__ void bitonic_sort_desc(unsigned long long *a, int m, int tid) {
     Sync sync;
@@ -258,7 +267,8 @@ __device__ __forceinline__ void bitonic_sort_desc(unsigned long long *a, int m, 
                 bool desc = ((lo & k2) == 0);
                 if ((x < y) == desc) { a[lo] = y; a[hi] = x; }
             }
-            sync();
+            const int jn = (j > 1) ? (j >> 1) : k2;          // partner distance of the next stage
+            if (j >= 64 || jn >= 64 || (k2 == m && j == 1)) sync(); else __syncwarp();
         }
     }
 }

@@ -744,28 +744,35 @@ sonic_exact_kernel(const KParams P) {
     unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192);
     uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8);
 
-    // Every CTA marks, for ALL rows, which ones need this path (their class, or a failure recorded
-    // by the merge kernel); the marked rows are then dealt round-robin to the clusters, so the
-    // work is balanced whatever the rows' positions.  All CTAs derive the same list.
+    // Two rounds.  Round 0: the rows that belong to this path by class (known from the inputs alone,
+    // so this round may run while the merge kernel is still busy).  Round 1, after the merge kernel
+    // has completed: the rows it could not prove.  In each round every CTA marks the rows of ALL
+    // requests and the marked rows are dealt round-robin to the clusters (all CTAs derive the same list).
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;
     const int nwords = (P.rows + 31) >> 5;
-    for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
-    __syncthreads();
-    for (int row = x.tid; row < P.rows; row += EX_THREADS) {
-        const RowCfg c = load_cfg(P, row);
-        const unsigned int status = __ldcg(&P.rs[row].status);
-        if (c.cls == CLS_EXACT || (status & ST_FAILED)) atomicOr(&need[row >> 5], 1u << (row & 31));
-    }
-    __syncthreads();
-    int ordinal = 0;
-    for (int w = 0; w < nwords; ++w) {
-        uint32_t bits = need[w];
-        while (bits) {
-            const int row = (w << 5) + __ffs(bits) - 1;
-            bits &= bits - 1;
-            if (ordinal % ncl == cid) exact_row<DT>(P, row, x, sortbuf);
-            ++ordinal;
+    for (int round = 0; round < 2; ++round) {
+        if (round == 1) pdl_wait_primary();
+        __syncthreads();
+        for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
+        __syncthreads();
+        for (int row = x.tid; row < P.rows; row += EX_THREADS) {
+            const RowCfg c = load_cfg(P, row);
+            bool mine;
+            if (round == 0) mine = (c.cls == CLS_EXACT);
+            else mine = (c.cls != CLS_EXACT) && (__ldcg(&P.rs[row].status) & ST_FAILED);
+            if (mine) atomicOr(&need[row >> 5], 1u << (row & 31));
+        }
+        __syncthreads();
+        int ordinal = 0;
+        for (int w = 0; w < nwords; ++w) {
+            uint32_t bits = need[w];
+            while (bits) {
+                const int row = (w << 5) + __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (ordinal % ncl == cid) exact_row<DT>(P, row, x, sortbuf);
+                ++ordinal;
+            }
         }
     }
 }

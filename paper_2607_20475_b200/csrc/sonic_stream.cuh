@@ -27,8 +27,8 @@
 namespace sonic {
 
 template <int DT> struct VecTraits;
-template <> struct VecTraits<0> { static constexpr int VEC = 4, NV = 8, NSTAGE = 3, ELT = 4; };
-template <> struct VecTraits<1> { static constexpr int VEC = 8, NV = 4, NSTAGE = 4, ELT = 2; };
+template <> struct VecTraits<0> { static constexpr int VEC = 4, NV = 8, NSTAGE = 2, ELT = 4; };
+template <> struct VecTraits<1> { static constexpr int VEC = 8, NV = 4, NSTAGE = 2, ELT = 2; };
 
 constexpr int STREAM_CTA_THREADS = STREAM_THREADS + 32;      // eight consumer warps + the producer warp
 constexpr unsigned int WAIT_LIMIT = 1u << 22;                // try_wait rounds before a wait gives up
@@ -103,7 +103,7 @@ __device__ __forceinline__ void emit_row(const KParams &P, const RowCfg &c, int 
 #define MERGE_STAMP(i) do { } while (0)
 #endif
 
-constexpr int RANK_SORT_MAX = 1024;           // at most this many candidates: sort by rank counting
+constexpr int RANK_SORT_MAX = 512;            // at most this many candidates: sort by rank counting
 constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
 struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
 
@@ -175,6 +175,89 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     else if (complete && P.op != OP_TOPK) n = Pn;
     else return false;
     unsigned long long *sorted = buf;
+    int Pn2 = Pn;
+    if (n >= 64 && Pn > n + n / 2 + 64) {
+        // far more proven candidates than needed: bisect a key threshold that keeps between n and
+        // about next_pow2(n) of them (any such threshold keeps the n best), then sort only those
+        const int want_hi = max(next_pow2(n), n + n / 8);
+        unsigned long long lo = 0ull, hi = ~0ull;          // count(>= lo) >= n > count(>= hi)
+        {
+            // start from the range the keys actually span
+            unsigned long long mn = ~0ull, mx = 0ull;
+            for (int i = tid; i < Pn; i += THREADS) { mn = min(mn, buf[i]); mx = max(mx, buf[i]); }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                mn = min(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+                mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+            }
+            unsigned long long *red = reinterpret_cast<unsigned long long *>(sh.scratch);
+            if ((tid & 31) == 0) { red[tid >> 5] = mn; red[THREADS / 32 + (tid >> 5)] = mx; }
+            csync();
+            for (int w = 0; w < THREADS / 32; ++w) { mn = min(mn, red[w]); mx = max(mx, red[THREADS / 32 + w]); }
+            csync();
+            lo = mn; hi = mx + 1ull;
+        }
+        MERGE_STAMP(11);
+        // eight-way search: seven interior thresholds per pass, one reduction for all of them
+        for (int it = 0; it < 24 && hi - lo > 1ull; ++it) {
+            const unsigned long long step = (hi - lo) >> 3;
+            unsigned long long th[7];
+#pragma unroll
+            for (int q = 0; q < 7; ++q) th[q] = (step > 0) ? lo + step * (q + 1) : min(hi - 1ull, lo + 1ull + q);
+            int cnt[7] = {0, 0, 0, 0, 0, 0, 0};
+            for (int i = tid; i < Pn; i += THREADS) {
+                const unsigned long long key = buf[i];
+#pragma unroll
+                for (int q = 0; q < 7; ++q) cnt[q] += (key >= th[q]) ? 1 : 0;
+            }
+            int *redi = reinterpret_cast<int *>(sh.scratch);
+#pragma unroll
+            for (int q = 0; q < 7; ++q) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) cnt[q] += __shfl_xor_sync(0xFFFFFFFFu, cnt[q], off);
+                if ((tid & 31) == 0) redi[(tid >> 5) * 8 + q] = cnt[q];
+            }
+            csync();
+            bool done = false;
+#pragma unroll
+            for (int q = 6; q >= 0; --q) {                 // the highest threshold that still keeps n
+                int tot = 0;
+                for (int w = 0; w < THREADS / 32; ++w) tot += redi[w * 8 + q];
+                if (!done && tot >= n) {
+                    lo = th[q];
+                    if (q < 6) hi = th[q + 1];
+                    done = true;
+                    if (tot <= want_hi) it = 1000;          // tight enough
+                }
+            }
+            if (!done) hi = th[0];
+            csync();
+        }
+        // keep the keys >= lo, packed to the front (every position written is at or below one already read)
+        if (tid == 0) sh.count = 0;
+        csync();
+        for (int i0 = 0; i0 < Pn; i0 += THREADS) {
+            const int i = i0 + tid;
+            const unsigned long long key = (i < Pn) ? buf[i] : 0ull;
+            const bool keep = (i < Pn) && key >= lo;
+            const unsigned int mk = __ballot_sync(0xFFFFFFFFu, keep);
+            csync();                                        // all reads of this trip precede its writes
+            int base = 0;
+            if ((tid & 31) == 0 && mk) base = atomicAdd(&sh.count, __popc(mk));
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if (keep) buf[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
+            csync();
+        }
+        Pn2 = sh.count;
+        csync();
+    }
+    MERGE_STAMP(12);
+#ifdef SONIC_TRACE
+    if (tid == 0 && row == (int)P.error[4]) P.error[29] = Pn2;
+#endif
+    const int PnAll = Pn;
+    (void)PnAll;
+#define Pn Pn2
     if (Pn <= RANK_SORT_MAX) {
         // few candidates: each key counts the keys above it (keys are distinct) and lands at its rank
         unsigned long long *dst = buf + MERGE_CAP / 2;
@@ -194,6 +277,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         bitonic_sort_desc<THREADS, Sync>(buf, m, tid);
     }
     (void)sorted;
+#undef Pn
     MERGE_STAMP(3);
 #ifdef SONIC_TRACE
     if (tid == 0 && row == (int)P.error[4]) { P.error[30] = Pn; P.error[31] = n; }
@@ -347,7 +431,7 @@ struct StreamShared {
 };
 
 template <int DT>
-__global__ void __launch_bounds__(STREAM_CTA_THREADS, 2)
+__global__ void __launch_bounds__(STREAM_CTA_THREADS, 3)
 sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
     constexpr int VEC = VecTraits<DT>::VEC, NV = VecTraits<DT>::NV, NSTAGE = VecTraits<DT>::NSTAGE;
     constexpr int ELT = VecTraits<DT>::ELT;
@@ -365,6 +449,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_launch_dependents();                   // the merge kernel may start launching; it waits for this grid to finish
 
     if (warp == STREAM_WARPS) {
         // ------------------------------------------------------------ producer warp
@@ -644,8 +729,10 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     __shared__ MergeShared<MERGE_THREADS> s_merge;
     const int row = blockIdx.x;
     const int tid = threadIdx.x;
-    const RowCfg c = load_cfg(P, row);
+    pdl_launch_dependents();                   // the exact kernel may start on the rows that are its own by class
+    const RowCfg c = load_cfg(P, row);         // inputs only: independent of the streaming kernel
     if (c.cls == CLS_EXACT) return;
+    pdl_wait_primary();                        // tile records and candidates of the streaming kernel
     RowState *rs = P.rs + row;
     const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
     const unsigned int status = rs->status;
