@@ -491,17 +491,12 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
         const int row = item / tiles, tile = item - row * tiles;
         const int tile_base = tile * CTA_TILE;
         const int wbase = tile_base + warp * WARP_TILE;
-        // requests that depend only on (row, tile) go out before the wait
-        uint32_t mw[NV];
+        // requests that depend only on (row, tile) go out before the wait: the warp tile's 32 grammar
+        // words in one coalesced load (handed to the lanes that need them by shuffles later)
+        uint32_t mword = 0xFFFFFFFFu;
         if (P.bitmask) {
-            const uint32_t *mrow = P.bitmask + (size_t)row * P.bitmask_stride;
-            const int nwords = (P.V + 31) >> 5;
-#pragma unroll
-            for (int j = 0; j < NV; ++j) {
-                const int first = wbase + j * 32 * VEC + lane * VEC;
-                const int w = first >> 5;
-                mw[j] = ((w < nwords) ? __ldg(mrow + w) : 0u) >> (first & 31);
-            }
+            const int w = (wbase >> 5) + lane;
+            mword = (w < ((P.V + 31) >> 5)) ? __ldg(P.bitmask + (size_t)row * P.bitmask_stride + w) : 0u;
         }
         // the first entries of the row's sparse lists as well (lengths are checked once the configuration is known)
         const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
@@ -594,13 +589,22 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
             } else {
                 read_raw();
             }
-            if (masked || tail) {
+            if (masked && !tail) {
+                // the common masked case: one select per element, no bounds test
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const uint32_t bits = __shfl_sync(0xFFFFFFFFu, mword, (j * 32 * VEC + lane * VEC) >> 5) >> ((lane * VEC) & 31);
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) e[j * VEC + q] = (bits & (1u << q)) ? e[j * VEC + q] : -CUDART_INF_F;
+                }
+            } else if (tail) {
 #pragma unroll
                 for (int j = 0; j < NV; ++j) {
                     const int first = wbase + j * 32 * VEC + lane * VEC;
+                    const uint32_t bits = __shfl_sync(0xFFFFFFFFu, mword, (j * 32 * VEC + lane * VEC) >> 5) >> (first & 31);
 #pragma unroll
                     for (int q = 0; q < VEC; ++q) {
-                        const bool dead = (tail && first + q >= P.V) || (masked && !((mw[j] >> q) & 1u));
+                        const bool dead = (first + q >= P.V) || (masked && !((bits >> q) & 1u));
                         if (dead) e[j * VEC + q] = -CUDART_INF_F;
                     }
                 }
