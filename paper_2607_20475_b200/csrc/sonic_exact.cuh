@@ -48,6 +48,7 @@ struct ExactShared {
     unsigned long long xch[2][CL][XV];
     unsigned long long vals[XV];
     unsigned long long wtot[EX_WARPS];
+    unsigned long long wcnt[EX_WARPS];
     unsigned long long red_mass[HBINS / CL];
     unsigned int red_cnt[HBINS / CL];
     unsigned int ucount;
@@ -126,76 +127,122 @@ __device__ __forceinline__ unsigned long long qweight(uint32_t key, float Mf) {
     return __float2ull_rn(w * 1099511627776.0f);
 }
 
-// Ordered crossing: elements are visited in vocabulary-index order (warp w owns a
-// contiguous run of the slice, lanes interleaved), each with weight wf(local index).
-// Computes the row total and, if want_cross, the first element whose inclusive
-// running sum exceeds `target` over the whole row (its global index, -1 if
-// none).  Results are identical in every CTA.  T is a 64-bit type.
-template <typename T, typename WF>
-__device__ int ordered_cross(ExactCtx &x, T target, bool want_cross, WF wf, T &total_out) {
+// Ordered passes: elements are visited in vocabulary-index order (warp w owns a
+// contiguous run of the slice, lanes interleaved), each with weight wf(local index)
+// of a 64-bit type T (fixed-point mass, a count, or fp64).
+template <typename T>
+struct OrderedState {
+    T cta_off;            // sum over the CTAs before this one
+    T warp_off;           // sum over this CTA's warps before this warp
+    T total;              // row total
+    T cta_tot[CL];        // per-CTA totals
+};
+
+// Row total of wf (and of the 0/1 indicator cf, returned in count_out); leaves the per-warp totals of wf in
+// shared memory for a following ordered_find.  One cluster barrier.
+template <typename T, typename WF, typename CF>
+__device__ void ordered_totals(ExactCtx &x, WF wf, CF cf, OrderedState<T> &st, unsigned long long &count_out) {
     const int wch = x.per / EX_WARPS;                    // elements per warp (multiple of 32)
     const int wlo = x.warp * wch;
     T wt = T(0);
-    for (int i = wlo + x.lane; i < wlo + wch; i += 32) wt += wf(i);
+    unsigned long long cn = 0;
+#pragma unroll 4
+    for (int i = wlo + x.lane; i < wlo + wch; i += 32) { wt += wf(i); cn += cf(i); }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) wt += __shfl_xor_sync(0xFFFFFFFFu, wt, off);
-    __syncthreads();
-    if (x.lane == 0) x.sh->wtot[x.warp] = *reinterpret_cast<unsigned long long *>(&wt);
-    __syncthreads();
-    T cta_total = T(0), my_woff = T(0);
-    for (int w = 0; w < EX_WARPS; ++w) {
-        T v = *reinterpret_cast<T *>(&x.sh->wtot[w]);
-        if (w == x.warp) my_woff = cta_total;
-        cta_total += v;
+    for (int off = 16; off > 0; off >>= 1) {
+        wt += __shfl_xor_sync(0xFFFFFFFFu, wt, off);
+        cn += __shfl_xor_sync(0xFFFFFFFFu, cn, off);
     }
-    unsigned long long v[XV] = {*reinterpret_cast<unsigned long long *>(&cta_total), 0, 0, 0};
+    __syncthreads();
+    if (x.lane == 0) { x.sh->wtot[x.warp] = *reinterpret_cast<unsigned long long *>(&wt); x.sh->wcnt[x.warp] = cn; }
+    __syncthreads();
+    T cta_total = T(0);
+    unsigned long long cta_cnt = 0;
+    st.warp_off = T(0);
+    for (int w = 0; w < EX_WARPS; ++w) {
+        const T v = *reinterpret_cast<T *>(&x.sh->wtot[w]);
+        if (w == x.warp) st.warp_off = cta_total;
+        cta_total += v;
+        cta_cnt += x.sh->wcnt[w];
+    }
+    unsigned long long v[XV] = {*reinterpret_cast<unsigned long long *>(&cta_total), cta_cnt, 0, 0};
     unsigned long long all[CL][XV];
     allgather(x, v, all);
-    T off = T(0), total = T(0);
-    int cross_rank = -1;
+    st.total = T(0);
+    st.cta_off = T(0);
+    count_out = 0;
     for (int r = 0; r < CL; ++r) {
-        T t = *reinterpret_cast<T *>(&all[r][0]);
-        if (r == x.rank) off = total;
-        if (cross_rank < 0 && total + t > target) cross_rank = r;
-        total += t;
+        const T t = *reinterpret_cast<T *>(&all[r][0]);
+        st.cta_tot[r] = t;
+        if (r == x.rank) st.cta_off = st.total;
+        st.total += t;
+        count_out += all[r][1];
     }
-    total_out = total;
-    if (!want_cross) return -1;
+}
+
+// First element (index order) whose inclusive running sum of wf exceeds `target`; uses the warp totals left by
+// ordered_totals for the same wf.  Returns its global index (-1 if none) and its weight, in every CTA.  One
+// cluster barrier.
+template <typename T, typename WF>
+__device__ int ordered_find(ExactCtx &x, T target, WF wf, const OrderedState<T> &st, T &weight_out) {
+    const int wch = x.per / EX_WARPS;
+    const int wlo = x.warp * wch;
+    int cross_rank = -1;
+    {
+        T acc = T(0);
+        for (int r = 0; r < CL; ++r) {
+            if (cross_rank < 0 && acc + st.cta_tot[r] > target) cross_rank = r;
+            acc += st.cta_tot[r];
+        }
+    }
     if (cross_rank == x.rank) {
         int cross_warp = -1;
-        T acc = off;
+        T acc = st.cta_off;
         for (int w = 0; w < EX_WARPS; ++w) {
-            T v2 = *reinterpret_cast<T *>(&x.sh->wtot[w]);
+            const T v2 = *reinterpret_cast<T *>(&x.sh->wtot[w]);
             if (cross_warp < 0 && acc + v2 > target) cross_warp = w;
             acc += v2;
         }
         if (cross_warp < 0) cross_warp = EX_WARPS - 1;    // rounding between levels
         if (x.warp == cross_warp) {
-            T run = off + my_woff;
+            T run = st.cta_off + st.warp_off;
             int found = -1, last_member = -1;
+            T fw = T(0), lw = T(0);
             for (int i = wlo; i < wlo + wch; i += 32) {
-                T wv = wf(i + x.lane);
+                const T wv = wf(i + x.lane);
                 T incl = wv;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    const T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
                     if (x.lane >= o) incl += up;
                 }
-                unsigned int hit = __ballot_sync(0xFFFFFFFFu, (run + incl > target) && (wv > T(0)));
-                unsigned int pos = __ballot_sync(0xFFFFFFFFu, wv > T(0));
-                if (hit) { found = x.lo + i + (__ffs(hit) - 1); break; }
-                if (pos) last_member = x.lo + i + (31 - __clz(pos));
+                const unsigned int hit = __ballot_sync(0xFFFFFFFFu, (run + incl > target) && (wv > T(0)));
+                const unsigned int pos = __ballot_sync(0xFFFFFFFFu, wv > T(0));
+                if (hit) {
+                    const int l = __ffs(hit) - 1;
+                    found = x.lo + i + l;
+                    fw = __shfl_sync(0xFFFFFFFFu, wv, l);
+                    break;
+                }
+                if (pos) {
+                    const int l = 31 - __clz(pos);
+                    last_member = x.lo + i + l;
+                    lw = __shfl_sync(0xFFFFFFFFu, wv, l);
+                }
                 run += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
-            if (found < 0) found = last_member;            // rounding between levels: last positive element
-            if (x.lane == 0) x.sh->flag = found;
+            if (found < 0) { found = last_member; fw = lw; }   // rounding between levels: last positive element
+            if (x.lane == 0) { x.sh->flag = found; x.sh->vals[3] = *reinterpret_cast<unsigned long long *>(&fw); }
         }
     }
     __syncthreads();
     unsigned long long v2[XV] = {0, 0, 0, 0};
-    if (cross_rank == x.rank) v2[0] = (unsigned long long)(long long)x.sh->flag;
+    if (cross_rank == x.rank) { v2[0] = (unsigned long long)(long long)x.sh->flag; v2[1] = x.sh->vals[3]; }
+    unsigned long long all[CL][XV];
     allgather(x, v2, all);
+    weight_out = T(0);
     if (cross_rank < 0) return -1;
+    weight_out = *reinterpret_cast<T *>(&all[cross_rank][1]);
     return (int)(long long)all[cross_rank][0];
 }
 
@@ -208,10 +255,11 @@ __device__ int ordered_cross(ExactCtx &x, T target, bool want_cross, WF wf, T &t
 // ceil(p * total mass) first.  Two cluster barriers.
 template <typename DF>
 __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first, float p, int nbins, DF digit,
-                          unsigned long long &target, unsigned long long &in_bin) {
+                          unsigned long long &target, unsigned long long &in_bin, unsigned long long *stg) {
     for (int i = x.tid; i < nbins; i += EX_THREADS) { x.hcnt[i] = 0; x.hm0[i] = 0; x.hm1[i] = 0; x.hm2[i] = 0; }
     __syncthreads();
-    for (int i0 = 0; i0 < x.len; i0 += EX_THREADS) {
+#pragma unroll 4
+    for (int i0 = 0; i0 < x.per; i0 += EX_THREADS) {
         const int i = i0 + x.tid;
         int bin = -1;
         uint32_t key = 0;
@@ -233,29 +281,61 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
             if (by_mass) { q0 = __reduce_add_sync(active, q0); q1 = __reduce_add_sync(active, q1); q2 = __reduce_add_sync(active, q2); }
             if ((int)(__ffs(active) - 1) == x.lane) {
                 atomicAdd(&x.hcnt[bin], n);
-                if (by_mass) { atomicAdd(&x.hm0[bin], q0); atomicAdd(&x.hm1[bin], q1); atomicAdd(&x.hm2[bin], q2); }
+                if (q0) atomicAdd(&x.hm0[bin], q0);
+                if (q1) atomicAdd(&x.hm1[bin], q1);
+                if (q2) atomicAdd(&x.hm2[bin], q2);
             }
         } else {
             atomicAdd(&x.hcnt[bin], 1u);
-            if (by_mass) { atomicAdd(&x.hm0[bin], q0); atomicAdd(&x.hm1[bin], q1); atomicAdd(&x.hm2[bin], q2); }
+            if (q0) atomicAdd(&x.hm0[bin], q0);            // small weights leave the upper limbs untouched
+            if (q1) atomicAdd(&x.hm1[bin], q1);
+            if (q2) atomicAdd(&x.hm2[bin], q2);
         }
     }
+    if (first) SONIC_STAMP(17);
     cg::this_cluster().sync();
-    // CTA r reduces bins [r*bpr, (r+1)*bpr) over the cluster
+    if (first) SONIC_STAMP(18);
+    // CTA r reduces bins [r*bpr, (r+1)*bpr) over the cluster.  Remote shared-memory reads are slow, so
+    // all of them are issued at once: thread t fetches (bin, rank) pairs t, t + EX_THREADS, ... into a
+    // local staging area (the sort buffer, idle during histogram levels), then the owners add locally.
     const int bpr = nbins / CL;
-    unsigned long long sc = 0, sm = 0;
-    if (x.tid < bpr) {
-        const int bin = x.rank * bpr + x.tid;
-        unsigned int cc = 0;
-        unsigned long long mm = 0;
-        for (int r = 0; r < CL; ++r) {
-            cc += *cg::this_cluster().map_shared_rank(&x.hcnt[bin], r);
-            if (by_mass) {
-                mm += (unsigned long long)*cg::this_cluster().map_shared_rank(&x.hm0[bin], r)
-                    + ((unsigned long long)*cg::this_cluster().map_shared_rank(&x.hm1[bin], r) << 14)
-                    + ((unsigned long long)*cg::this_cluster().map_shared_rank(&x.hm2[bin], r) << 28);
+    unsigned int *stg_cnt = reinterpret_cast<unsigned int *>(stg);                    // [CL][bpr]
+    unsigned long long *stg_mass = stg + (CL * (HBINS / CL)) / 2;                       // [CL][bpr]
+    {
+        constexpr int TRIPS = (CL * (HBINS / CL) + EX_THREADS - 1) / EX_THREADS;       // 4
+        unsigned int cc[TRIPS], a0[TRIPS], a1[TRIPS], a2[TRIPS];
+#pragma unroll
+        for (int u = 0; u < TRIPS; ++u) {
+            const int pair = x.tid + u * EX_THREADS;
+            const int r = pair / bpr, bl = pair - r * bpr;
+            cc[u] = a0[u] = a1[u] = a2[u] = 0;
+            if (r < CL) {
+                const int bin = x.rank * bpr + bl;
+                cc[u] = *cg::this_cluster().map_shared_rank(&x.hcnt[bin], r);
+                if (by_mass) {
+                    a0[u] = *cg::this_cluster().map_shared_rank(&x.hm0[bin], r);
+                    a1[u] = *cg::this_cluster().map_shared_rank(&x.hm1[bin], r);
+                    a2[u] = *cg::this_cluster().map_shared_rank(&x.hm2[bin], r);
+                }
             }
         }
+#pragma unroll
+        for (int u = 0; u < TRIPS; ++u) {
+            const int pair = x.tid + u * EX_THREADS;
+            const int r = pair / bpr, bl = pair - r * bpr;
+            if (r < CL) {
+                stg_cnt[r * bpr + bl] = cc[u];
+                stg_mass[r * bpr + bl] = (unsigned long long)a0[u] + ((unsigned long long)a1[u] << 14) + ((unsigned long long)a2[u] << 28);
+            }
+        }
+    }
+    __syncthreads();
+    unsigned long long sc = 0, sm = 0;
+    if (x.tid < bpr) {
+        unsigned int cc = 0;
+        unsigned long long mm = 0;
+#pragma unroll
+        for (int r = 0; r < CL; ++r) { cc += stg_cnt[r * bpr + x.tid]; mm += stg_mass[r * bpr + x.tid]; }
         x.sh->red_cnt[x.tid] = cc;
         x.sh->red_mass[x.tid] = mm;
         sc = cc; sm = mm;
@@ -265,6 +345,7 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
     unsigned long long v[XV] = {sc, sm, 0, 0};
     unsigned long long all[CL][XV];
     allgather(x, v, all);                      // every remote histogram read precedes this barrier
+    if (first) SONIC_STAMP(19);
     if (by_mass && first) {
         unsigned long long Zq = 0;
         for (int r = 0; r < CL; ++r) Zq += all[r][1];
@@ -290,15 +371,26 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
     const unsigned int *rc = cg::this_cluster().map_shared_rank(&x.sh->red_cnt[0], seg);
     const unsigned long long *rm = cg::this_cluster().map_shared_rank(&x.sh->red_mass[0], seg);
     if (x.tid < 32) {
-        // warp 0: lanes take bins from the top in chunks of 32
+        // warp 0: lanes take bins from the top in chunks of 32; all remote reads are issued before the scan
+        constexpr int CH = (HBINS / CL) / 32;        // 8 chunks at most
+        unsigned long long pv[CH];
+        unsigned int pc[CH];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {
+            const int t = bpr - 1 - ch * 32 - x.lane;
+            pv[ch] = 0; pc[ch] = 0;
+            if (t >= 0) { pc[ch] = rc[t]; pv[ch] = by_mass ? rm[t] : (unsigned long long)pc[ch]; }
+        }
         unsigned long long c2 = cum;
         int found = -1;
         unsigned long long rest = 0, cnt = 0;
-        for (int top = bpr - 1; top >= 0 && found < 0; top -= 32) {
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {
+            const int top = bpr - 1 - ch * 32;
+            if (top < 0 || found >= 0) continue;
             const int t = top - x.lane;
-            unsigned long long val = 0;
-            unsigned int cval = 0;
-            if (t >= 0) { cval = rc[t]; val = by_mass ? rm[t] : (unsigned long long)cval; }
+            const unsigned long long val = pv[ch];
+            const unsigned int cval = pc[ch];
             unsigned long long incl = val;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -331,6 +423,7 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
 }
 
 constexpr int GATHER_CAP = MAX_TOPK;          // elements CTA 0 can sort
+constexpr int GATHER_FAST = 256;              // above this many elements in the crossing bin a second level pays off
 
 // Selection inside `base`:
 //   by_mass == false: the cut of the `need`-th largest element (1 <= need <= count inside base)
@@ -347,7 +440,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         float t = fminf(__fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f), 2047.0f);
         return 2047 - (int)t;
     };
-    const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin);
+    const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin, sortbuf);
     SONIC_STAMP(4);
     auto dig_b = [&](uint32_t key) -> int {
         float t = __fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f);
@@ -357,34 +450,36 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         return 2047 - (int)f;
     };
     int b = -1;
-    if (in_bin > (unsigned long long)GATHER_CAP) b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin);
+    if (in_bin > (unsigned long long)GATHER_FAST) b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin, sortbuf);
     SONIC_STAMP(5);
     auto in_range = [&](uint32_t key) -> bool {
         if (dig_a(key) != a) return false;
         return b < 0 || dig_b(key) == b;
     };
     if (in_bin <= (unsigned long long)GATHER_CAP) {
-        // gather the bin into CTA 0, sort it there, pick the element that completes the target
+        // every CTA packs its elements of the bin into its own list, then the lists are laid end to end in
+        // CTA 0, which sorts them and picks the element that completes the target
         if (x.tid == 0) x.sh->ucount = 0;
         __syncthreads();
-        unsigned long long cnt = 0;
-        for (int i = x.tid; i < x.len; i += EX_THREADS) {
-            uint32_t key = x.keys[i];
-            cnt += (member(base, key, x.lo + i) && in_range(key)) ? 1 : 0;
+#pragma unroll 4
+        for (int i0 = 0; i0 < x.per; i0 += EX_THREADS) {
+            const int i = i0 + x.tid;
+            const uint32_t key = (i < x.len) ? x.keys[i] : 0u;
+            const bool want = (i < x.len) && member(base, key, x.lo + i) && in_range(key);
+            const unsigned int pos = warp_append(&x.sh->ucount, want, x.lane);
+            if (want && pos < (unsigned int)GATHER_CAP) sortbuf[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
         }
-        cnt = block_sum_u64(x, cnt);
-        unsigned long long v[XV] = {cnt, 0, 0, 0};
+        __syncthreads();
+        const unsigned int mine = min(x.sh->ucount, (unsigned int)GATHER_CAP);
+        unsigned long long v[XV] = {mine, 0, 0, 0};
         unsigned long long all[CL][XV];
         allgather(x, v, all);
         unsigned int off = 0, n = 0;
         for (int r = 0; r < CL; ++r) { if (r < x.rank) off += (unsigned int)all[r][0]; n += (unsigned int)all[r][0]; }
-        unsigned long long *dst = cg::this_cluster().map_shared_rank(sortbuf, 0);
-        for (int i0 = 0; i0 < x.len; i0 += EX_THREADS) {
-            const int i = i0 + x.tid;
-            const uint32_t key = (i < x.len) ? x.keys[i] : 0u;
-            const bool want = (i < x.len) && member(base, key, x.lo + i) && in_range(key);
-            const unsigned int pos = off + warp_append(&x.sh->ucount, want, x.lane);
-            if (want && pos < (unsigned int)GATHER_CAP) dst[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+        if (x.rank != 0) {                      // CTA 0's own entries already sit at the front of its buffer
+            unsigned long long *dst = cg::this_cluster().map_shared_rank(sortbuf, 0);
+            for (unsigned int i = x.tid; i < mine; i += EX_THREADS)
+                if (off + i < (unsigned int)GATHER_CAP) dst[off + i] = sortbuf[i];
         }
         cg::this_cluster().sync();
         SONIC_STAMP(6);
@@ -442,7 +537,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
             if (!in_range(key)) return -1;
             return (int)((key >> shift) & ((1u << nb) - 1u));
         };
-        const int d = hist_level(x, base, by_mass, false, p, 1 << nb, dig_k, target, in_bin);
+        const int d = hist_level(x, base, by_mass, false, p, 1 << nb, dig_k, target, in_bin, sortbuf);
         prefix = (prefix << nb) | (uint32_t)d;
         pbits += nb;
     }
@@ -455,13 +550,13 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     if (r < 1) r = 1;
     if (r > in_bin) r = in_bin;
     const uint32_t v = prefix;
-    unsigned long long tot;
-    int idx = ordered_cross<unsigned long long>(
-        x, r - 1, true,
-        [&](int i) -> unsigned long long {
-            return (i < x.len && x.keys[i] == v && member(base, v, x.lo + i)) ? 1ull : 0ull;
-        },
-        tot);
+    auto tie = [&](int i) -> unsigned long long {
+        return (i < x.len && x.keys[i] == v && member(base, v, x.lo + i)) ? 1ull : 0ull;
+    };
+    OrderedState<unsigned long long> st;
+    unsigned long long ntie, wdummy;
+    ordered_totals<unsigned long long>(x, tie, tie, st, ntie);
+    const int idx = ordered_find<unsigned long long>(x, r - 1, tie, st, wdummy);
     Cut c;
     c.v = v;
     c.idx = idx;
@@ -652,30 +747,25 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         Cut cm; cm.v = tk - 1; cm.idx = -1;                // key >= tk
         if (tighter(cm, cut)) cut = cm;
     }
-    // final support: size, mass, draw in index order
-    unsigned long long cnt = 0;
-    for (int i = x.tid; i < x.len; i += EX_THREADS) cnt += member(cut, x.keys[i], x.lo + i) ? 1 : 0;
-    cnt = block_sum_u64(x, cnt);
-    {
-        unsigned long long v[XV] = {cnt, 0, 0, 0};
-        allgather(x, v, all);
-    }
-    unsigned long long nS = 0;
-    for (int r = 0; r < CL; ++r) nS += all[r][0];
-
+    // final support: size and mass in one ordered pass, then the draw in index order
     uint32_t a_acc, a_draw;
     draw_cells(P, c, a_acc, a_draw);
     auto wq = [&](int i) -> unsigned long long {
         return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? qweight(x.keys[i], x.Mf) : 0ull;
     };
-    // total mass first (target depends on it): a crossing search with an unreachable target
-    unsigned long long Wq;
-    ordered_cross<unsigned long long>(x, ~0ull, false, wq, Wq);
+    auto inS = [&](int i) -> unsigned long long {
+        return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? 1ull : 0ull;
+    };
+    OrderedState<unsigned long long> stq;
+    unsigned long long nS;
+    ordered_totals<unsigned long long>(x, wq, inS, stq, nS);
+    const unsigned long long Wq = stq.total;
     SONIC_STAMP(10);
     const unsigned long long mul = 2ull * a_draw + 1ull;               // u = mul / 2^25
     const unsigned long long T = (__umul64hi(Wq, mul) << 39) | ((Wq * mul) >> 25);
-    unsigned long long dummy;
-    int token = ordered_cross<unsigned long long>(x, T, true, wq, dummy);
+    unsigned long long qt = 0;
+    int token = ordered_find<unsigned long long>(x, T, wq, stq, qt);
+    double token_prob = (double)qt / (double)Wq;
     SONIC_STAMP(11);
 
     uint32_t flags = F_FALLBACK;
@@ -693,37 +783,31 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);
         p_draft = (float)Pd;
         if (accept) flags |= F_ACCEPT;
-        // residual max(0, p - q) over the support, weights in fp64
+        // residual max(0, p - q) over the support, weights in fp64 (p - q cancels, so the weights must be accurate)
         const double Md = (double)x.Mf;
         auto wd = [&](int i) -> double {
             return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? exp((double)unkey(x.keys[i]) - Md) : 0.0;
         };
-        double Wd;
-        ordered_cross<double>(x, CUDART_INF, false, wd, Wd);
+        OrderedState<double> std_;
+        unsigned long long cdummy;
+        ordered_totals<double>(x, wd, inS, std_, cdummy);
+        const double Wd = std_.total;
         auto rd = [&](int i) -> double {
             if (!(i < x.len && member(cut, x.keys[i], x.lo + i))) return 0.0;
             double r = exp((double)unkey(x.keys[i]) - Md) / Wd - (double)__ldg(q + x.lo + i);
             return r > 0.0 ? r : 0.0;
         };
-        double R;
-        ordered_cross<double>(x, CUDART_INF, false, rd, R);
-        if (R > 0.0) {
-            double dummy2;
-            int t2 = ordered_cross<double>(x, cell_to_u(a_draw) * R, true, rd, dummy2);
-            if (t2 >= 0) token = t2;
+        OrderedState<double> str;
+        ordered_totals<double>(x, rd, inS, str, cdummy);
+        if (str.total > 0.0) {
+            double rw;
+            const int t2 = ordered_find<double>(x, cell_to_u(a_draw) * str.total, rd, str, rw);
+            if (t2 >= 0) token = t2;           // (verification rows report p(d), not the probability of this token)
         }
     }
-    // probability of the chosen token under the final distribution
-    {
-        unsigned long long v[XV] = {0, 0, 0, 0};
-        if (token >= x.lo && token < x.lo + x.len) v[0] = wq(token - x.lo) + 1ull;
-        allgather(x, v, all);
-        unsigned long long qt = 0;
-        for (int r = 0; r < CL; ++r) if (all[r][0]) qt = all[r][0] - 1ull;
-        if (leader) {
-            emit_row(P, c, row, token, (float)((double)qt / (double)Wq), flags, (int)nS, p_draft);
-            rs->status = 0;
-        }
+    if (leader) {
+        emit_row(P, c, row, token, (float)token_prob, flags, (int)nS, p_draft);
+        rs->status = 0;
     }
     cg::this_cluster().sync();
 }

@@ -142,29 +142,107 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     const bool strict = c.temp && !complete;            // keys are compared after the temperature division
     const uint32_t tykey = c.temp ? okey(__fdiv_rn(unkey(tkey), c.tau)) : tkey;
     const int total = sh.tcnt[tiles];
-    for (int j0 = 0; j0 < total; j0 += THREADS) {
-        const int j = j0 + tid;
-        bool keep = false;
-        unsigned long long out = 0ull;
-        if (j < total) {
-            int t = 0;
-            while (sh.tcnt[t + 1] <= j) ++t;
-            const unsigned long long cd = __ldcg(P.cand + (size_t)row * CAND_CAP + (size_t)t * cap_t + (j - sh.tcnt[t]));
-            const uint32_t zk = (uint32_t)(cd >> 32);
-            uint32_t yk = zk;
-            if (c.temp) yk = okey(__fdiv_rn(unkey(zk), c.tau));
-            keep = (zk >= tkey) && !(strict && yk <= tykey);
-            out = ((unsigned long long)yk << 32) | (uint32_t)cd;
+    // candidates are fetched eight per thread at a time (independent loads), then filtered and packed
+    constexpr int GB = 8;
+    auto fetch = [&](int j0, unsigned long long (&cd)[GB]) {
+#pragma unroll
+        for (int u = 0; u < GB; ++u) {
+            const int j = j0 + u * THREADS + tid;
+            cd[u] = 0ull;
+            if (j < total) {
+                int t = 0;
+                while (sh.tcnt[t + 1] <= j) ++t;
+                cd[u] = __ldcg(P.cand + (size_t)row * CAND_CAP + (size_t)t * cap_t + (j - sh.tcnt[t]));
+            }
         }
-        // one shared-memory atomic per warp, not per candidate
-        const unsigned int m = __ballot_sync(0xFFFFFFFFu, keep);
-        int base = 0;
-        if ((tid & 31) == 0 && m) base = atomicAdd(&sh.count, __popc(m));
-        base = __shfl_sync(0xFFFFFFFFu, base, 0);
-        if (keep) {
-            const int pos = base + __popc(m & ((1u << (tid & 31)) - 1u));
-            if (pos < MERGE_CAP) buf[pos] = out;
+    };
+    // proven candidate -> its key after the temperature division (0 if it is not proven)
+    auto proven_key = [&](unsigned long long cd, int j) -> unsigned long long {
+        const uint32_t zk = (uint32_t)(cd >> 32);
+        uint32_t yk = zk;
+        if (c.temp) yk = okey(__fdiv_rn(unkey(zk), c.tau));
+        const bool keep = (j < total) && (zk >= tkey) && !(strict && yk <= tykey);
+        return keep ? (((unsigned long long)yk << 32) | (uint32_t)cd) : 0ull;
+    };
+    unsigned long long floor_key = 1ull;           // keys below it are left out (1: every proven candidate)
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        unsigned long long kmax = 0ull;
+        for (int j0 = 0; j0 < total; j0 += GB * THREADS) {
+            unsigned long long cd[GB];
+            fetch(j0, cd);
+#pragma unroll
+            for (int u = 0; u < GB; ++u) {
+                if (j0 + u * THREADS >= total) break;              // uniform over the CTA
+                const unsigned long long out = proven_key(cd[u], j0 + u * THREADS + tid);
+                const bool keep = out >= floor_key;
+                kmax = max(kmax, out);
+                // one shared-memory atomic per warp, not per candidate
+                const unsigned int m = __ballot_sync(0xFFFFFFFFu, keep);
+                int base = 0;
+                if ((tid & 31) == 0 && m) base = atomicAdd(&sh.count, __popc(m));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (keep) {
+                    const int pos = base + __popc(m & ((1u << (tid & 31)) - 1u));
+                    if (pos < MERGE_CAP) buf[pos] = out;
+                }
+            }
         }
+        csync();
+        if (attempt == 1 || sh.count <= MERGE_CAP || sh.count < c.k) break;
+        // More proven candidates than the buffer holds (large k): find a key floor that keeps between k and
+        // MERGE_CAP of them by an eight-way search over the candidates in global memory, then pack again.
+        unsigned long long *red = reinterpret_cast<unsigned long long *>(sh.scratch);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, off));
+        if ((tid & 31) == 0) red[tid >> 5] = kmax;
+        csync();
+        for (int w = 0; w < THREADS / 32; ++w) kmax = max(kmax, red[w]);
+        csync();
+        unsigned long long lo = 1ull, hi = kmax + 1ull;              // count(>= lo) >= k > ... count(>= hi) = 0
+        for (int it = 0; it < 24 && hi - lo > 1ull; ++it) {
+            const unsigned long long step = (hi - lo) >> 3;
+            unsigned long long th[7];
+#pragma unroll
+            for (int q = 0; q < 7; ++q) th[q] = (step > 0) ? lo + step * (q + 1) : min(hi - 1ull, lo + 1ull + q);
+            int cnt[7] = {0, 0, 0, 0, 0, 0, 0};
+            for (int j0 = 0; j0 < total; j0 += GB * THREADS) {
+                unsigned long long cd[GB];
+                fetch(j0, cd);
+#pragma unroll
+                for (int u = 0; u < GB; ++u) {
+                    const unsigned long long out = proven_key(cd[u], j0 + u * THREADS + tid);
+#pragma unroll
+                    for (int q = 0; q < 7; ++q) cnt[q] += (out >= th[q]) ? 1 : 0;
+                }
+            }
+            int *redi = reinterpret_cast<int *>(sh.scratch);
+#pragma unroll
+            for (int q = 0; q < 7; ++q) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) cnt[q] += __shfl_xor_sync(0xFFFFFFFFu, cnt[q], off);
+                if ((tid & 31) == 0) redi[(tid >> 5) * 8 + q] = cnt[q];
+            }
+            csync();
+            bool done = false;
+            bool fits = false;
+#pragma unroll
+            for (int q = 6; q >= 0; --q) {                 // the highest threshold that still keeps k
+                int tot = 0;
+                for (int w = 0; w < THREADS / 32; ++w) tot += redi[w * 8 + q];
+                if (!done && tot >= c.k) {
+                    lo = th[q];
+                    if (q < 6) hi = th[q + 1];
+                    done = true;
+                    fits = tot <= MERGE_CAP;
+                }
+            }
+            if (!done) hi = th[0];
+            csync();
+            if (fits) break;
+        }
+        floor_key = lo;
+        if (tid == 0) sh.count = 0;
+        csync();
     }
     csync();
     const int Pn = sh.count;
@@ -176,10 +254,10 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     else return false;
     unsigned long long *sorted = buf;
     int Pn2 = Pn;
-    if (n >= 64 && Pn > n + n / 2 + 64) {
+    if (Pn > RANK_SORT_MAX && Pn > n + n / 2 + 64) {
         // far more proven candidates than needed: bisect a key threshold that keeps between n and
         // about next_pow2(n) of them (any such threshold keeps the n best), then sort only those
-        const int want_hi = max(next_pow2(n), n + n / 8);
+        const int want_hi = next_pow2(n);                   // so that the sort below runs on the smallest power of two
         unsigned long long lo = 0ull, hi = ~0ull;          // count(>= lo) >= n > count(>= hi)
         {
             // start from the range the keys actually span
