@@ -125,6 +125,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     csync();
     if (tid < tiles) {
         const unsigned int cnt = __ldcg(&rec[tid].cnt);
+        P.tiles[(size_t)row * MAX_TILES + tid].cnt = 0u;           // the streaming kernel accumulates into it
         sh.tcnt[tid + 1] = (int)cnt;
         atomicMax(&sh.tkey, __ldcg(&rec[tid].tkey));
         if (cnt > (unsigned int)cap_t) sh.found = 1;     // a tile overflowed its slot
@@ -342,7 +343,15 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         for (int i = tid; i < Pn; i += THREADS) {
             const unsigned long long key = buf[i];
             int rank = 0;
-            for (int j = 0; j < Pn; ++j) rank += (buf[j] > key) ? 1 : 0;
+            int j = 0;
+            for (; j + 8 <= Pn; j += 8) {                  // eight independent broadcast reads per trip
+                unsigned long long o[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) o[u] = buf[j + u];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) rank += (o[u] > key) ? 1 : 0;
+            }
+            for (; j < Pn; ++j) rank += (buf[j] > key) ? 1 : 0;
             dst[rank] = key;
         }
         csync();
@@ -428,12 +437,31 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
     const double W = cs[n - 1];
     csync();
     // survivors in vocabulary-index order
-    const int m2 = next_pow2(n);
-    for (int j = tid; j < m2; j += THREADS)
-        ik[j] = (j < n) ? ((buf[j] << 32) | (unsigned long long)j) : 0ull;
-    csync();
     MERGE_STAMP(6);
-    bitonic_sort_desc<THREADS, Sync>(ik, m2, tid);
+    if (n <= RANK_SORT_MAX) {
+        // few survivors: each lands at the number of survivors with a smaller index
+        for (int j = tid; j < n; j += THREADS) {
+            const uint32_t mine = (uint32_t)buf[j];                  // ~index: larger means smaller index
+            int pos = 0;
+            int t = 0;
+            for (; t + 8 <= n; t += 8) {
+                uint32_t o[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) o[u] = (uint32_t)buf[t + u];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) pos += (o[u] > mine) ? 1 : 0;
+            }
+            for (; t < n; ++t) pos += ((uint32_t)buf[t] > mine) ? 1 : 0;
+            ik[pos] = ((unsigned long long)mine << 32) | (unsigned long long)j;
+        }
+        csync();
+    } else {
+        const int m2 = next_pow2(n);
+        for (int j = tid; j < m2; j += THREADS)
+            ik[j] = (j < n) ? ((buf[j] << 32) | (unsigned long long)j) : 0ull;
+        csync();
+        bitonic_sort_desc<THREADS, Sync>(ik, m2, tid);
+    }
     MERGE_STAMP(7);
 
     uint32_t a_acc, a_draw;
@@ -503,9 +531,10 @@ struct StreamShared {
     unsigned long long full[NSTAGE];           // producer -> consumers: tile landed (transaction bytes)
     unsigned long long empty[NSTAGE];          // consumers -> producer: stage free (one arrival per consumer warp)
     StageMeta meta[NSTAGE];
-    float tw[STREAM_WARPS];
-    int wcnt[STREAM_WARPS];
-    unsigned long long best[STREAM_WARPS];
+    // per-stage scratch of the consumer warps (a fast warp may already be on the next tile, in the other stage)
+    float tw[NSTAGE][STREAM_WARPS];
+    unsigned int ncand[NSTAGE];
+    unsigned long long best[NSTAGE][STREAM_WARPS];
 };
 
 template <int DT>
@@ -531,9 +560,15 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
 
     if (warp == STREAM_WARPS) {
         // ------------------------------------------------------------ producer warp
+        // The row configuration of the NEXT tile is resolved while the ring is still full, so that a freed
+        // stage gets its bulk copy issued at once (the configuration is a chain of dependent global loads).
         int n = 0;
-        for (int item = blockIdx.x; item < nitems; item += gridDim.x, ++n) {
+        int item = blockIdx.x;
+        RowCfg c_next;
+        if (item < nitems) c_next = load_cfg(P, item / tiles);
+        for (; item < nitems; item += gridDim.x, ++n) {
             const int s = n % NSTAGE;
+            const RowCfg c = c_next;
             if (n >= NSTAGE) {
                 if (!mbar_wait(&sh.empty[s], ((n / NSTAGE) - 1) & 1)) {
                     if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
@@ -541,7 +576,6 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                 }
             }
             const int row = item / tiles, tile = item - row * tiles;
-            const RowCfg c = load_cfg(P, row);
             if (lane == 0) {
                 StageMeta &m = sh.meta[s];
                 m.cfg = c; m.row = row; m.tile = tile; m.skip = (c.cls == CLS_EXACT) ? 1 : 0;
@@ -558,6 +592,8 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                 }
             }
             __syncwarp();
+            const int nxt = item + gridDim.x;
+            if (nxt < nitems) c_next = load_cfg(P, nxt / tiles);
         }
         return;
     }
@@ -722,12 +758,12 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                     for (int off = 16; off > 0; off >>= 1) best = min(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
                     key = ((unsigned long long)okey(wm) << 32) | (uint32_t)(~(uint32_t)best);
                 }
-                if (lane == 0) sh.best[warp] = key;
+                if (lane == 0) sh.best[s][warp] = key;
                 csync();
                 if (tid == 0) {
-                    unsigned long long b = sh.best[0];
+                    unsigned long long b = sh.best[s][0];
 #pragma unroll
-                    for (int w = 1; w < STREAM_WARPS; ++w) b = max(b, sh.best[w]);
+                    for (int w = 1; w < STREAM_WARPS; ++w) b = max(b, sh.best[s][w]);
                     rec->best = b;
                 }
             } else {
@@ -745,12 +781,14 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                         g = (off < L) ? fmaxf(g, o) : fminf(g, o);
                     }
                 }
-                if (lane == 0) sh.tw[warp] = g;
+                if (lane == 0) sh.tw[s][warp] = g;
+                if (tid == 0) sh.ncand[s] = 0;
                 csync();
-                float t = sh.tw[0];
+                float t = sh.tw[s][0];
 #pragma unroll
-                for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, sh.tw[w]);
-                // every finite element >= t goes to the tile's candidate slot
+                for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, sh.tw[s][w]);
+                // every finite element >= t goes to the tile's candidate slot; a warp reserves its share of the
+                // slot with one shared-memory atomic and adds it to the tile record (no second barrier)
                 int cnt = 0;
 #pragma unroll
                 for (int j = 0; j < NV; ++j) {
@@ -765,16 +803,15 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                     const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
                     if (lane >= off) incl += o;
                 }
-                if (lane == 31) sh.wcnt[warp] = incl;
-                csync();
-                int base = 0, total = 0;
-#pragma unroll
-                for (int w = 0; w < STREAM_WARPS; ++w) {
-                    if (w == warp) base = total;
-                    total += sh.wcnt[w];
+                const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                unsigned int base = 0;
+                if (lane == 0 && total > 0) {
+                    base = atomicAdd(&sh.ncand[s], (unsigned int)total);
+                    atomicAdd(&rec->cnt, (unsigned int)total);          // zero before the call; the merge kernel clears it
                 }
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
                 const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
-                if (cnt > 0 && total <= cap_t) {
+                if (cnt > 0 && (int)base + total <= cap_t) {
                     unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + (size_t)tile * cap_t + base + (incl - cnt);
 #pragma unroll
                     for (int j = 0; j < NV; ++j) {
@@ -790,7 +827,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                         }
                     }
                 }
-                if (tid == 0) { rec->cnt = (unsigned int)total; rec->tkey = okey(t); }
+                if (tid == 0) rec->tkey = okey(t);
             }
 
             // generic-proxy writes into the stage (in-place patches) precede the next bulk copy into it
@@ -819,6 +856,7 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
     const unsigned int status = rs->status;
     if (c.bad || (status & ST_BADID)) {
+        if (tid < tiles) P.tiles[(size_t)row * MAX_TILES + tid].cnt = 0u;      // leave the tile counts clean
         if (tid == 0) { emit_row(P, c, row, -1, 0.0f, F_BADPARAM, 0, 0.0f); rs->status = 0; }
         return;
     }
