@@ -410,9 +410,39 @@ def w0_dtype(w):
     return w.sample.dtype if hasattr(w, "sample") else w.dtype
 
 
+def quick_topk(k, binding, reps=10):
+    """sonic_topk on the c5 'normal' regime (B=256, V=262144, fp32), two input copies (> 2x L2), one k."""
+    import torch
+    tw = wl.config5("normal")
+    ws = binding.new_workspace(tw.B)
+    devs = [binding.DeviceTopK(tw, k, ws=ws), binding.DeviceTopK(tw, k, ws=ws)]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for d in devs:
+            d.run()
+    for _ in range(2):
+        g.replay()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s.record()
+    for _ in range(reps):
+        g.replay()
+    e.record()
+    torch.cuda.synchronize()
+    us = s.elapsed_time(e) * 1000.0 / (reps * 2)
+    peak, _ = peaks()
+    nbytes = tw.logits.nbytes
+    del devs, g
+    torch.cuda.empty_cache()
+    return {"us_per_call": us, "algorithmic_bytes": int(nbytes), "achieved_gbs": nbytes / us / 1e3,
+            "frac": nbytes / us / 1e3 / peak, "copies": 2, "k": k}
+
+
 def quick_measure(name, binding, reps=30):
     """Short cold-input timing of another configuration (not the headline line)."""
     import torch
+    if name.startswith("c5k"):
+        return quick_topk(int(name[3:]), binding)
     w0 = make_workload(name)
     bytes_call = algorithmic_bytes(name, w0)
     copies = int(min(8, max(2, np.ceil(2.0 * L2_BYTES / bytes_call))))
@@ -443,7 +473,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="sonic", choices=["sonic", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4"])
-    ap.add_argument("--also", default="c3,c4", help="other configurations to time briefly (comma separated, '' for none)")
+    ap.add_argument("--also", default="c1,c3,c4,c5k1,c5k64", help="other configurations to time briefly (comma separated, '' for none)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

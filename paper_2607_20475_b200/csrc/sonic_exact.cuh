@@ -58,7 +58,7 @@ struct ExactShared {
 struct ExactCtx {
     ExactShared *sh;
     uint32_t *keys;
-    unsigned int *hcnt, *hm0, *hm1, *hm2;      // per-bin count and mass in three 14-bit limbs (32-bit adds only)
+    unsigned int *hcnt, *hm0, *hm1;            // per-bin count and 64-bit mass as two 32-bit words (32-bit adds, explicit carry)
     int rank, lo, len, per, tid, lane, warp;
     int phase;
     int trace;
@@ -146,8 +146,19 @@ __device__ void ordered_totals(ExactCtx &x, WF wf, CF cf, OrderedState<T> &st, u
     const int wlo = x.warp * wch;
     T wt = T(0);
     unsigned long long cn = 0;
-#pragma unroll 4
-    for (int i = wlo + x.lane; i < wlo + wch; i += 32) { wt += wf(i); cn += cf(i); }
+    for (int i = wlo + x.lane; i < wlo + wch; i += 128) {      // four independent elements per trip (wch is a multiple of 64)
+        T w4[4];
+        unsigned long long c4[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int ii = i + 32 * u;
+            const bool in = ii < wlo + wch;
+            w4[u] = in ? wf(ii) : T(0);
+            c4[u] = in ? cf(ii) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { wt += w4[u]; cn += c4[u]; }
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         wt += __shfl_xor_sync(0xFFFFFFFFu, wt, off);
@@ -256,40 +267,56 @@ __device__ int ordered_find(ExactCtx &x, T target, WF wf, const OrderedState<T> 
 template <typename DF>
 __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first, float p, int nbins, DF digit,
                           unsigned long long &target, unsigned long long &in_bin, unsigned long long *stg) {
-    for (int i = x.tid; i < nbins; i += EX_THREADS) { x.hcnt[i] = 0; x.hm0[i] = 0; x.hm1[i] = 0; x.hm2[i] = 0; }
+    for (int i = x.tid; i < nbins; i += EX_THREADS) { x.hcnt[i] = 0; x.hm0[i] = 0; x.hm1[i] = 0; }
     __syncthreads();
-#pragma unroll 4
-    for (int i0 = 0; i0 < x.per; i0 += EX_THREADS) {
-        const int i = i0 + x.tid;
-        int bin = -1;
-        uint32_t key = 0;
-        if (i < x.len) {
-            key = x.keys[i];
-            if (member(base, key, x.lo + i)) bin = digit(key);
-        }
-        const unsigned int active = __ballot_sync(0xFFFFFFFFu, bin >= 0);
-        if (bin < 0) continue;
-        unsigned int q0 = 0, q1 = 0, q2 = 0;
-        if (by_mass) {
-            unsigned long long q = qweight(key, x.Mf);
-            q0 = (unsigned int)(q & 0x3FFFu); q1 = (unsigned int)((q >> 14) & 0x3FFFu); q2 = (unsigned int)(q >> 28);
-        }
-        int same;
-        __match_all_sync(active, bin, &same);
-        if (same) {                                   // the whole warp hits one bin: one lane adds for all
-            unsigned int n = __popc(active);
-            if (by_mass) { q0 = __reduce_add_sync(active, q0); q1 = __reduce_add_sync(active, q1); q2 = __reduce_add_sync(active, q2); }
-            if ((int)(__ffs(active) - 1) == x.lane) {
-                atomicAdd(&x.hcnt[bin], n);
-                if (q0) atomicAdd(&x.hm0[bin], q0);
-                if (q1) atomicAdd(&x.hm1[bin], q1);
-                if (q2) atomicAdd(&x.hm2[bin], q2);
+    // four elements per thread and trip: their keys, bins and weights are computed first (independent chains
+    // that overlap), then added to the histogram
+    // The mass of a bin is a 64-bit integer kept as two 32-bit words: the low word takes one atomic add whose
+    // returned old value reveals a carry; the high word is touched only on a carry or by weights >= 2^-8.
+    auto add_mass = [&](int b, unsigned long long q) {
+        const unsigned int lo = (unsigned int)q, hi = (unsigned int)(q >> 32);
+        unsigned int carry = 0;
+        if (lo) { const unsigned int old = atomicAdd(&x.hm0[b], lo); carry = (old + lo < old) ? 1u : 0u; }
+        if (hi + carry) atomicAdd(&x.hm1[b], hi + carry);
+    };
+    for (int i0 = 0; i0 < x.per; i0 += 4 * EX_THREADS) {
+        int bin[4];
+        unsigned long long q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * EX_THREADS + x.tid;
+            bin[u] = -1; q[u] = 0ull;
+            if (i < x.len) {
+                const uint32_t key = x.keys[i];
+                if (member(base, key, x.lo + i)) {
+                    bin[u] = digit(key);
+                    if (by_mass && bin[u] >= 0) q[u] = qweight(key, x.Mf);
+                }
             }
-        } else {
-            atomicAdd(&x.hcnt[bin], 1u);
-            if (q0) atomicAdd(&x.hm0[bin], q0);            // small weights leave the upper limbs untouched
-            if (q1) atomicAdd(&x.hm1[bin], q1);
-            if (q2) atomicAdd(&x.hm2[bin], q2);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned int active = __ballot_sync(0xFFFFFFFFu, bin[u] >= 0);
+            if (bin[u] < 0) continue;
+            int same;
+            __match_all_sync(active, bin[u], &same);
+            if (same) {                               // the whole warp hits one bin: one lane adds for all
+                const unsigned int n = __popc(active);
+                unsigned long long qs = q[u];
+                if (by_mass) {                        // 20-bit pieces: 32 of them sum below 2^25
+                    const unsigned int p0 = __reduce_add_sync(active, (unsigned int)(q[u] & 0xFFFFFu));
+                    const unsigned int p1 = __reduce_add_sync(active, (unsigned int)((q[u] >> 20) & 0xFFFFFu));
+                    const unsigned int p2 = __reduce_add_sync(active, (unsigned int)(q[u] >> 40));
+                    qs = (unsigned long long)p0 + ((unsigned long long)p1 << 20) + ((unsigned long long)p2 << 40);
+                }
+                if ((int)(__ffs(active) - 1) == x.lane) {
+                    atomicAdd(&x.hcnt[bin[u]], n);
+                    if (by_mass) add_mass(bin[u], qs);
+                }
+            } else {
+                atomicAdd(&x.hcnt[bin[u]], 1u);
+                if (by_mass) add_mass(bin[u], q[u]);
+            }
         }
     }
     if (first) SONIC_STAMP(17);
@@ -315,7 +342,6 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
                 if (by_mass) {
                     a0[u] = *cg::this_cluster().map_shared_rank(&x.hm0[bin], r);
                     a1[u] = *cg::this_cluster().map_shared_rank(&x.hm1[bin], r);
-                    a2[u] = *cg::this_cluster().map_shared_rank(&x.hm2[bin], r);
                 }
             }
         }
@@ -325,7 +351,7 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
             const int r = pair / bpr, bl = pair - r * bpr;
             if (r < CL) {
                 stg_cnt[r * bpr + bl] = cc[u];
-                stg_mass[r * bpr + bl] = (unsigned long long)a0[u] + ((unsigned long long)a1[u] << 14) + ((unsigned long long)a2[u] << 28);
+                stg_mass[r * bpr + bl] = (unsigned long long)a0[u] | ((unsigned long long)a1[u] << 32);
             }
         }
     }
@@ -461,13 +487,21 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         // CTA 0, which sorts them and picks the element that completes the target
         if (x.tid == 0) x.sh->ucount = 0;
         __syncthreads();
-#pragma unroll 4
-        for (int i0 = 0; i0 < x.per; i0 += EX_THREADS) {
-            const int i = i0 + x.tid;
-            const uint32_t key = (i < x.len) ? x.keys[i] : 0u;
-            const bool want = (i < x.len) && member(base, key, x.lo + i) && in_range(key);
-            const unsigned int pos = warp_append(&x.sh->ucount, want, x.lane);
-            if (want && pos < (unsigned int)GATHER_CAP) sortbuf[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+        for (int i0 = 0; i0 < x.per; i0 += 4 * EX_THREADS) {
+            uint32_t key[4];
+            bool want[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * EX_THREADS + x.tid;
+                key[u] = (i < x.len) ? x.keys[i] : 0u;
+                want[u] = (i < x.len) && member(base, key[u], x.lo + i) && in_range(key[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * EX_THREADS + x.tid;
+                const unsigned int pos = warp_append(&x.sh->ucount, want[u], x.lane);
+                if (want[u] && pos < (unsigned int)GATHER_CAP) sortbuf[pos] = ((unsigned long long)key[u] << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+            }
         }
         __syncthreads();
         const unsigned int mine = min(x.sh->ucount, (unsigned int)GATHER_CAP);
@@ -650,15 +684,21 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     bad = __syncthreads_or(bad);
     SONIC_STAMP(1);
     uint32_t kmax = 0;
-    unsigned long long nfin = 0;
-    for (int li = x.tid; li < x.per; li += EX_THREADS) {
-        float z = zf[li];
-        float y = c.temp ? __fdiv_rn(z, c.tau) : z;
-        uint32_t k = okey(y);
-        x.keys[li] = k;
-        kmax = max(kmax, k);
-        nfin += (k > KEY_NEG_INF && li < x.len) ? 1 : 0;
+    unsigned int nfin32 = 0;
+    for (int l0 = x.tid * 4; l0 < x.per; l0 += EX_THREADS * 4) {   // per is a multiple of 1024: whole float4s
+        const float4 z4 = *reinterpret_cast<const float4 *>(zf + l0);
+        const float zz[4] = {z4.x, z4.y, z4.z, z4.w};
+        uint32_t kk[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float y = c.temp ? __fdiv_rn(zz[u], c.tau) : zz[u];
+            kk[u] = okey(y);
+            kmax = max(kmax, kk[u]);
+            nfin32 += (kk[u] > KEY_NEG_INF && l0 + u < x.len) ? 1u : 0u;
+        }
+        *reinterpret_cast<uint4 *>(x.keys + l0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
     }
+    unsigned long long nfin = nfin32;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, off));
     nfin = block_sum_u64(x, nfin);
@@ -823,7 +863,7 @@ sonic_exact_kernel(const KParams P) {
     x.phase = 0;
     x.keys = reinterpret_cast<uint32_t *>(smem_raw);
     x.hcnt = reinterpret_cast<unsigned int *>(smem_raw + SLICE_MAX * 4);
-    x.hm0 = x.hcnt + HBINS; x.hm1 = x.hcnt + 2 * HBINS; x.hm2 = x.hcnt + 3 * HBINS;
+    x.hm0 = x.hcnt + HBINS; x.hm1 = x.hcnt + 2 * HBINS;
     x.sh = reinterpret_cast<ExactShared *>(smem_raw + SLICE_MAX * 4 + HBINS * 16);
     unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192);
     uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8);
