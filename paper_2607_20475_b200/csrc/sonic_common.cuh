@@ -28,6 +28,14 @@ constexpr int STREAM_THREADS = 256;
 constexpr int STREAM_WARPS = STREAM_THREADS / 32;
 constexpr int CTA_TILE = WARP_TILE * STREAM_WARPS;   // 8192
 constexpr int MAX_TILES = (262144 + CTA_TILE - 1) / CTA_TILE;   // 32 tiles at the largest vocabulary
+// Sparse lists in the stream kernel: the producer warp keeps a request's lists in registers (up to FILTER_HIST
+// history entries, id and count packed in one word, and FILTER_BIAS bias entries) and hands each tile the
+// entries that fall into it; longer lists are scanned by the consumer threads.
+constexpr int FILTER_HIST = 512;
+constexpr int FILTER_BIAS = 32;
+constexpr int FILTER_COUNT_MAX = (1 << 14) - 1;   // largest count that packs beside an 18-bit id
+constexpr int HIT_PEN_CAP = 320;              // history entries of one tile the producer can hand over
+constexpr int HIT_BIAS_CAP = FILTER_BIAS;
 constexpr uint32_t CAND_CAP = 32768;          // candidate slots per row, divided evenly among the row's tiles
 constexpr int MERGE_THREADS = 512;
 constexpr int MERGE_CAP = 8192;               // 64-bit keys the row merge can sort (64 KB of shared memory)
@@ -148,11 +156,39 @@ __device__ __forceinline__ int pick_groups(int k, int V) {
     return -1;
 }
 
-__device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) {
+// The per-request parameters as read from global memory.  Every array that exists is read at once (one
+// global-memory latency, not a chain behind the mode word); values whose mode bit is clear are dropped by
+// resolve_cfg.
+struct CfgRaw {
+    uint32_t z;
+    float tau, p, theta, alpha, beta, gamma;
+    int k, hl, bl;
+};
+__device__ __forceinline__ CfgRaw fetch_cfg(const KParams &P, int row) {
+    const int b = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
+    CfgRaw r;
+    r.z = (P.op == OP_TOPK) ? M_TOP_K : P.mode[b];
+    r.tau = P.temperature ? P.temperature[b] : 1.0f;
+    r.k = (P.op != OP_TOPK && P.top_k) ? P.top_k[b] : 0;
+    r.p = P.top_p ? P.top_p[b] : 1.0f;
+    r.theta = P.min_p ? P.min_p[b] : 0.0f;
+    r.alpha = P.rep ? P.rep[b] : 1.0f;
+    r.beta = P.freq ? P.freq[b] : 0.0f;
+    r.gamma = P.pres ? P.pres[b] : 0.0f;
+    r.hl = P.hist_len ? P.hist_len[b] : 0;
+    r.bl = P.bias_len ? P.bias_len[b] : 0;
+    return r;
+}
+
+// memo_k / memo_G: the caller's memory of the last (k, G) pair, so that runs of rows with one k skip pick_groups
+__device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const CfgRaw &raw, int *memo_k = nullptr, int *memo_G = nullptr) {
     RowCfg c;
     c.b = row; c.l = 0;
     if (P.op == OP_VERIFY) { c.b = row / (P.K + 1); c.l = row - c.b * (P.K + 1); }
-    c.z = (P.op == OP_TOPK) ? M_TOP_K : P.mode[c.b];
+    const uint32_t z_in = raw.z;
+    const float v_tau = raw.tau, v_p = raw.p, v_theta = raw.theta, v_alpha = raw.alpha, v_beta = raw.beta, v_gamma = raw.gamma;
+    const int v_k = raw.k, v_hl = raw.hl, v_bl = raw.bl;
+    c.z = z_in;
     uint32_t z = c.z;
     c.bad = false;
     // a set bit whose parameter array is missing cannot be honoured
@@ -168,15 +204,15 @@ __device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) {
     if ((z & M_GRAMMAR) && !P.bitmask) { c.bad = true; z &= ~M_GRAMMAR; }
     c.z = z;
     c.temp = (z & M_TEMPERATURE) != 0;
-    c.tau = c.temp ? P.temperature[c.b] : 1.0f;
-    c.k = (P.op == OP_TOPK) ? P.ktop : ((z & M_TOP_K) ? P.top_k[c.b] : 0);
-    c.p = (z & M_TOP_P) ? P.top_p[c.b] : 1.0f;
-    c.theta = (z & M_MIN_P) ? P.min_p[c.b] : 0.0f;
-    c.alpha = (z & M_REPETITION) ? P.rep[c.b] : 1.0f;
-    c.beta = (z & M_FREQUENCY) ? P.freq[c.b] : 0.0f;
-    c.gamma = (z & M_PRESENCE) ? P.pres[c.b] : 0.0f;
-    c.hist_len = (z & M_PENALTIES) ? P.hist_len[c.b] : 0;
-    c.bias_len = (z & M_BIAS) ? P.bias_len[c.b] : 0;
+    c.tau = c.temp ? v_tau : 1.0f;
+    c.k = (P.op == OP_TOPK) ? P.ktop : ((z & M_TOP_K) ? v_k : 0);
+    c.p = (z & M_TOP_P) ? v_p : 1.0f;
+    c.theta = (z & M_MIN_P) ? v_theta : 0.0f;
+    c.alpha = (z & M_REPETITION) ? v_alpha : 1.0f;
+    c.beta = (z & M_FREQUENCY) ? v_beta : 0.0f;
+    c.gamma = (z & M_PRESENCE) ? v_gamma : 0.0f;
+    c.hist_len = (z & M_PENALTIES) ? min(max(v_hl, 0), P.hist_stride) : 0;   // never past the request's slice
+    c.bias_len = (z & M_BIAS) ? min(max(v_bl, 0), P.bias_stride) : 0;
     bool greedy = (z & M_GREEDY) != 0;
     if (c.temp && !(c.tau > 0.0f && c.tau < CUDART_INF_F)) c.bad = true;
     if (!greedy) {
@@ -194,12 +230,19 @@ __device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) {
         int kfast = (P.op == OP_TOPK) ? KFAST_TOPK : KFAST_SAMPLE;
         c.cls = CLS_EXACT;
         if (c.k > 0 && c.k <= kfast) {
-            int G = pick_groups(c.k, P.V);
+            int G;
+            if (memo_k && *memo_k == c.k) G = *memo_G;
+            else {
+                G = pick_groups(c.k, P.V);
+                if (memo_k) { *memo_k = c.k; *memo_G = G; }
+            }
             if (G >= 0) { c.cls = CLS_TOPK; c.G = G; }
         }
     }
     return c;
 }
+
+__device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) { return resolve_cfg(P, row, fetch_cfg(P, row)); }
 
 // ---------------------------------------------------------------- Philox4x32-10
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,

@@ -58,10 +58,18 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned int 
     }
     return false;
 }
-// One bulk copy global -> this CTA's shared memory; bytes and both addresses are multiples of 16.
-__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned int bytes, unsigned long long *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+// One bulk copy global -> this CTA's shared memory; bytes and both addresses are multiples of 16.  The logits are
+// read once, so the copy carries an evict-first L2 policy: the stream does not push the workspace (candidates,
+// tile records) and the kernels' code out of L2.
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned int bytes, unsigned long long *bar,
+                                          unsigned long long policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -109,6 +117,8 @@ struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwar
 
 template <int NT, typename Sync, typename SH>
 __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid);
+template <int THREADS, typename SH>
+__device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid);
 
 // Row merge for top-k class rows (one CTA per row).  buf is MERGE_CAP 64-bit
 // words of shared memory.  Returns false if the candidates cannot prove the
@@ -168,23 +178,48 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     unsigned long long floor_key = 1ull;           // keys below it are left out (1: every proven candidate)
     for (int attempt = 0; attempt < 2; ++attempt) {
         unsigned long long kmax = 0ull;
-        for (int j0 = 0; j0 < total; j0 += GB * THREADS) {
-            unsigned long long cd[GB];
-            fetch(j0, cd);
+        // tile-major: a warp takes tiles w and w + NW together, its lanes the slots' entries (no search for the
+        // tile of an entry; the loads of both tiles are in flight at once)
+        constexpr int NW = THREADS / 32, HB = GB / 2;
+        const int lane = tid & 31, warp = tid >> 5;
+        for (int ta = warp; ta < tiles; ta += 2 * NW) {
+            const int tb = ta + NW;
+            const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
+            const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
+            const unsigned long long *pa = P.cand + (size_t)row * CAND_CAP + (size_t)ta * cap_t;
+            const unsigned long long *pb = P.cand + (size_t)row * CAND_CAP + (size_t)tb * cap_t;
+            for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
+                unsigned long long cd[GB];
 #pragma unroll
-            for (int u = 0; u < GB; ++u) {
-                if (j0 + u * THREADS >= total) break;              // uniform over the CTA
-                const unsigned long long out = proven_key(cd[u], j0 + u * THREADS + tid);
-                const bool keep = out >= floor_key;
-                kmax = max(kmax, out);
-                // one shared-memory atomic per warp, not per candidate
-                const unsigned int m = __ballot_sync(0xFFFFFFFFu, keep);
+                for (int u = 0; u < HB; ++u) {
+                    const int j = j0 + u * 32 + lane;
+                    cd[u] = (j < na) ? __ldcg(pa + j) : 0ull;
+                    cd[HB + u] = (j < nb) ? __ldcg(pb + j) : 0ull;
+                }
+                // filter all of the batch, then reserve room with ONE shared-memory atomic per warp and batch
+                // (every warp adds to the same counter: per-candidate or per-slot atomics would queue up there)
+                unsigned long long out[GB];
+                unsigned int km[GB];
+                int nkeep = 0;
+#pragma unroll
+                for (int u = 0; u < GB; ++u) {
+                    const int j = j0 + (u % HB) * 32 + lane;
+                    const bool valid = (u < HB) ? (j < na) : (j < nb);
+                    out[u] = proven_key(cd[u], valid ? 0 : total);
+                    kmax = max(kmax, out[u]);
+                    km[u] = __ballot_sync(0xFFFFFFFFu, out[u] >= floor_key);
+                    nkeep += __popc(km[u]);
+                }
                 int base = 0;
-                if ((tid & 31) == 0 && m) base = atomicAdd(&sh.count, __popc(m));
+                if (lane == 0 && nkeep) base = atomicAdd(&sh.count, nkeep);
                 base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                if (keep) {
-                    const int pos = base + __popc(m & ((1u << (tid & 31)) - 1u));
-                    if (pos < MERGE_CAP) buf[pos] = out;
+#pragma unroll
+                for (int u = 0; u < GB; ++u) {
+                    if (out[u] >= floor_key) {
+                        const int pos = base + __popc(km[u] & ((1u << lane) - 1u));
+                        if (pos < MERGE_CAP) buf[pos] = out[u];
+                    }
+                    base += __popc(km[u]);
                 }
             }
         }
@@ -219,8 +254,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             int *redi = reinterpret_cast<int *>(sh.scratch);
 #pragma unroll
             for (int q = 0; q < 7; ++q) {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) cnt[q] += __shfl_xor_sync(0xFFFFFFFFu, cnt[q], off);
+                cnt[q] = (int)__reduce_add_sync(0xFFFFFFFFu, (unsigned int)cnt[q]);
                 if ((tid & 31) == 0) redi[(tid >> 5) * 8 + q] = cnt[q];
             }
             csync();
@@ -256,9 +290,10 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     unsigned long long *sorted = buf;
     int Pn2 = Pn;
     if (Pn > RANK_SORT_MAX && Pn > n + n / 2 + 64) {
-        // far more proven candidates than needed: bisect a key threshold that keeps between n and
-        // about next_pow2(n) of them (any such threshold keeps the n best), then sort only those
-        const int want_hi = next_pow2(n);                   // so that the sort below runs on the smallest power of two
+        // far more proven candidates than needed: search a key threshold that keeps between n and a little more
+        // than n of them (any such threshold keeps the n best), then sort only those.  The upper end is what the
+        // rank-counting sort takes in one go, else the next power of two (the bitonic sort's size).
+        const int want_hi = (n + n / 2 + 16 <= RANK_SORT_MAX) ? n + n / 2 + 16 : next_pow2(n);
         unsigned long long lo = 0ull, hi = ~0ull;          // count(>= lo) >= n > count(>= hi)
         {
             // start from the range the keys actually span
@@ -292,8 +327,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             int *redi = reinterpret_cast<int *>(sh.scratch);
 #pragma unroll
             for (int q = 0; q < 7; ++q) {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) cnt[q] += __shfl_xor_sync(0xFFFFFFFFu, cnt[q], off);
+                cnt[q] = (int)__reduce_add_sync(0xFFFFFFFFu, (unsigned int)cnt[q]);
                 if ((tid & 31) == 0) redi[(tid >> 5) * 8 + q] = cnt[q];
             }
             csync();
@@ -338,21 +372,43 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     (void)PnAll;
 #define Pn Pn2
     if (Pn <= RANK_SORT_MAX) {
-        // few candidates: each key counts the keys above it (keys are distinct) and lands at its rank
+        // few candidates, one per thread: every warp sorts its 32 keys with shuffles, then a key's rank is its
+        // place in its own run plus, for every other run, the number of keys there above it (a binary search
+        // in the sorted run; keys are distinct, 0 pads the last run).  Two block barriers.
+        static_assert(RANK_SORT_MAX <= THREADS, "one candidate per thread");
         unsigned long long *dst = buf + MERGE_CAP / 2;
-        for (int i = tid; i < Pn; i += THREADS) {
-            const unsigned long long key = buf[i];
-            int rank = 0;
-            int j = 0;
-            for (; j + 8 <= Pn; j += 8) {                  // eight independent broadcast reads per trip
-                unsigned long long o[8];
+        {
+            const int lane = tid & 31, warp = tid >> 5;
+            unsigned long long key = (tid < Pn) ? buf[tid] : 0ull;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) o[u] = buf[j + u];
+            for (int kk = 2; kk <= 32; kk <<= 1) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) rank += (o[u] > key) ? 1 : 0;
+                for (int jj = kk >> 1; jj > 0; jj >>= 1) {
+                    const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
+                    const bool up = ((lane & kk) == 0);            // this block of kk sorts descending
+                    const bool first = ((lane & jj) == 0);         // the lower lane of the pair
+                    const bool take_max = (up == first);
+                    key = take_max ? max(key, o) : min(key, o);
+                }
             }
-            for (; j < Pn; ++j) rank += (buf[j] > key) ? 1 : 0;
-            dst[rank] = key;
+            csync();                                               // every thread has read its key from buf
+            buf[tid] = key;                                        // sorted runs of 32 (descending), in place
+            csync();
+            const int runs = (Pn + 31) >> 5;
+            if (key != 0ull) {
+                int rank = lane;
+                for (int r = 0; r < runs; ++r) {
+                    if (r == warp) continue;
+                    const unsigned long long *run = buf + r * 32;
+                    int lo = 0;                                    // number of keys of the run above `key`
+#pragma unroll
+                    for (int step = 16; step > 0; step >>= 1)
+                        if (run[lo + step - 1] > key) lo += step;
+                    if (lo < 32 && run[lo] > key) ++lo;            // covers a run whose 32 keys are all above
+                    rank += lo;
+                }
+                dst[rank] = key;
+            }
         }
         csync();
         for (int i = tid; i < Pn; i += THREADS) buf[i] = dst[i];
@@ -384,7 +440,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     }
     // small supports are finished by one warp without block barriers
     if (n <= WARP_EPILOGUE_MAX) {
-        if (tid < 32) merge_epilogue<32, WarpSync>(P, c, row, n, buf, sh, tid);
+        merge_epilogue_small<THREADS>(P, c, row, n, buf, sh, tid);
     } else {
         merge_epilogue<THREADS, Sync>(P, c, row, n, buf, sh, tid);
     }
@@ -393,40 +449,54 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
 
 // Truncation epilogue and token selection over the n best candidates, sorted in
 // buf[0, n) (TopK already applied): TopP, MinP, index-order CDF, Philox draw,
-// and for verification rows the accept test and the residual.  Run by NT
-// threads that synchronise with Sync (a whole CTA, or one warp).
-template <int NT, typename Sync, typename SH>
-__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
-    Sync csync;
-    constexpr int THREADS = NT;
-    // shared-memory layout after the sort (n <= KFAST_SAMPLE = MERGE_CAP / 4):
-    //   buf[0, n)     sorted keys (value key << 32 | ~index)
-    //   w             weights exp(y - M) in ranking order
-    //   cs            cumulative sums (ranking order), later residual / CDF in index order
-    //   ik            (~index << 32 | ranking position), sorted descending = index ascending
-    double *w = reinterpret_cast<double *>(buf + KFAST_SAMPLE);
-    double *cs = reinterpret_cast<double *>(buf + 2 * KFAST_SAMPLE);
-    unsigned long long *ik = buf + 3 * KFAST_SAMPLE;
+// and for verification rows the accept test and the residual.  Three parts:
+// the front (weights, cumulative sums, TopP / MinP: linear work), the index
+// order of the survivors (quadratic rank counting, or a sort), and the tail
+// (linear again).  Large supports run all three on the whole CTA; small ones
+// run the linear parts on one warp, without block barriers, and only the
+// quadratic part on all threads.
+//
+// shared-memory layout after the sort (n <= KFAST_SAMPLE = MERGE_CAP / 4):
+//   buf[0, n)     sorted keys (value key << 32 | ~index)
+//   w             weights exp(y - M) in ranking order
+//   cs            cumulative sums (ranking order), later residual / CDF in index order
+//   ik            (~index << 32 | ranking position), sorted descending = index ascending
+struct EpiView {
+    double *w, *cs;
+    unsigned long long *ik;
+    __device__ explicit EpiView(unsigned long long *buf)
+        : w(reinterpret_cast<double *>(buf + KFAST_SAMPLE)), cs(reinterpret_cast<double *>(buf + 2 * KFAST_SAMPLE)),
+          ik(buf + 3 * KFAST_SAMPLE) {}
+};
+
+// weights of the candidates (all threads of the caller's group)
+template <int NT>
+__device__ __forceinline__ void epilogue_weights(int n, unsigned long long *buf, int tid) {
+    EpiView v(buf);
     const double M = (double)unkey((uint32_t)(buf[0] >> 32));
-    for (int j = tid; j < n; j += THREADS) {
+    for (int j = tid; j < n; j += NT) {
         double y = (double)unkey((uint32_t)(buf[j] >> 32));
         double wj = exp(y - M);
-        w[j] = wj; cs[j] = wj;
+        v.w[j] = wj; v.cs[j] = wj;
     }
-    if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
-    csync();
-    MERGE_STAMP(4);
-    block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
-    MERGE_STAMP(5);
-    const double Z = cs[n - 1];
+}
+
+// cumulative sums and the TopP / MinP cuts; returns the surviving prefix length (also left in sh.n_p)
+template <int NT, typename Sync, typename SH>
+__device__ __forceinline__ int epilogue_truncate(const RowCfg &c, int n, unsigned long long *buf, SH &sh, int tid) {
+    Sync csync;
+    EpiView v(buf);
+    const double M = (double)unkey((uint32_t)(buf[0] >> 32));
+    block_inclusive_scan<NT, Sync>(v.cs, n, sh.scratch, tid);
+    const double Z = v.cs[n - 1];
     if (c.z & M_TOP_P) {
         const double target = (double)c.p * Z;
-        for (int j = tid; j < n; j += THREADS)
-            if (cs[j] >= target && (j == 0 || cs[j - 1] < target)) sh.n_p = j + 1;
+        for (int j = tid; j < n; j += NT)
+            if (v.cs[j] >= target && (j == 0 || v.cs[j - 1] < target)) sh.n_p = j + 1;
     }
     if (c.z & M_MIN_P) {
         const double thr = M + log((double)c.theta);
-        for (int j = tid; j < n; j += THREADS) {
+        for (int j = tid; j < n; j += NT) {
             bool in = (double)unkey((uint32_t)(buf[j] >> 32)) >= thr;
             bool prev_in = (j == 0) || ((double)unkey((uint32_t)(buf[j - 1] >> 32)) >= thr);
             if (!in && prev_in) sh.n_m = j;
@@ -434,36 +504,58 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
     }
     csync();
     n = min(n, min(sh.n_p, sh.n_m));
-    const double W = cs[n - 1];
     csync();
-    // survivors in vocabulary-index order
-    MERGE_STAMP(6);
+    if (tid == 0) sh.n_p = n;
+    csync();
+    return n;
+}
+
+// survivors in vocabulary-index order
+template <int NT, typename Sync>
+__device__ __forceinline__ void epilogue_index_order(int n, unsigned long long *buf, int tid) {
+    Sync csync;
+    EpiView v(buf);
     if (n <= RANK_SORT_MAX) {
-        // few survivors: each lands at the number of survivors with a smaller index
-        for (int j = tid; j < n; j += THREADS) {
-            const uint32_t mine = (uint32_t)buf[j];                  // ~index: larger means smaller index
+        // few survivors: each lands at the number of survivors with a smaller index; S threads share a survivor
+        const int S = min(32, max(1, NT / next_pow2(n)));
+        for (int j0 = 0; j0 < n; j0 += NT / S) {
+            const int j = j0 + tid / S, seg = tid % S;
+            const uint32_t mine = (j < n) ? (uint32_t)buf[j] : 0xFFFFFFFFu;      // ~index: larger means smaller index
+            const int tlo = (int)(((long long)n * seg) / S), thi = (int)(((long long)n * (seg + 1)) / S);
             int pos = 0;
-            int t = 0;
-            for (; t + 8 <= n; t += 8) {
+            int t = tlo;
+            for (; t + 8 <= thi; t += 8) {
                 uint32_t o[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) o[u] = (uint32_t)buf[t + u];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) pos += (o[u] > mine) ? 1 : 0;
             }
-            for (; t < n; ++t) pos += ((uint32_t)buf[t] > mine) ? 1 : 0;
-            ik[pos] = ((unsigned long long)mine << 32) | (unsigned long long)j;
+            for (; t < thi; ++t) pos += ((uint32_t)buf[t] > mine) ? 1 : 0;
+            for (int off = 1; off < S; off <<= 1) pos += __shfl_xor_sync(0xFFFFFFFFu, pos, off);
+            if (seg == 0 && j < n) v.ik[pos] = ((unsigned long long)mine << 32) | (unsigned long long)j;
         }
         csync();
     } else {
         const int m2 = next_pow2(n);
-        for (int j = tid; j < m2; j += THREADS)
-            ik[j] = (j < n) ? ((buf[j] << 32) | (unsigned long long)j) : 0ull;
+        for (int j = tid; j < m2; j += NT)
+            v.ik[j] = (j < n) ? ((buf[j] << 32) | (unsigned long long)j) : 0ull;
         csync();
-        bitonic_sort_desc<THREADS, Sync>(ik, m2, tid);
+        bitonic_sort_desc<NT, Sync>(v.ik, m2, tid);
     }
-    MERGE_STAMP(7);
+}
 
+// draw, verification, selection and the row's outputs
+template <int NT, typename Sync, typename SH>
+__device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+    Sync csync;
+    constexpr int THREADS = NT;
+    EpiView v(buf);
+    double *w = v.w, *cs = v.cs;
+    unsigned long long *ik = v.ik;
+    const double W = cs[n - 1];                 // still the ranking-order cumulative sums here
+    csync();
+    MERGE_STAMP(7);
     uint32_t a_acc, a_draw;
     draw_cells(P, c, a_acc, a_draw);
     const double u_draw = cell_to_u(a_draw);
@@ -518,23 +610,60 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
     MERGE_STAMP(9);
 }
 
+
+template <int NT, typename Sync, typename SH>
+__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+    Sync csync;
+    epilogue_weights<NT>(n, buf, tid);
+    if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
+    csync();
+    MERGE_STAMP(4);
+    n = epilogue_truncate<NT, Sync>(c, n, buf, sh, tid);
+    MERGE_STAMP(6);
+    epilogue_index_order<NT, Sync>(n, buf, tid);
+    epilogue_tail<NT, Sync>(P, c, row, n, buf, sh, tid);
+}
+
+// Small supports: the linear parts on warp 0 (warp-level synchronisation only), the weights and the quadratic
+// index ranking on the whole CTA.  Three block barriers in all.
+template <int THREADS, typename SH>
+__device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+    epilogue_weights<THREADS>(n, buf, tid);
+    if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
+    __syncthreads();
+    MERGE_STAMP(4);
+    if (tid < 32) epilogue_truncate<32, WarpSync>(c, n, buf, sh, tid);
+    __syncthreads();
+    n = sh.n_p;
+    MERGE_STAMP(6);
+    epilogue_index_order<THREADS, BlockSync>(n, buf, tid);
+    if (tid < 32) epilogue_tail<32, WarpSync>(P, c, row, n, buf, sh, tid);
+}
+
 // What the producer hands to the consumers with each stage.
 struct StageMeta {
     RowCfg cfg;
     int row, tile;
     int skip;                                  // the row belongs to the exact kernel: nothing was loaded
+    int patch;                                 // 0 none, 1 the producer filtered the lists into hits[], 2 consumers scan the lists
+    int npen, nbias;                           // hits of this tile
+    int hb;                                    // which hit buffer holds them
 };
+struct Hit { int li; int payload; };           // element within the tile; history count, or the bias as float bits
 
 template <int DT>
 struct StreamShared {
     static constexpr int NSTAGE = VecTraits<DT>::NSTAGE;
-    unsigned long long full[NSTAGE];           // producer -> consumers: tile landed (transaction bytes)
+    unsigned long long full[NSTAGE];           // producer -> consumers: stage described, copy issued (one arrival + the copy's bytes)
     unsigned long long empty[NSTAGE];          // consumers -> producer: stage free (one arrival per consumer warp)
     StageMeta meta[NSTAGE];
     // per-stage scratch of the consumer warps (a fast warp may already be on the next tile, in the other stage)
     float tw[NSTAGE][STREAM_WARPS];
     unsigned int ncand[NSTAGE];
     unsigned long long best[NSTAGE][STREAM_WARPS];
+    // hit lists: one buffer more than stages, so that the producer fills the next tile's while both stages are busy
+    Hit pen[NSTAGE + 1][HIT_PEN_CAP];
+    Hit bias[NSTAGE + 1][HIT_BIAS_CAP];
 };
 
 template <int DT>
@@ -558,27 +687,132 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
     __syncthreads();
     pdl_launch_dependents();                   // the merge kernel may start launching; it waits for this grid to finish
 
+    // this CTA's contiguous share of the (row, tile) items
+    const int item_lo = (int)(((long long)nitems * blockIdx.x) / gridDim.x);
+    const int item_hi = (int)(((long long)nitems * (blockIdx.x + 1)) / gridDim.x);
+
     if (warp == STREAM_WARPS) {
         // ------------------------------------------------------------ producer warp
-        // The row configuration of the NEXT tile is resolved while the ring is still full, so that a freed
-        // stage gets its bulk copy issued at once (the configuration is a chain of dependent global loads).
-        int n = 0;
-        int item = blockIdx.x;
+        // A CTA takes a contiguous run of tiles, so consecutive tiles mostly belong to one row.  Per tile the
+        // producer (1) waits for a free stage, describes the tile and issues its bulk copy, then (2) prepares
+        // the NEXT tile while the ring is busy.  On a new row that means one round of global loads (parameters
+        // and sparse lists, kept in registers for the row's other tiles); on every tile, picking the list
+        // entries that fall into it and writing them to a hit buffer, so that the consumers patch only what is
+        // there, each warp only its own part of the tile.
+        static_assert(SONIC_MAX_VOCAB <= (1 << 18), "packed history entries hold an 18-bit id");
+        constexpr int HPL = FILTER_HIST / 32;      // packed history entries per lane
+        struct Prep { int patch, npen, nbias; };
+        int memo_k = -1, memo_G = -1;
         RowCfg c_next;
-        if (item < nitems) c_next = load_cfg(P, item / tiles);
-        for (; item < nitems; item += gridDim.x, ++n) {
+        uint32_t packed[HPL];                      // id | count << 18; 0 = no entry
+        int b_id = -1;
+        float b_val = 0.0f;
+        int row_patch = 0, cached_row = -1;
+        auto load_row = [&](int row) {
+            const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
+            const int *hid = P.hist_ids ? P.hist_ids + (size_t)req * P.hist_stride : nullptr;
+            const int *hct = P.hist_counts ? P.hist_counts + (size_t)req * P.hist_stride : nullptr;
+            const int *bid = P.bias_ids ? P.bias_ids + (size_t)req * P.bias_stride : nullptr;
+            const float *bvl = P.bias_vals ? P.bias_vals + (size_t)req * P.bias_stride : nullptr;
+            // the first round of loads goes out before the first use (the lengths arrive with the parameters:
+            // bound by the strides); the second half of a long history follows in a round of its own
+            constexpr int HALF = HPL / 2;
+            const CfgRaw raw = fetch_cfg(P, row);
+            int id[HALF], ct[HALF];
+#pragma unroll
+            for (int u = 0; u < HALF; ++u) {
+                const int t = lane + 32 * u;
+                id[u] = -1; ct[u] = 0;
+                if (hid && hct && t < P.hist_stride) { id[u] = __ldg(hid + t); ct[u] = __ldg(hct + t); }
+            }
+            int b0 = -1; float v0 = 0.0f;
+            if (bid && bvl && lane < P.bias_stride) { b0 = __ldg(bid + lane); v0 = __ldg(bvl + lane); }
+            c_next = resolve_cfg(P, row, raw, &memo_k, &memo_G);
+            cached_row = row;
+            row_patch = 0;
+            if (c_next.cls == CLS_EXACT || !(c_next.hist_len > 0 || c_next.bias_len > 0)) return;
+            row_patch = 2;
+            if (c_next.hist_len > FILTER_HIST || c_next.bias_len > FILTER_BIAS) return;
+            bool bad = false, big = false;
+            auto pack = [&](int t, int i, int cnt) -> uint32_t {
+                if (t >= c_next.hist_len) return 0u;
+                if (i < 0 || i >= P.V) { bad = true; return 0u; }
+                if (cnt > FILTER_COUNT_MAX) { big = true; return 0u; }
+                return (cnt > 0) ? ((uint32_t)i | ((uint32_t)cnt << 18)) : 0u;
+            };
+#pragma unroll
+            for (int u = 0; u < HALF; ++u) packed[u] = pack(lane + 32 * u, id[u], ct[u]);
+#pragma unroll
+            for (int u = 0; u < HALF; ++u) packed[HALF + u] = 0u;
+            if (c_next.hist_len > 32 * HALF) {
+#pragma unroll
+                for (int u = 0; u < HALF; ++u) {
+                    const int t = lane + 32 * (HALF + u);
+                    id[u] = -1; ct[u] = 0;
+                    if (t < c_next.hist_len) { id[u] = __ldg(hid + t); ct[u] = __ldg(hct + t); }
+                }
+#pragma unroll
+                for (int u = 0; u < HALF; ++u) packed[HALF + u] = pack(lane + 32 * (HALF + u), id[u], ct[u]);
+            }
+            b_id = -1; b_val = 0.0f;
+            if (lane < c_next.bias_len) {
+                if (b0 < 0 || b0 >= P.V) bad = true;
+                else { b_id = b0; b_val = v0; }
+            }
+            if (bad) atomicOr(&P.rs[row].status, ST_BADID);
+            if (__any_sync(0xFFFFFFFFu, big)) return;          // a count too large to pack: consumers scan
+            row_patch = 1;
+        };
+        auto prepare = [&](int row, int tile, int hb) -> Prep {
+            if (row != cached_row) load_row(row);
+            Prep r{row_patch, 0, 0};
+            if (row_patch != 1) return r;
+            const int first = tile * CTA_TILE;
+#pragma unroll
+            for (int u = 0; u < HPL; ++u) {
+                const unsigned int li = (packed[u] & 0x3FFFFu) - (unsigned int)first;
+                const bool hit = packed[u] != 0u && li < (unsigned int)CTA_TILE;
+                const unsigned int hm = __ballot_sync(0xFFFFFFFFu, hit);
+                if (hit) {
+                    const int pos = r.npen + __popc(hm & ((1u << lane) - 1u));
+                    if (pos < HIT_PEN_CAP) { sh.pen[hb][pos].li = (int)li; sh.pen[hb][pos].payload = (int)(packed[u] >> 18); }
+                }
+                r.npen += __popc(hm);
+            }
+            {
+                const unsigned int li = (unsigned int)(b_id - first);
+                const bool hit = b_id >= 0 && li < (unsigned int)CTA_TILE;
+                const unsigned int hm = __ballot_sync(0xFFFFFFFFu, hit);
+                if (hit) {
+                    const int pos = __popc(hm & ((1u << lane) - 1u));
+                    sh.bias[hb][pos].li = (int)li; sh.bias[hb][pos].payload = __float_as_int(b_val);
+                }
+                r.nbias = __popc(hm);
+            }
+            if (r.npen > HIT_PEN_CAP) r.patch = 2;             // crowded tile: the consumers scan the lists
+            return r;
+        };
+        const unsigned long long l2_policy = l2_evict_first_policy();
+        int n = 0;
+        Prep p_next{0, 0, 0};
+        if (item_lo < item_hi) p_next = prepare(item_lo / tiles, item_lo % tiles, 0);
+        for (int item = item_lo; item < item_hi; ++item, ++n) {
             const int s = n % NSTAGE;
             const RowCfg c = c_next;
+            const Prep pr = p_next;
             if (n >= NSTAGE) {
+                // the consumers have left tile n - NSTAGE: its stage and its hit buffer are free
                 if (!mbar_wait(&sh.empty[s], ((n / NSTAGE) - 1) & 1)) {
                     if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
                     return;
                 }
             }
             const int row = item / tiles, tile = item - row * tiles;
+            __syncwarp();                              // the hit buffer's entries, written by all lanes, precede the arrival
             if (lane == 0) {
                 StageMeta &m = sh.meta[s];
                 m.cfg = c; m.row = row; m.tile = tile; m.skip = (c.cls == CLS_EXACT) ? 1 : 0;
+                m.patch = pr.patch; m.npen = pr.npen; m.nbias = pr.nbias; m.hb = n % (NSTAGE + 1);
                 if (c.cls == CLS_EXACT) {
                     mbar_arrive(&sh.full[s]);
                 } else {
@@ -588,19 +822,19 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                     const unsigned char *src = reinterpret_cast<const unsigned char *>(P.logits) +
                                                ((size_t)row * (size_t)P.row_stride + (size_t)first) * ELT;
                     mbar_arrive_expect_tx(&sh.full[s], bytes);
-                    bulk_load(stages + (size_t)s * STAGE_BYTES, src, bytes, &sh.full[s]);
+                    bulk_load(stages + (size_t)s * STAGE_BYTES, src, bytes, &sh.full[s], l2_policy);
                 }
             }
             __syncwarp();
-            const int nxt = item + gridDim.x;
-            if (nxt < nitems) c_next = load_cfg(P, nxt / tiles);
+            // hit buffer (n + 1) % (NSTAGE + 1) was last used by tile n - NSTAGE, which the consumers have left
+            if (item + 1 < item_hi) p_next = prepare((item + 1) / tiles, (item + 1) % tiles, (n + 1) % (NSTAGE + 1));
         }
         return;
     }
 
     // ---------------------------------------------------------------- consumer warps
     int n = 0;
-    for (int item = blockIdx.x; item < nitems; item += gridDim.x, ++n) {
+    for (int item = item_lo; item < item_hi; ++item, ++n) {
         const int s = n % NSTAGE;
         const int row = item / tiles, tile = item - row * tiles;
         const int tile_base = tile * CTA_TILE;
@@ -612,19 +846,6 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
             const int w = (wbase >> 5) + lane;
             mword = (w < ((P.V + 31) >> 5)) ? __ldg(P.bitmask + (size_t)row * P.bitmask_stride + w) : 0u;
         }
-        // the first entries of the row's sparse lists as well (lengths are checked once the configuration is known)
-        const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
-        int h_id0 = -1, h_ct0 = 0, h_id1 = -1, h_ct1 = 0, b_id0 = -1;
-        float b_v0 = 0.0f;
-        const int *hid = P.hist_ids ? P.hist_ids + (size_t)req * P.hist_stride : nullptr;
-        const int *hct = P.hist_counts ? P.hist_counts + (size_t)req * P.hist_stride : nullptr;
-        const int *bid = P.bias_ids ? P.bias_ids + (size_t)req * P.bias_stride : nullptr;
-        const float *bvl = P.bias_vals ? P.bias_vals + (size_t)req * P.bias_stride : nullptr;
-        if (hid && hct) {
-            if (tid < P.hist_stride) { h_id0 = __ldg(hid + tid); h_ct0 = __ldg(hct + tid); }
-            if (tid + STREAM_THREADS < P.hist_stride) { h_id1 = __ldg(hid + tid + STREAM_THREADS); h_ct1 = __ldg(hct + tid + STREAM_THREADS); }
-        }
-        if (bid && bvl && tid < P.bias_stride) { b_id0 = __ldg(bid + tid); b_v0 = __ldg(bvl + tid); }
         if (!mbar_wait(&sh.full[s], (n / NSTAGE) & 1)) {
             if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
             return;
@@ -637,7 +858,8 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
             unsigned char *stage = stages + (size_t)s * STAGE_BYTES;
             const bool masked = (c.z & M_GRAMMAR) != 0;
             const bool tail = tile_base + CTA_TILE > P.V;
-            const bool patched = (c.hist_len > 0 || c.bias_len > 0);
+            const int patch = meta.patch;
+            const bool patched = patch != 0;
             float *ptile = (DT == 0) ? reinterpret_cast<float *>(stage) : conv;    // fp32 view the sparse lists patch
 
             float e[EPL];
@@ -665,38 +887,52 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                     }
                 }
             };
-            if (patched) {
-                if (DT == 1) {
-                    // widen the bf16 tile to fp32 in shared memory so single entries can be rewritten
-                    read_raw();
+            auto widen = [&]() {                      // bf16 only: the warp's part of the tile as fp32 in shared memory
 #pragma unroll
-                    for (int j = 0; j < NV; ++j) {
-                        float *p = conv + warp * WARP_TILE + j * 32 * VEC + lane * VEC;
+                for (int j = 0; j < NV; ++j) {
+                    float *p = conv + warp * WARP_TILE + j * 32 * VEC + lane * VEC;
 #pragma unroll
-                        for (int q = 0; q < VEC; q += 4)
-                            *reinterpret_cast<float4 *>(p + q) = make_float4(e[j * VEC + q], e[j * VEC + q + 1], e[j * VEC + q + 2], e[j * VEC + q + 3]);
-                    }
+                    for (int q = 0; q < VEC; q += 4)
+                        *reinterpret_cast<float4 *>(p + q) = make_float4(e[j * VEC + q], e[j * VEC + q + 1], e[j * VEC + q + 2], e[j * VEC + q + 3]);
+                }
+            };
+            // penalties and biases commute with the mask (a masked logit stays -inf), so they are applied to
+            // the unmasked tile and the mask is applied when the lanes read their elements
+            if (patch == 1) {
+                // the producer listed this tile's entries: every warp patches its own part, no block-wide barrier
+                if (DT == 1) { read_raw(); widen(); }
+                __syncwarp();
+                for (int h = lane; h < meta.npen; h += 32) {
+                    const Hit x = sh.pen[meta.hb][h];
+                    if (x.li / WARP_TILE == warp) ptile[x.li] = apply_penalties(ptile[x.li], x.payload, c);
+                }
+                __syncwarp();
+                for (int h = lane; h < meta.nbias; h += 32) {
+                    const Hit x = sh.bias[meta.hb][h];
+                    if (x.li / WARP_TILE == warp) ptile[x.li] = __fadd_rn(ptile[x.li], __int_as_float(x.payload));
+                }
+                __syncwarp();
+                read_f32(ptile);
+            } else if (patch == 2) {
+                // long or crowded lists: all consumer threads scan them together
+                if (DT == 1) { read_raw(); widen(); csync(); }
+                const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
+                const int *hid = P.hist_ids + (size_t)req * P.hist_stride;
+                const int *hct = P.hist_counts + (size_t)req * P.hist_stride;
+                bool bad = false;
+                for (int t = tid; t < c.hist_len; t += STREAM_THREADS) {
+                    const int id = __ldg(hid + t);
+                    if (id < 0 || id >= P.V) { bad = true; continue; }
+                    const int li = id - tile_base;
+                    if (li >= 0 && li < CTA_TILE) ptile[li] = apply_penalties(ptile[li], __ldg(hct + t), c);
                 }
                 csync();
-                // penalties and biases commute with the mask (a masked logit stays -inf), so they are applied to
-                // the unmasked tile and the mask is applied when the lanes read their elements
-                bool bad = false;
-                auto pen = [&](int id, int ct) {
-                    if (id < 0 || id >= P.V) { bad = true; return; }
+                for (int t = tid; t < c.bias_len; t += STREAM_THREADS) {
+                    const int id = __ldg(P.bias_ids + (size_t)req * P.bias_stride + t);
+                    if (id < 0 || id >= P.V) { bad = true; continue; }
                     const int li = id - tile_base;
-                    if (li >= 0 && li < CTA_TILE) ptile[li] = apply_penalties(ptile[li], ct, c);
-                };
-                if (tid < c.hist_len) pen(h_id0, h_ct0);
-                if (tid + STREAM_THREADS < c.hist_len) pen(h_id1, h_ct1);
-                for (int t = tid + 2 * STREAM_THREADS; t < c.hist_len; t += STREAM_THREADS) pen(__ldg(hid + t), __ldg(hct + t));
-                csync();
-                auto add = [&](int id, float v) {
-                    if (id < 0 || id >= P.V) { bad = true; return; }
-                    const int li = id - tile_base;
-                    if (li >= 0 && li < CTA_TILE) ptile[li] = __fadd_rn(ptile[li], v);
-                };
-                if (tid < c.bias_len) add(b_id0, b_v0);
-                for (int t = tid + STREAM_THREADS; t < c.bias_len; t += STREAM_THREADS) add(__ldg(bid + t), __ldg(bvl + t));
+                    if (li >= 0 && li < CTA_TILE) ptile[li] = __fadd_rn(ptile[li], __ldg(P.bias_vals + (size_t)req * P.bias_stride + t));
+                }
                 if (bad && tile == 0) atomicOr(&rs->status, ST_BADID);
                 csync();
                 read_f32(ptile);
@@ -788,42 +1024,42 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
 #pragma unroll
                 for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, sh.tw[s][w]);
                 // every finite element >= t goes to the tile's candidate slot; a warp reserves its share of the
-                // slot with one shared-memory atomic and adds it to the tile record (no second barrier)
-                int cnt = 0;
+                // slot with one shared-memory atomic and adds it to the tile record (no second barrier).
+                // Most warps hold no candidate at all and leave after one vote.  The others mark their
+                // candidates in a bit mask and fetch the values again from the tile in shared memory (a
+                // candidate is neither masked nor past the row's end, so the tile holds its value).
+                const float t2 = fmaxf(t, -CUDART_MAX_NORMAL_F);           // e >= t2  <=>  e >= t and e is not -inf
+                if (__any_sync(0xFFFFFFFFu, lm >= t2)) {
+                    unsigned int cm = 0;
 #pragma unroll
-                for (int j = 0; j < NV; ++j) {
-                    if (mv[j] >= t) {
+                    for (int q = 0; q < EPL; ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
+                    const int cnt = __popc(cm);
+                    int incl = cnt;
 #pragma unroll
-                        for (int q = 0; q < VEC; ++q) cnt += (e[j * VEC + q] >= t && e[j * VEC + q] > -CUDART_INF_F) ? 1 : 0;
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                        if (lane >= off) incl += o;
                     }
-                }
-                int incl = cnt;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                    if (lane >= off) incl += o;
-                }
-                const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                unsigned int base = 0;
-                if (lane == 0 && total > 0) {
-                    base = atomicAdd(&sh.ncand[s], (unsigned int)total);
-                    atomicAdd(&rec->cnt, (unsigned int)total);          // zero before the call; the merge kernel clears it
-                }
-                base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
-                if (cnt > 0 && (int)base + total <= cap_t) {
-                    unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + (size_t)tile * cap_t + base + (incl - cnt);
-#pragma unroll
-                    for (int j = 0; j < NV; ++j) {
-                        if (mv[j] >= t) {
-#pragma unroll
-                            for (int q = 0; q < VEC; ++q) {
-                                const float v = e[j * VEC + q];
-                                if (v >= t && v > -CUDART_INF_F) {
-                                    const int idx = slot_index<DT>(wbase, lane, j * VEC + q);
-                                    *dst++ = ((unsigned long long)okey(v) << 32) | (uint32_t)(~(uint32_t)idx);
-                                }
-                            }
+                    const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                    unsigned int base = 0;
+                    if (lane == 0) {
+                        base = atomicAdd(&sh.ncand[s], (unsigned int)total);
+                        atomicAdd(&rec->cnt, (unsigned int)total);      // zero before the call; the merge kernel clears it
+                    }
+                    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                    const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
+                    if ((int)base + total <= cap_t) {
+                        unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + (size_t)tile * cap_t + base + (incl - cnt);
+                        const int lbase = warp * WARP_TILE + lane * VEC;
+                        while (cm) {
+                            const int q = __ffs(cm) - 1;
+                            cm &= cm - 1;
+                            const int li = lbase + (q / VEC) * (32 * VEC) + (q % VEC);
+                            float v;
+                            if (DT == 0 || patched) v = ptile[li];
+                            else v = __uint_as_float((uint32_t)reinterpret_cast<const unsigned short *>(stage)[li] << 16);
+                            if (c.div_all) v = __fdiv_rn(v, c.tau);
+                            *dst++ = ((unsigned long long)okey(v) << 32) | (uint32_t)(~(uint32_t)(tile_base + li));
                         }
                     }
                 }

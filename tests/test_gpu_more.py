@@ -136,3 +136,28 @@ def test_many_list_entries_in_one_tile(sonic, oracle):
     got = dev.results()
     ref = oracle.sample(w)
     compare_sample(got, ref, w)
+
+
+@pytest.mark.parametrize("dtype", [wl.DTYPE_F32, wl.DTYPE_BF16])
+@pytest.mark.parametrize("n_hist,n_bias", [(300, 50), (383, 64), (500, 20), (200, 100)])
+def test_short_lists_per_tile_hit_lists(sonic, oracle, dtype, n_hist, n_bias):
+    # lists short enough to be filtered per tile: below, at and above what one tile's hit lists hold (all ids in
+    # one tile, which crowds it), ids present in both lists (penalty first, then bias), a ragged last tile
+    V = 3 * 8192 + 17
+    rng = np.random.default_rng(1000 + n_hist + n_bias)
+    x = (rng.standard_normal((4, V)) * 2).astype(np.float32)
+    ids = rng.choice(8192, max(n_hist, n_bias), replace=False) + 8192
+    far = [0, 5, 8191, 2 * 8192, V - 1]                      # a few entries in the other tiles
+    hist = [{**{int(i): int(c) for i, c in zip(ids[:n_hist], rng.integers(1, 5, n_hist))}, **{i: 2 for i in far}}] * 4
+    bias = [{**{int(i): float(v) for i, v in zip(ids[:n_bias], rng.uniform(-4, 4, n_bias))}, **{i: 1.5 for i in far[:3]}}] * 4
+    mode = wl.REPETITION | wl.FREQUENCY | wl.PRESENCE | wl.BIAS
+    w = make_sample(x, [mode | wl.GREEDY, mode | wl.TOP_K | wl.TEMPERATURE, mode | wl.TOP_P, mode | wl.TOP_K | wl.TOP_P | wl.MIN_P],
+                    dtype=dtype, rep=[1.3] * 4, freq=[0.15] * 4, pres=[0.25] * 4, temperature=[1, 0.7, 1, 1],
+                    top_k=[0, 40, 0, 300], top_p=[1, 1, 0.8, 0.9], min_p=[1, 1, 1, 0.01], hist=hist, bias=bias,
+                    seed=[3, 4, 5, 6])
+    dev = sonic.DeviceSample(w)
+    dev.run()
+    got = dev.results()
+    assert header_error_word(dev) == 0
+    ref = oracle.sample(w)
+    compare_sample(got, ref, w)
