@@ -48,6 +48,7 @@ constexpr int CLS_GREEDY = 0;                 // streaming path, argmax only
 constexpr int CLS_TOPK = 1;                   // streaming path, candidates + merge
 constexpr int CLS_EXACT = 2;                  // full-vocabulary exact path only
 
+constexpr int WS_FAILED_ROWS = 1;              // workspace header word: rows of the current call the merge kernel could not prove
 constexpr uint32_t ST_FAILED = 0x1;           // streaming path could not prove the row
 constexpr uint32_t ST_BADID = 0x2;            // a list id was out of range
 constexpr unsigned int ERR_TIMEOUT = 0x1;     // workspace header: a bounded mbarrier wait expired
@@ -315,6 +316,65 @@ __device__ __forceinline__ void bitonic_sort_desc(unsigned long long *a, int m, 
             const int jn = (j > 1) ? (j >> 1) : k2;          // partner distance of the next stage
             if (j >= 64 || jn >= 64 || (k2 == m && j == 1)) sync(); else __syncwarp();
         }
+    }
+}
+
+// The same sort by a whole CTA, with every thread holding two adjacent elements in registers: the stages whose
+// partner distance is at most 32 run on shuffles (distance 1 inside the thread) and only the wider ones go
+// through shared memory with a block barrier.  m is a power of two; zeros may pad the tail.  Not inlined and
+// with rolled loops: one compact copy of the code serves every caller.
+template <int THREADS>
+__device__ __noinline__ void bitonic_sort_desc_cta(unsigned long long *a, int m, int tid) {
+    const int mm = max(m, 64);                           // whole warps take part (64 elements each)
+    auto tail = [&](unsigned long long &x0, unsigned long long &x1, int e, int k2, int jtop) {
+        const bool desc = ((e & k2) == 0);
+#pragma unroll 1
+        for (int j = jtop; j >= 2; j >>= 1) {
+            const unsigned long long o0 = __shfl_xor_sync(0xFFFFFFFFu, x0, j >> 1);
+            const unsigned long long o1 = __shfl_xor_sync(0xFFFFFFFFu, x1, j >> 1);
+            const bool take_max = (desc == ((e & j) == 0));
+            x0 = take_max ? max(x0, o0) : min(x0, o0);
+            x1 = take_max ? max(x1, o1) : min(x1, o1);
+        }
+        const unsigned long long hi = max(x0, x1), lo = min(x0, x1);
+        x0 = desc ? hi : lo;
+        x1 = desc ? lo : hi;
+    };
+#pragma unroll 1
+    for (int base = 0; base < mm; base += 2 * THREADS) {
+        const int e = base + 2 * tid;
+        if (e < mm) {                                    // uniform over the warp
+            unsigned long long x0 = (e < m) ? a[e] : 0ull, x1 = (e + 1 < m) ? a[e + 1] : 0ull;
+#pragma unroll 1
+            for (int k2 = 2; k2 <= 64; k2 <<= 1) tail(x0, x1, e, k2, k2 >> 1);
+            if (e < m) a[e] = x0;
+            if (e + 1 < m) a[e + 1] = x1;
+        }
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int k2 = 128; k2 <= mm; k2 <<= 1) {
+#pragma unroll 1
+        for (int j = k2 >> 1; j >= 64; j >>= 1) {
+            for (int i = tid; i < (mm >> 1); i += THREADS) {
+                const int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
+                const int hi = lo | j;
+                const unsigned long long x = a[lo], y = a[hi];
+                const bool desc = ((lo & k2) == 0);
+                if ((x < y) == desc) { a[lo] = y; a[hi] = x; }
+            }
+            __syncthreads();
+        }
+#pragma unroll 1
+        for (int base = 0; base < mm; base += 2 * THREADS) {
+            const int e = base + 2 * tid;
+            if (e < mm) {
+                unsigned long long x0 = a[e], x1 = a[e + 1];
+                tail(x0, x1, e, k2, 32);
+                a[e] = x0; a[e + 1] = x1;
+            }
+        }
+        __syncthreads();
     }
 }
 

@@ -523,7 +523,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
             const int m = next_pow2(nn);
             for (int i = nn + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
             __syncthreads();
-            bitonic_sort_desc<EX_THREADS>(sortbuf, m, x.tid);
+            bitonic_sort_desc_cta<EX_THREADS>(sortbuf, m, x.tid);
             SONIC_STAMP(7);
             // running count / mass in ranking order; each thread owns a contiguous chunk of the sorted list
             const int chunk = (nn + EX_THREADS - 1) / EX_THREADS;
@@ -753,7 +753,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
             const int m = next_pow2(n);
             for (int i = n + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
             __syncthreads();
-            bitonic_sort_desc<EX_THREADS>(sortbuf, m, x.tid);
+            bitonic_sort_desc_cta<EX_THREADS>(sortbuf, m, x.tid);
             for (int j = x.tid; j < n; j += EX_THREADS) {
                 unsigned long long kv = sortbuf[j];
                 P.out_vals[(size_t)row * P.ktop + j] = unkey((uint32_t)(kv >> 32));
@@ -823,6 +823,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);
         p_draft = (float)Pd;
         if (accept) flags |= F_ACCEPT;
+        SONIC_STAMP(20);
         // residual max(0, p - q) over the support, weights in fp64 (p - q cancels, so the weights must be accurate)
         const double Md = (double)x.Mf;
         auto wd = [&](int i) -> double {
@@ -832,6 +833,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         unsigned long long cdummy;
         ordered_totals<double>(x, wd, inS, std_, cdummy);
         const double Wd = std_.total;
+        SONIC_STAMP(21);
         auto rd = [&](int i) -> double {
             if (!(i < x.len && member(cut, x.keys[i], x.lo + i))) return 0.0;
             double r = exp((double)unkey(x.keys[i]) - Md) / Wd - (double)__ldg(q + x.lo + i);
@@ -844,6 +846,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
             const int t2 = ordered_find<double>(x, cell_to_u(a_draw) * str.total, rd, str, rw);
             if (t2 >= 0) token = t2;           // (verification rows report p(d), not the probability of this token)
         }
+        SONIC_STAMP(22);
     }
     if (leader) {
         emit_row(P, c, row, token, (float)token_prob, flags, (int)nS, p_draft);
@@ -876,7 +879,10 @@ sonic_exact_kernel(const KParams P) {
     const int cid = blockIdx.x / CL;
     const int nwords = (P.rows + 31) >> 5;
     for (int round = 0; round < 2; ++round) {
-        if (round == 1) pdl_wait_primary();
+        if (round == 1) {
+            pdl_wait_primary();
+            if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u) return;     // the merge kernel proved every row: nothing to scan
+        }
         __syncthreads();
         for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
         __syncthreads();

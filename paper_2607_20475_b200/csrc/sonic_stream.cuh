@@ -417,7 +417,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         const int m = next_pow2(Pn);
         for (int i = Pn + tid; i < m; i += THREADS) buf[i] = 0ull;
         csync();
-        bitonic_sort_desc<THREADS, Sync>(buf, m, tid);
+        bitonic_sort_desc_cta<THREADS>(buf, m, tid);
     }
     (void)sorted;
 #undef Pn
@@ -541,7 +541,8 @@ __device__ __forceinline__ void epilogue_index_order(int n, unsigned long long *
         for (int j = tid; j < m2; j += NT)
             v.ik[j] = (j < n) ? ((buf[j] << 32) | (unsigned long long)j) : 0ull;
         csync();
-        bitonic_sort_desc<NT, Sync>(v.ik, m2, tid);
+        if constexpr (NT >= 64) bitonic_sort_desc_cta<NT>(v.ik, m2, tid);
+        else bitonic_sort_desc<NT, Sync>(v.ik, m2, tid);
     }
 }
 
@@ -684,6 +685,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], STREAM_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (blockIdx.x == 0 && tid == 0) P.error[WS_FAILED_ROWS] = 0u;     // this call's count of rows the merge kernel cannot prove
     __syncthreads();
     pdl_launch_dependents();                   // the merge kernel may start launching; it waits for this grid to finish
 
@@ -1123,7 +1125,7 @@ sonic_merge_kernel(const KParams P, const int tiles) {
         return;
     }
     const bool ok = merge_topk_row<MERGE_THREADS, BlockSync>(P, c, row, tiles, reinterpret_cast<unsigned long long *>(smem_raw), s_merge, tid);
-    if (tid == 0 && !ok) rs->status = ST_FAILED;
+    if (tid == 0 && !ok) { rs->status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
 }
 
 }  // namespace sonic
