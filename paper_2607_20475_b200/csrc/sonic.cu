@@ -65,8 +65,14 @@ static size_t ws_bytes_for(int rows) { return WS_HEADER + (size_t)rows * WS_ROW;
 
 static int g_max_clusters[64];      // co-resident 8-CTA clusters of the exact kernel, per device
 static int g_sm_count[64];
+// Per device: a side stream and two events.  The exact kernel's first round (rows that are its own by class) is
+// forked onto the side stream at the start of a call and joined at its end, so that it runs beside the
+// streaming and merge kernels of the caller's stream.  One call at a time uses them (g_launch_mutex).
+static cudaStream_t g_side[64];
+static cudaEvent_t g_fork[64], g_join[64];
+static std::mutex g_launch_mutex[64];
 
-static int configure_once(int *max_clusters, int *sm_count) {
+static int configure_once(int *max_clusters, int *sm_count, int *device) {
     static std::once_flag once[64];
     static cudaError_t result[64];
     int dev = 0;
@@ -99,12 +105,16 @@ static int configure_once(int *max_clusters, int *sm_count) {
             r = cudaOccupancyMaxActiveClusters(&n, (const void *)sonic_exact_kernel<0>, &cfg);
         }
         g_max_clusters[dev] = n;
+        if (r == cudaSuccess) r = cudaStreamCreateWithFlags(&g_side[dev], cudaStreamNonBlocking);
+        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_fork[dev], cudaEventDisableTiming);
+        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_join[dev], cudaEventDisableTiming);
         result[dev] = r;
     });
     if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "kernel configuration");
     if (g_max_clusters[dev] < 1) return fail(SONIC_ECUDA, "no 8-CTA cluster of the exact kernel fits on this device");
     *max_clusters = g_max_clusters[dev];
     *sm_count = g_sm_count[dev] > 0 ? g_sm_count[dev] : 1;
+    *device = dev;
     return SONIC_OK;
 }
 
@@ -112,8 +122,8 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
     if (ws_bytes < ws_bytes_for(P.rows)) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows");
-    int max_clusters = 0, sm_count = 1;
-    int rc = configure_once(&max_clusters, &sm_count);
+    int max_clusters = 0, sm_count = 1, dev = 0;
+    int rc = configure_once(&max_clusters, &sm_count, &dev);
     if (rc != SONIC_OK) return rc;
     // the layout depends on the row capacity the workspace was sized for, recovered from its size
     const size_t cap_rows = (ws_bytes - WS_HEADER) / WS_ROW;
@@ -128,13 +138,35 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     const long long nitems_ll = (long long)tiles * P.rows;
     if (nitems_ll > 0x7FFFFFFF) return fail(SONIC_ESHAPE, "rows x tiles too large");
     const int nitems = (int)nitems_ll;
+    std::lock_guard<std::mutex> lock(g_launch_mutex[dev]);
+    cudaError_t e;
+
+    // Fork: the exact kernel's first round goes to the side stream BEFORE the streaming kernel is launched, so that
+    // its clusters (one SM per CTA) are placed first; clusters without a row leave at once and the streaming
+    // kernel's CTAs, which take their tiles from a queue, fill whatever is free.
+    cudaLaunchConfig_t xcfg;
+    memset(&xcfg, 0, sizeof(xcfg));
+    xcfg.gridDim = dim3((P.rows < max_clusters ? P.rows : max_clusters) * CL);
+    xcfg.blockDim = dim3(EX_THREADS);
+    xcfg.dynamicSmemBytes = EXACT_SMEM;
+    xcfg.stream = g_side[dev];
+    if ((e = cudaEventRecord(g_fork[dev], st)) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+    if ((e = cudaStreamWaitEvent(g_side[dev], g_fork[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
+    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<0>, P, 1);
+    else e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<1>, P, 1);
+    if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (first round)");
+    if ((e = cudaEventRecord(g_join[dev], g_side[dev])) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+
     const int grid1 = nitems < sm_count * 3 ? nitems : sm_count * 3;       // persistent: three CTAs per SM
-    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems);
-    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems);
-    cudaError_t e = cudaGetLastError();
+    // a CTA's first request to the work queue: seven eighths of an even share, at least one item
+    int chunk = (int)((7ll * nitems) / (8ll * grid1));
+    chunk = chunk < 1 ? 1 : chunk;
+    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems, chunk);
+    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems, chunk);
+    e = cudaGetLastError();
     if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
-    // merge and exact kernels are programmatic dependents: they may begin launching while their
-    // predecessor still runs and synchronise on it inside the kernel
+    // the merge kernel and the exact kernel's second round are programmatic dependents: they may begin launching
+    // while their predecessor still runs and synchronise on it inside the kernel
     cudaLaunchAttribute pdl;
     pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl.val.programmaticStreamSerializationAllowed = 1;
@@ -149,13 +181,15 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     e = cudaLaunchKernelEx(&cfg, sonic_merge_kernel, P, tiles);
     if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
 
-    cfg.gridDim = dim3((P.rows < max_clusters ? P.rows : max_clusters) * CL);
+    cfg.gridDim = xcfg.gridDim;
     cfg.blockDim = dim3(EX_THREADS);
     cfg.dynamicSmemBytes = EXACT_SMEM;
-    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P);
-    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P);
-    if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch");
+    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P, 2);
+    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P, 2);
+    if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (second round)");
 
+    // join: everything after this call in the caller's stream sees the first round's rows too
+    if ((e = cudaStreamWaitEvent(st, g_join[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
     if (P.op == OP_VERIFY) {
         sonic_verify_combine_kernel<<<(B_requests + 127) / 128, 128, 0, st>>>(P, B_requests);
         e = cudaGetLastError();

@@ -858,7 +858,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
 // Persistent clusters over the rows that need this path.
 template <int DT>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
-sonic_exact_kernel(const KParams P) {
+sonic_exact_kernel(const KParams P, const int rounds) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     ExactCtx x;
     x.rank = (int)cg::this_cluster().block_rank();
@@ -871,14 +871,16 @@ sonic_exact_kernel(const KParams P) {
     unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192);
     uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8);
 
-    // Two rounds.  Round 0: the rows that belong to this path by class (known from the inputs alone,
-    // so this round may run while the merge kernel is still busy).  Round 1, after the merge kernel
-    // has completed: the rows it could not prove.  In each round every CTA marks the rows of ALL
-    // requests and the marked rows are dealt round-robin to the clusters (all CTAs derive the same list).
+    // Two rounds, launched separately (`rounds` is the set this launch runs).  Round 0: the rows that belong to
+    // this path by class, known from the inputs alone, so this launch runs beside the streaming and merge
+    // kernels.  Round 1, a programmatic dependent of the merge kernel: the rows that kernel could not prove.  In
+    // each round every CTA marks the rows of ALL requests and the marked rows are dealt round-robin to the
+    // clusters (all CTAs derive the same list).
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;
     const int nwords = (P.rows + 31) >> 5;
     for (int round = 0; round < 2; ++round) {
+        if (!((rounds >> round) & 1)) continue;
         if (round == 1) {
             pdl_wait_primary();
             if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u) return;     // the merge kernel proved every row: nothing to scan

@@ -649,6 +649,8 @@ struct StageMeta {
     int patch;                                 // 0 none, 1 the producer filtered the lists into hits[], 2 consumers scan the lists
     int npen, nbias;                           // hits of this tile
     int hb;                                    // which hit buffer holds them
+    int stop;                                  // no more tiles for this CTA (nothing else in the entry is valid)
+    int next_row, next_tile;                   // the tile that follows (-1: none, or not known yet)
 };
 struct Hit { int li; int payload; };           // element within the tile; history count, or the bias as float bits
 
@@ -669,7 +671,7 @@ struct StreamShared {
 
 template <int DT>
 __global__ void __launch_bounds__(STREAM_CTA_THREADS, 3)
-sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
+sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const int chunk) {
     constexpr int VEC = VecTraits<DT>::VEC, NV = VecTraits<DT>::NV, NSTAGE = VecTraits<DT>::NSTAGE;
     constexpr int ELT = VecTraits<DT>::ELT;
     constexpr int STAGE_BYTES = CTA_TILE * ELT;
@@ -689,13 +691,11 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
     __syncthreads();
     pdl_launch_dependents();                   // the merge kernel may start launching; it waits for this grid to finish
 
-    // this CTA's contiguous share of the (row, tile) items
-    const int item_lo = (int)(((long long)nitems * blockIdx.x) / gridDim.x);
-    const int item_hi = (int)(((long long)nitems * (blockIdx.x + 1)) / gridDim.x);
-
     if (warp == STREAM_WARPS) {
         // ------------------------------------------------------------ producer warp
-        // A CTA takes a contiguous run of tiles, so consecutive tiles mostly belong to one row.  Per tile the
+        // The (row, tile) items are handed out through a counter in the workspace, so CTAs that become resident
+        // late (the SMs may be shared with the exact kernel) find less or no work instead of holding back a fixed
+        // share.  Per tile the
         // producer (1) waits for a free stage, describes the tile and issues its bulk copy, then (2) prepares
         // the NEXT tile while the ring is busy.  On a new row that means one round of global loads (parameters
         // and sparse lists, kept in registers for the row's other tiles); on every tile, picking the list
@@ -795,10 +795,30 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
             return r;
         };
         const unsigned long long l2_policy = l2_evict_first_policy();
+        // Work queue: one counter of items.  A CTA first asks for `chunk` consecutive items (seven eighths of an
+        // even share: a contiguous run like a static split would give it) and then for single items, each
+        // requested one tile ahead (lane 0 keeps the raw result of the atomic until it is needed, so nothing
+        // waits for it).  The single items even out the tail and whatever CTAs that started late did not take.
+        unsigned int *queue = P.error + WS_QUEUE;
+        int run_lo = nitems, run_hi = nitems, nxt_raw = nitems;
+        if (lane == 0) run_lo = (int)atomicAdd(queue, (unsigned int)chunk);
+        run_lo = __shfl_sync(0xFFFFFFFFu, run_lo, 0);
+        run_hi = min(run_lo + chunk, nitems);
+        if (lane == 0 && run_lo < nitems) nxt_raw = (int)atomicAdd(queue, 1u);
+        auto current_item = [&]() -> int { return run_lo < run_hi ? run_lo : -1; };
+        auto advance = [&]() {
+            ++run_lo;
+            if (run_lo >= run_hi) {
+                run_lo = __shfl_sync(0xFFFFFFFFu, nxt_raw, 0);
+                run_hi = min(run_lo + 1, nitems);
+                if (lane == 0 && run_lo < nitems) nxt_raw = (int)atomicAdd(queue, 1u);
+            }
+        };
         int n = 0;
         Prep p_next{0, 0, 0};
-        if (item_lo < item_hi) p_next = prepare(item_lo / tiles, item_lo % tiles, 0);
-        for (int item = item_lo; item < item_hi; ++item, ++n) {
+        int item = current_item();
+        if (item >= 0) p_next = prepare(item / tiles, item % tiles, 0);
+        for (;; ++n) {
             const int s = n % NSTAGE;
             const RowCfg c = c_next;
             const Prep pr = p_next;
@@ -809,12 +829,21 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
                     return;
                 }
             }
+            if (item < 0) {                            // out of work: tell the consumers
+                if (lane == 0) { sh.meta[s].stop = 1; mbar_arrive(&sh.full[s]); }
+                break;
+            }
+            advance();
+            const int nxt = current_item();
             const int row = item / tiles, tile = item - row * tiles;
             __syncwarp();                              // the hit buffer's entries, written by all lanes, precede the arrival
             if (lane == 0) {
                 StageMeta &m = sh.meta[s];
                 m.cfg = c; m.row = row; m.tile = tile; m.skip = (c.cls == CLS_EXACT) ? 1 : 0;
                 m.patch = pr.patch; m.npen = pr.npen; m.nbias = pr.nbias; m.hb = n % (NSTAGE + 1);
+                m.stop = 0;
+                m.next_row = (nxt >= 0) ? nxt / tiles : -1;
+                m.next_tile = (nxt >= 0) ? nxt % tiles : -1;
                 if (c.cls == CLS_EXACT) {
                     mbar_arrive(&sh.full[s]);
                 } else {
@@ -829,28 +858,36 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems) {
             }
             __syncwarp();
             // hit buffer (n + 1) % (NSTAGE + 1) was last used by tile n - NSTAGE, which the consumers have left
-            if (item + 1 < item_hi) p_next = prepare((item + 1) / tiles, (item + 1) % tiles, (n + 1) % (NSTAGE + 1));
+            if (nxt >= 0) p_next = prepare(nxt / tiles, nxt % tiles, (n + 1) % (NSTAGE + 1));
+            item = nxt;
         }
         return;
     }
 
     // ---------------------------------------------------------------- consumer warps
-    int n = 0;
-    for (int item = item_lo; item < item_hi; ++item, ++n) {
+    // The grammar words of a warp tile (32 words, one coalesced load, handed to the lanes that need them by
+    // shuffles later) are requested one tile ahead: each stage names the tile that follows it.
+    uint32_t mword_pre = 0u;
+    int pre_row = -1, pre_tile = -1;
+    auto load_mask_words = [&](int row, int tile) -> uint32_t {
+        const int w = ((tile * CTA_TILE + warp * WARP_TILE) >> 5) + lane;
+        return (w < ((P.V + 31) >> 5)) ? __ldg(P.bitmask + (size_t)row * P.bitmask_stride + w) : 0u;
+    };
+    for (int n = 0;; ++n) {
         const int s = n % NSTAGE;
-        const int row = item / tiles, tile = item - row * tiles;
-        const int tile_base = tile * CTA_TILE;
-        const int wbase = tile_base + warp * WARP_TILE;
-        // requests that depend only on (row, tile) go out before the wait: the warp tile's 32 grammar
-        // words in one coalesced load (handed to the lanes that need them by shuffles later)
-        uint32_t mword = 0xFFFFFFFFu;
-        if (P.bitmask) {
-            const int w = (wbase >> 5) + lane;
-            mword = (w < ((P.V + 31) >> 5)) ? __ldg(P.bitmask + (size_t)row * P.bitmask_stride + w) : 0u;
-        }
         if (!mbar_wait(&sh.full[s], (n / NSTAGE) & 1)) {
             if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
             return;
+        }
+        if (sh.meta[s].stop) break;
+        const int row = sh.meta[s].row, tile = sh.meta[s].tile;
+        const int tile_base = tile * CTA_TILE;
+        const int wbase = tile_base + warp * WARP_TILE;
+        uint32_t mword = 0xFFFFFFFFu;
+        if (P.bitmask) {
+            mword = (row == pre_row && tile == pre_tile) ? mword_pre : load_mask_words(row, tile);
+            pre_row = sh.meta[s].next_row; pre_tile = sh.meta[s].next_tile;
+            if (pre_row >= 0) mword_pre = load_mask_words(pre_row, pre_tile);
         }
         const StageMeta &meta = sh.meta[s];
         if (!meta.skip) {
@@ -1088,8 +1125,10 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     const int tid = threadIdx.x;
     pdl_launch_dependents();                   // the exact kernel may start on the rows that are its own by class
     const RowCfg c = load_cfg(P, row);         // inputs only: independent of the streaming kernel
-    if (c.cls == CLS_EXACT) return;
+    if (c.cls == CLS_EXACT && row != 0) return;
     pdl_wait_primary();                        // tile records and candidates of the streaming kernel
+    if (row == 0 && tid == 0) P.error[WS_QUEUE] = 0u;    // the streaming kernel is done with its work counter
+    if (c.cls == CLS_EXACT) return;
     RowState *rs = P.rs + row;
     const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
     const unsigned int status = rs->status;
