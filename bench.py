@@ -380,7 +380,7 @@ def run_sonic(args, rank, world, local_rank):
         B = w0.B
         rows = B * (w0.K + 1) if name == "c4" else B
         achieved = bytes_call / (us_call * 1e-6) / 1e9
-        launches_per_call = 4 if name == "c4" else 3
+        launches_per_call = 5 if name == "c4" else 4     # exact (first round), stream, merge, exact (second round) [, verify combine]
         cpu_us, cpu_desc = oracle_time(name, w0, budget_s=15.0)
         out = {
             "metric": METRIC, "value": job_value(us_call, world), "unit": "us", "n_gpus": world, "steps": steps,

@@ -52,7 +52,16 @@ size_t sonic_workspace_bytes(int max_rows);
 /* Zeroes the control words of a workspace once after allocation (a memset
  * enqueued on `stream`, a cudaStream_t passed as void*).  The kernels restore
  * those words at the end of every call, so replays need no re-initialisation.
- * Two calls that use the same workspace must not overlap on the device. */
+ * Two calls that use the same workspace must not overlap on the device.
+ *
+ * Streams: sonic_sample, sonic_verify and sonic_topk enqueue one of their kernels
+ * (the exact path's rows that are known from the inputs alone) on an internal
+ * per-device stream that is forked from `stream` at the start of the call and
+ * joined to it before the call returns, so that kernel runs beside the others;
+ * work enqueued on `stream` after the call is ordered after all of it, and under
+ * stream capture the internal stream is captured with `stream`.  The internal
+ * stream and two events are created by the first such call on a device (before
+ * any capture is begun); calls on one device enqueue one at a time (a host mutex). */
 int sonic_workspace_init(void *workspace, size_t bytes, void *stream);
 
 /*
@@ -145,7 +154,8 @@ int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, 
  * per call; larger B is rejected with SONIC_ESHAPE.  The scratch memory is a fixed array
  * of about 2.1 MB inside the library image (SONIC_STATIC_MAX_ROWS rows of candidate
  * slots and control words); every GPU that loads the library holds it until the process
- * exits.  The function calls no cudaMalloc, cudaFree or other allocating routine.
+ * exits.  The function calls no cudaMalloc, cudaFree or other allocating routine, and it
+ * creates no stream or event: all of its kernels go to `stream`.
  *
  * The first call on each device resolves the array's device address and configures the
  * kernels; that first call should come before any stream capture is begun.  All calls on a device share

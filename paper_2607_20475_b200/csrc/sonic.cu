@@ -105,9 +105,6 @@ static int configure_once(int *max_clusters, int *sm_count, int *device) {
             r = cudaOccupancyMaxActiveClusters(&n, (const void *)sonic_exact_kernel<0>, &cfg);
         }
         g_max_clusters[dev] = n;
-        if (r == cudaSuccess) r = cudaStreamCreateWithFlags(&g_side[dev], cudaStreamNonBlocking);
-        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_fork[dev], cudaEventDisableTiming);
-        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_join[dev], cudaEventDisableTiming);
         result[dev] = r;
     });
     if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "kernel configuration");
@@ -118,7 +115,21 @@ static int configure_once(int *max_clusters, int *sm_count, int *device) {
     return SONIC_OK;
 }
 
-static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, int B_requests) {
+// Creates the side stream and its events on first use (never for sonic_topk_static, which forks nothing).
+static int ensure_side(int dev) {
+    static std::once_flag once[64];
+    static cudaError_t result[64];
+    std::call_once(once[dev], [&] {
+        cudaError_t r = cudaStreamCreateWithFlags(&g_side[dev], cudaStreamNonBlocking);
+        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_fork[dev], cudaEventDisableTiming);
+        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_join[dev], cudaEventDisableTiming);
+        result[dev] = r;
+    });
+    if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "side stream creation");
+    return SONIC_OK;
+}
+
+static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, int B_requests, bool fork = true) {
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
     if (ws_bytes < ws_bytes_for(P.rows)) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows");
@@ -143,19 +154,24 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
 
     // Fork: the exact kernel's first round goes to the side stream BEFORE the streaming kernel is launched, so that
     // its clusters (one SM per CTA) are placed first; clusters without a row leave at once and the streaming
-    // kernel's CTAs, which take their tiles from a queue, fill whatever is free.
+    // kernel's CTAs, which take their tiles from a queue, fill whatever is free.  Without the fork (the entry
+    // point that creates no resources) both rounds run in one launch after the merge kernel.
     cudaLaunchConfig_t xcfg;
     memset(&xcfg, 0, sizeof(xcfg));
     xcfg.gridDim = dim3((P.rows < max_clusters ? P.rows : max_clusters) * CL);
     xcfg.blockDim = dim3(EX_THREADS);
     xcfg.dynamicSmemBytes = EXACT_SMEM;
-    xcfg.stream = g_side[dev];
-    if ((e = cudaEventRecord(g_fork[dev], st)) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
-    if ((e = cudaStreamWaitEvent(g_side[dev], g_fork[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
-    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<0>, P, 1);
-    else e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<1>, P, 1);
-    if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (first round)");
-    if ((e = cudaEventRecord(g_join[dev], g_side[dev])) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+    if (fork) {
+        rc = ensure_side(dev);
+        if (rc != SONIC_OK) return rc;
+        xcfg.stream = g_side[dev];
+        if ((e = cudaEventRecord(g_fork[dev], st)) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+        if ((e = cudaStreamWaitEvent(g_side[dev], g_fork[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
+        if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<0>, P, 1);
+        else e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<1>, P, 1);
+        if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (first round)");
+        if ((e = cudaEventRecord(g_join[dev], g_side[dev])) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+    }
 
     const int grid1 = nitems < sm_count * 3 ? nitems : sm_count * 3;       // persistent: three CTAs per SM
     // a CTA's first request to the work queue: seven eighths of an even share, at least one item
@@ -184,12 +200,13 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     cfg.gridDim = xcfg.gridDim;
     cfg.blockDim = dim3(EX_THREADS);
     cfg.dynamicSmemBytes = EXACT_SMEM;
-    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P, 2);
-    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P, 2);
+    const int rounds = fork ? 2 : 3;
+    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P, rounds);
+    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P, rounds);
     if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (second round)");
 
     // join: everything after this call in the caller's stream sees the first round's rows too
-    if ((e = cudaStreamWaitEvent(st, g_join[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
+    if (fork && (e = cudaStreamWaitEvent(st, g_join[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
     if (P.op == OP_VERIFY) {
         sonic_verify_combine_kernel<<<(B_requests + 127) / 128, 128, 0, st>>>(P, B_requests);
         e = cudaGetLastError();
@@ -348,7 +365,7 @@ int sonic_topk_static(const void *logits, int dtype, int B, int V, int64_t row_s
     P.op = OP_TOPK;
     P.rows = B; P.V = V; P.dtype = dtype; P.logits = logits; P.row_stride = row_stride; P.ktop = k;
     P.out_vals = out_vals; P.out_idx = out_idx;
-    return launch_all(P, ws, bytes, (cudaStream_t)stream, B);
+    return launch_all(P, ws, bytes, (cudaStream_t)stream, B, /*fork=*/false);     // creates no stream or event either
 }
 
 const char *sonic_last_error(void) { return g_err; }
