@@ -87,7 +87,7 @@ struct MergeShared {
     unsigned int tkey;
     int n_p, n_m, pick;
     int found;
-    double scratch[THREADS];
+    alignas(16) double scratch[THREADS];      // also read as int4
 };
 
 // Writes the per-row outputs of the sample / verify operations.
@@ -260,10 +260,16 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             csync();
             bool done = false;
             bool fits = false;
+            int tots[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int w = 0; w < THREADS / 32; ++w) {
+                const int4 a4 = reinterpret_cast<const int4 *>(redi)[w * 2], b4 = reinterpret_cast<const int4 *>(redi)[w * 2 + 1];
+                tots[0] += a4.x; tots[1] += a4.y; tots[2] += a4.z; tots[3] += a4.w;
+                tots[4] += b4.x; tots[5] += b4.y; tots[6] += b4.z; tots[7] += b4.w;
+            }
 #pragma unroll
             for (int q = 6; q >= 0; --q) {                 // the highest threshold that still keeps k
-                int tot = 0;
-                for (int w = 0; w < THREADS / 32; ++w) tot += redi[w * 8 + q];
+                const int tot = tots[q];
                 if (!done && tot >= c.k) {
                     lo = th[q];
                     if (q < 6) hi = th[q + 1];
@@ -312,8 +318,14 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             lo = mn; hi = mx + 1ull;
         }
         MERGE_STAMP(11);
-        // eight-way search: seven interior thresholds per pass, one reduction for all of them
-        for (int it = 0; it < 24 && hi - lo > 1ull; ++it) {
+        // eight-way search: seven interior thresholds per pass.  The warps add their counts into one of two sets
+        // of totals in shared memory (the other set is cleared meanwhile), so a pass costs two block barriers
+        // and every thread reads just the seven totals.
+        int *tot2 = reinterpret_cast<int *>(sh.scratch);          // [2][8]
+        if (tid < 16) tot2[tid] = 0;
+        csync();
+        int pass = 0;
+        for (int it = 0; it < 24 && hi - lo > 1ull; ++it, ++pass) {
             const unsigned long long step = (hi - lo) >> 3;
             unsigned long long th[7];
 #pragma unroll
@@ -324,43 +336,67 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
 #pragma unroll
                 for (int q = 0; q < 7; ++q) cnt[q] += (key >= th[q]) ? 1 : 0;
             }
-            int *redi = reinterpret_cast<int *>(sh.scratch);
+            int *tot = tot2 + (pass & 1) * 8;
 #pragma unroll
             for (int q = 0; q < 7; ++q) {
                 cnt[q] = (int)__reduce_add_sync(0xFFFFFFFFu, (unsigned int)cnt[q]);
-                if ((tid & 31) == 0) redi[(tid >> 5) * 8 + q] = cnt[q];
+                if ((tid & 31) == 0 && cnt[q]) atomicAdd(&tot[q], cnt[q]);
             }
+            if (tid < 8) tot2[((pass + 1) & 1) * 8 + tid] = 0;     // the next pass's set (last read before the previous barrier)
             csync();
+            const int4 a4 = reinterpret_cast<const int4 *>(tot)[0], b4 = reinterpret_cast<const int4 *>(tot)[1];
+            const int tots[7] = {a4.x, a4.y, a4.z, a4.w, b4.x, b4.y, b4.z};
             bool done = false;
 #pragma unroll
             for (int q = 6; q >= 0; --q) {                 // the highest threshold that still keeps n
-                int tot = 0;
-                for (int w = 0; w < THREADS / 32; ++w) tot += redi[w * 8 + q];
-                if (!done && tot >= n) {
+                if (!done && tots[q] >= n) {
                     lo = th[q];
                     if (q < 6) hi = th[q + 1];
                     done = true;
-                    if (tot <= want_hi) it = 1000;          // tight enough
+                    if (tots[q] <= want_hi) it = 1000;      // tight enough
                 }
             }
             if (!done) hi = th[0];
             csync();
+#ifdef SONIC_TRACE
+            if (tid == 0 && row == (int)P.error[4]) P.error[28] += 1u;
+#endif
         }
-        // keep the keys >= lo, packed to the front (every position written is at or below one already read)
+        // keep the keys >= lo, packed to the front
         if (tid == 0) sh.count = 0;
         csync();
-        for (int i0 = 0; i0 < Pn; i0 += THREADS) {
-            const int i = i0 + tid;
-            const unsigned long long key = (i < Pn) ? buf[i] : 0ull;
-            const bool keep = (i < Pn) && key >= lo;
-            const unsigned int mk = __ballot_sync(0xFFFFFFFFu, keep);
-            csync();                                        // all reads of this trip precede its writes
-            int base = 0;
-            if ((tid & 31) == 0 && mk) base = atomicAdd(&sh.count, __popc(mk));
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
-            if (keep) buf[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
+        if (Pn <= MERGE_CAP / 2) {
+            // room for a copy: pack into the upper half without barriers, then move the survivors down
+            unsigned long long *up = buf + MERGE_CAP / 2;
+            for (int i0 = 0; i0 < Pn; i0 += THREADS) {
+                const int i = i0 + tid;
+                const unsigned long long key = (i < Pn) ? buf[i] : 0ull;
+                const bool keep = (i < Pn) && key >= lo;
+                const unsigned int mk = __ballot_sync(0xFFFFFFFFu, keep);
+                int base = 0;
+                if ((tid & 31) == 0 && mk) base = atomicAdd(&sh.count, __popc(mk));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (keep) up[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
+            }
             csync();
+            const int kept = sh.count;
+            for (int i = tid; i < kept; i += THREADS) buf[i] = up[i];
+        } else {
+            // in place (every position written is at or below one already read)
+            for (int i0 = 0; i0 < Pn; i0 += THREADS) {
+                const int i = i0 + tid;
+                const unsigned long long key = (i < Pn) ? buf[i] : 0ull;
+                const bool keep = (i < Pn) && key >= lo;
+                const unsigned int mk = __ballot_sync(0xFFFFFFFFu, keep);
+                csync();                                        // all reads of this trip precede its writes
+                int base = 0;
+                if ((tid & 31) == 0 && mk) base = atomicAdd(&sh.count, __popc(mk));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (keep) buf[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
+                csync();
+            }
         }
+        csync();
         Pn2 = sh.count;
         csync();
     }
