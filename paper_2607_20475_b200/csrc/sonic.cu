@@ -45,6 +45,7 @@ constexpr size_t WS_HEADER = 256;
 constexpr int MERGE_SMEM = MERGE_CAP * 8;
 constexpr int STREAM_SMEM_F32 = VecTraits<0>::NSTAGE * CTA_TILE * 4 + (int)sizeof(StreamShared<0>);
 constexpr int STREAM_SMEM_BF16 = VecTraits<1>::NSTAGE * CTA_TILE * 2 + CTA_TILE * 4 + (int)sizeof(StreamShared<1>);
+constexpr int SECOND_ROUND_CLUSTERS = 4;      // clusters of the exact kernel's second launch (rows the merge kernel failed)
 constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8 + 8192;
 
 static thread_local char g_err[256] = "";
@@ -197,7 +198,11 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     e = cudaLaunchKernelEx(&cfg, sonic_merge_kernel, P, tiles);
     if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
 
-    cfg.gridDim = xcfg.gridDim;
+    // rows the merge kernel cannot prove are rare: a few clusters suffice for the second round (the full set when
+    // this launch also runs the first round)
+    const int clusters2 = fork ? (P.rows < SECOND_ROUND_CLUSTERS ? P.rows : (max_clusters < SECOND_ROUND_CLUSTERS ? max_clusters : SECOND_ROUND_CLUSTERS))
+                               : (P.rows < max_clusters ? P.rows : max_clusters);
+    cfg.gridDim = dim3(clusters2 * CL);
     cfg.blockDim = dim3(EX_THREADS);
     cfg.dynamicSmemBytes = EXACT_SMEM;
     const int rounds = fork ? 2 : 3;
