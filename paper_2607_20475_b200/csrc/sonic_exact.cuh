@@ -876,6 +876,7 @@ sonic_exact_kernel(const KParams P, const int rounds) {
     // kernels.  Round 1, a programmatic dependent of the merge kernel: the rows that kernel could not prove.  In
     // each round every CTA marks the rows of ALL requests and the marked rows are dealt round-robin to the
     // clusters (all CTAs derive the same list).
+    KERNEL_T0(rounds == 2 ? 3 : 2);
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;
     const int nwords = (P.rows + 31) >> 5;
@@ -902,7 +903,7 @@ sonic_exact_kernel(const KParams P, const int rounds) {
             while (bits) {
                 const int row = (w << 5) + __ffs(bits) - 1;
                 bits &= bits - 1;
-                if (ordinal % ncl == cid) exact_row<DT>(P, row, x, sortbuf);
+                if (ordinal % ncl == cid) { exact_row<DT>(P, row, x, sortbuf); KERNEL_T1(rounds == 2 ? 3 : 2); }
                 ++ordinal;
             }
         }

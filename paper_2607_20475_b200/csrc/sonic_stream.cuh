@@ -111,6 +111,17 @@ __device__ __forceinline__ void emit_row(const KParams &P, const RowCfg &c, int 
 #define MERGE_STAMP(i) do { } while (0)
 #endif
 
+#ifdef SONIC_TRACE
+__device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
+#define STREAM_STAMP(i) do { if ((int)blockIdx.x == (int)P.error[5] && lane == 0) P.error[40 + (i)] = gtimer_lo(); } while (0)
+// kernel-level timeline: earliest start and latest end of kernel k (0 stream, 1 merge, 2 exact first launch, 3 exact second launch)
+#define KERNEL_T0(k) do { if (threadIdx.x == 0) atomicMin(&P.error[48 + 2 * (k)], gtimer_lo()); } while (0)
+#define KERNEL_T1(k) do { if (threadIdx.x == 0) atomicMax(&P.error[49 + 2 * (k)], gtimer_lo()); } while (0)
+#else
+#define KERNEL_T0(k) do { } while (0)
+#define KERNEL_T1(k) do { } while (0)
+#define STREAM_STAMP(i) do { } while (0)
+#endif
 constexpr int RANK_SORT_MAX = 512;            // at most this many candidates: sort by rank counting
 constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
 struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
@@ -693,7 +704,7 @@ struct Hit { int li; int payload; };           // element within the tile; histo
 template <int DT>
 struct StreamShared {
     static constexpr int NSTAGE = VecTraits<DT>::NSTAGE;
-    unsigned long long full[NSTAGE];           // producer -> consumers: stage described, copy issued (one arrival + the copy's bytes)
+    unsigned long long full[NSTAGE];           // producer -> consumers: two arrivals (copy issued, stage described) + the copy's bytes
     unsigned long long empty[NSTAGE];          // consumers -> producer: stage free (one arrival per consumer warp)
     StageMeta meta[NSTAGE];
     // per-stage scratch of the consumer warps (a fast warp may already be on the next tile, in the other stage)
@@ -719,8 +730,10 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
     ConsumerSync csync;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (warp == 0) STREAM_STAMP(0);
+    KERNEL_T0(0);
     if (tid == 0) {
-        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], STREAM_WARPS); }
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&sh.full[s], 2); mbar_init(&sh.empty[s], STREAM_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (blockIdx.x == 0 && tid == 0) P.error[WS_FAILED_ROWS] = 0u;     // this call's count of rows the merge kernel cannot prove
@@ -752,45 +765,36 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             const int *hct = P.hist_counts ? P.hist_counts + (size_t)req * P.hist_stride : nullptr;
             const int *bid = P.bias_ids ? P.bias_ids + (size_t)req * P.bias_stride : nullptr;
             const float *bvl = P.bias_vals ? P.bias_vals + (size_t)req * P.bias_stride : nullptr;
-            // the first round of loads goes out before the first use (the lengths arrive with the parameters:
-            // bound by the strides); the second half of a long history follows in a round of its own
-            constexpr int HALF = HPL / 2;
+            // every load goes out before the first use, in one round (the lengths arrive with the parameters, so
+            // the list loads are bound by the strides)
             const CfgRaw raw = fetch_cfg(P, row);
-            int id[HALF], ct[HALF];
+            int id[HPL], ct[HPL];
 #pragma unroll
-            for (int u = 0; u < HALF; ++u) {
+            for (int u = 0; u < HPL; ++u) {
                 const int t = lane + 32 * u;
                 id[u] = -1; ct[u] = 0;
                 if (hid && hct && t < P.hist_stride) { id[u] = __ldg(hid + t); ct[u] = __ldg(hct + t); }
             }
             int b0 = -1; float v0 = 0.0f;
             if (bid && bvl && lane < P.bias_stride) { b0 = __ldg(bid + lane); v0 = __ldg(bvl + lane); }
+            if (cached_row < 0) STREAM_STAMP(3);
             c_next = resolve_cfg(P, row, raw, &memo_k, &memo_G);
+            if (cached_row < 0) STREAM_STAMP(4);
             cached_row = row;
             row_patch = 0;
             if (c_next.cls == CLS_EXACT || !(c_next.hist_len > 0 || c_next.bias_len > 0)) return;
             row_patch = 2;
             if (c_next.hist_len > FILTER_HIST || c_next.bias_len > FILTER_BIAS) return;
             bool bad = false, big = false;
-            auto pack = [&](int t, int i, int cnt) -> uint32_t {
-                if (t >= c_next.hist_len) return 0u;
-                if (i < 0 || i >= P.V) { bad = true; return 0u; }
-                if (cnt > FILTER_COUNT_MAX) { big = true; return 0u; }
-                return (cnt > 0) ? ((uint32_t)i | ((uint32_t)cnt << 18)) : 0u;
-            };
 #pragma unroll
-            for (int u = 0; u < HALF; ++u) packed[u] = pack(lane + 32 * u, id[u], ct[u]);
-#pragma unroll
-            for (int u = 0; u < HALF; ++u) packed[HALF + u] = 0u;
-            if (c_next.hist_len > 32 * HALF) {
-#pragma unroll
-                for (int u = 0; u < HALF; ++u) {
-                    const int t = lane + 32 * (HALF + u);
-                    id[u] = -1; ct[u] = 0;
-                    if (t < c_next.hist_len) { id[u] = __ldg(hid + t); ct[u] = __ldg(hct + t); }
+            for (int u = 0; u < HPL; ++u) {
+                uint32_t pk = 0u;
+                if (lane + 32 * u < c_next.hist_len) {
+                    if (id[u] < 0 || id[u] >= P.V) bad = true;
+                    else if (ct[u] > FILTER_COUNT_MAX) big = true;
+                    else if (ct[u] > 0) pk = (uint32_t)id[u] | ((uint32_t)ct[u] << 18);
                 }
-#pragma unroll
-                for (int u = 0; u < HALF; ++u) packed[HALF + u] = pack(lane + 32 * (HALF + u), id[u], ct[u]);
+                packed[u] = pk;
             }
             b_id = -1; b_val = 0.0f;
             if (lane < c_next.bias_len) {
@@ -853,11 +857,19 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
         int n = 0;
         Prep p_next{0, 0, 0};
         int item = current_item();
-        if (item >= 0) p_next = prepare(item / tiles, item % tiles, 0);
+        STREAM_STAMP(1);
+        bool prepared = false;
+        auto issue_copy = [&](int row, int tile, int s) {         // lane 0: the tile's bulk copy (first arrival on full[s])
+            const int first = tile * CTA_TILE;
+            const int elems = min(CTA_TILE, ((P.V - first) + VEC - 1) / VEC * VEC);
+            const unsigned int bytes = (unsigned int)elems * ELT;
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(P.logits) +
+                                       ((size_t)row * (size_t)P.row_stride + (size_t)first) * ELT;
+            mbar_arrive_expect_tx(&sh.full[s], bytes);
+            bulk_load(stages + (size_t)s * STAGE_BYTES, src, bytes, &sh.full[s], l2_policy);
+        };
         for (;; ++n) {
             const int s = n % NSTAGE;
-            const RowCfg c = c_next;
-            const Prep pr = p_next;
             if (n >= NSTAGE) {
                 // the consumers have left tile n - NSTAGE: its stage and its hit buffer are free
                 if (!mbar_wait(&sh.empty[s], ((n / NSTAGE) - 1) & 1)) {
@@ -866,12 +878,25 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 }
             }
             if (item < 0) {                            // out of work: tell the consumers
-                if (lane == 0) { sh.meta[s].stop = 1; mbar_arrive(&sh.full[s]); }
+                if (lane == 0) { sh.meta[s].stop = 1; mbar_arrive(&sh.full[s]); mbar_arrive(&sh.full[s]); }
+                STREAM_STAMP(5);
                 break;
             }
+            const int row = item / tiles, tile = item - row * tiles;
+            bool early = false;
+            if (!prepared) {
+                // the CTA's first tile: its copy goes out before the row's parameters and lists are fetched (a
+                // row of the exact class is copied for nothing, once)
+                if (lane == 0) issue_copy(row, tile, s);
+                early = true;
+                p_next = prepare(row, tile, n % (NSTAGE + 1));
+                prepared = true;
+                STREAM_STAMP(2);
+            }
+            const RowCfg c = c_next;
+            const Prep pr = p_next;
             advance();
             const int nxt = current_item();
-            const int row = item / tiles, tile = item - row * tiles;
             __syncwarp();                              // the hit buffer's entries, written by all lanes, precede the arrival
             if (lane == 0) {
                 StageMeta &m = sh.meta[s];
@@ -880,16 +905,10 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 m.stop = 0;
                 m.next_row = (nxt >= 0) ? nxt / tiles : -1;
                 m.next_tile = (nxt >= 0) ? nxt % tiles : -1;
-                if (c.cls == CLS_EXACT) {
-                    mbar_arrive(&sh.full[s]);
-                } else {
-                    const int first = tile * CTA_TILE;
-                    const int elems = min(CTA_TILE, ((P.V - first) + VEC - 1) / VEC * VEC);
-                    const unsigned int bytes = (unsigned int)elems * ELT;
-                    const unsigned char *src = reinterpret_cast<const unsigned char *>(P.logits) +
-                                               ((size_t)row * (size_t)P.row_stride + (size_t)first) * ELT;
-                    mbar_arrive_expect_tx(&sh.full[s], bytes);
-                    bulk_load(stages + (size_t)s * STAGE_BYTES, src, bytes, &sh.full[s], l2_policy);
+                mbar_arrive(&sh.full[s]);              // second arrival: the stage is described
+                if (!early) {
+                    if (c.cls == CLS_EXACT) mbar_arrive(&sh.full[s]);
+                    else issue_copy(row, tile, s);
                 }
             }
             __syncwarp();
@@ -915,7 +934,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
             return;
         }
-        if (sh.meta[s].stop) break;
+        if (sh.meta[s].stop) { if (warp == 0) STREAM_STAMP(6); KERNEL_T1(0); break; }
         const int row = sh.meta[s].row, tile = sh.meta[s].tile;
         const int tile_base = tile * CTA_TILE;
         const int wbase = tile_base + warp * WARP_TILE;
@@ -1160,6 +1179,7 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     const int row = blockIdx.x;
     const int tid = threadIdx.x;
     pdl_launch_dependents();                   // the exact kernel may start on the rows that are its own by class
+    KERNEL_T0(1);
     const RowCfg c = load_cfg(P, row);         // inputs only: independent of the streaming kernel
     if (c.cls == CLS_EXACT && row != 0) return;
     pdl_wait_primary();                        // tile records and candidates of the streaming kernel
@@ -1201,6 +1221,7 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     }
     const bool ok = merge_topk_row<MERGE_THREADS, BlockSync>(P, c, row, tiles, reinterpret_cast<unsigned long long *>(smem_raw), s_merge, tid);
     if (tid == 0 && !ok) { rs->status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
+    KERNEL_T1(1);
 }
 
 }  // namespace sonic
