@@ -704,7 +704,7 @@ struct Hit { int li; int payload; };           // element within the tile; histo
 template <int DT>
 struct StreamShared {
     static constexpr int NSTAGE = VecTraits<DT>::NSTAGE;
-    unsigned long long full[NSTAGE];           // producer -> consumers: two arrivals (copy issued, stage described) + the copy's bytes
+    unsigned long long full[NSTAGE];           // producer -> consumers: stage described and copy issued (one arrival + the copy's bytes)
     unsigned long long empty[NSTAGE];          // consumers -> producer: stage free (one arrival per consumer warp)
     StageMeta meta[NSTAGE];
     // per-stage scratch of the consumer warps (a fast warp may already be on the next tile, in the other stage)
@@ -733,7 +733,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
     if (warp == 0) STREAM_STAMP(0);
     KERNEL_T0(0);
     if (tid == 0) {
-        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&sh.full[s], 2); mbar_init(&sh.empty[s], STREAM_WARPS); }
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], STREAM_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (blockIdx.x == 0 && tid == 0) P.error[WS_FAILED_ROWS] = 0u;     // this call's count of rows the merge kernel cannot prove
@@ -765,36 +765,45 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             const int *hct = P.hist_counts ? P.hist_counts + (size_t)req * P.hist_stride : nullptr;
             const int *bid = P.bias_ids ? P.bias_ids + (size_t)req * P.bias_stride : nullptr;
             const float *bvl = P.bias_vals ? P.bias_vals + (size_t)req * P.bias_stride : nullptr;
-            // every load goes out before the first use, in one round (the lengths arrive with the parameters, so
-            // the list loads are bound by the strides)
+            // the first round of loads goes out before the first use (the lengths arrive with the parameters:
+            // bound by the strides); the second half of a long history follows in a round of its own
+            constexpr int HALF = HPL / 2;
             const CfgRaw raw = fetch_cfg(P, row);
-            int id[HPL], ct[HPL];
+            int id[HALF], ct[HALF];
 #pragma unroll
-            for (int u = 0; u < HPL; ++u) {
+            for (int u = 0; u < HALF; ++u) {
                 const int t = lane + 32 * u;
                 id[u] = -1; ct[u] = 0;
                 if (hid && hct && t < P.hist_stride) { id[u] = __ldg(hid + t); ct[u] = __ldg(hct + t); }
             }
             int b0 = -1; float v0 = 0.0f;
             if (bid && bvl && lane < P.bias_stride) { b0 = __ldg(bid + lane); v0 = __ldg(bvl + lane); }
-            if (cached_row < 0) STREAM_STAMP(3);
             c_next = resolve_cfg(P, row, raw, &memo_k, &memo_G);
-            if (cached_row < 0) STREAM_STAMP(4);
             cached_row = row;
             row_patch = 0;
             if (c_next.cls == CLS_EXACT || !(c_next.hist_len > 0 || c_next.bias_len > 0)) return;
             row_patch = 2;
             if (c_next.hist_len > FILTER_HIST || c_next.bias_len > FILTER_BIAS) return;
             bool bad = false, big = false;
+            auto pack = [&](int t, int i, int cnt) -> uint32_t {
+                if (t >= c_next.hist_len) return 0u;
+                if (i < 0 || i >= P.V) { bad = true; return 0u; }
+                if (cnt > FILTER_COUNT_MAX) { big = true; return 0u; }
+                return (cnt > 0) ? ((uint32_t)i | ((uint32_t)cnt << 18)) : 0u;
+            };
 #pragma unroll
-            for (int u = 0; u < HPL; ++u) {
-                uint32_t pk = 0u;
-                if (lane + 32 * u < c_next.hist_len) {
-                    if (id[u] < 0 || id[u] >= P.V) bad = true;
-                    else if (ct[u] > FILTER_COUNT_MAX) big = true;
-                    else if (ct[u] > 0) pk = (uint32_t)id[u] | ((uint32_t)ct[u] << 18);
+            for (int u = 0; u < HALF; ++u) packed[u] = pack(lane + 32 * u, id[u], ct[u]);
+#pragma unroll
+            for (int u = 0; u < HALF; ++u) packed[HALF + u] = 0u;
+            if (c_next.hist_len > 32 * HALF) {
+#pragma unroll
+                for (int u = 0; u < HALF; ++u) {
+                    const int t = lane + 32 * (HALF + u);
+                    id[u] = -1; ct[u] = 0;
+                    if (t < c_next.hist_len) { id[u] = __ldg(hid + t); ct[u] = __ldg(hct + t); }
                 }
-                packed[u] = pk;
+#pragma unroll
+                for (int u = 0; u < HALF; ++u) packed[HALF + u] = pack(lane + 32 * (HALF + u), id[u], ct[u]);
             }
             b_id = -1; b_val = 0.0f;
             if (lane < c_next.bias_len) {
@@ -859,7 +868,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
         int item = current_item();
         STREAM_STAMP(1);
         bool prepared = false;
-        auto issue_copy = [&](int row, int tile, int s) {         // lane 0: the tile's bulk copy (first arrival on full[s])
+        auto issue_copy = [&](int row, int tile, int s) {         // lane 0: the tile's bulk copy (the arrival on full[s])
             const int first = tile * CTA_TILE;
             const int elems = min(CTA_TILE, ((P.V - first) + VEC - 1) / VEC * VEC);
             const unsigned int bytes = (unsigned int)elems * ELT;
@@ -878,17 +887,12 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 }
             }
             if (item < 0) {                            // out of work: tell the consumers
-                if (lane == 0) { sh.meta[s].stop = 1; mbar_arrive(&sh.full[s]); mbar_arrive(&sh.full[s]); }
+                if (lane == 0) { sh.meta[s].stop = 1; mbar_arrive(&sh.full[s]); }
                 STREAM_STAMP(5);
                 break;
             }
             const int row = item / tiles, tile = item - row * tiles;
-            bool early = false;
-            if (!prepared) {
-                // the CTA's first tile: its copy goes out before the row's parameters and lists are fetched (a
-                // row of the exact class is copied for nothing, once)
-                if (lane == 0) issue_copy(row, tile, s);
-                early = true;
+            if (!prepared) {                           // the CTA's first tile: nothing was prepared ahead
                 p_next = prepare(row, tile, n % (NSTAGE + 1));
                 prepared = true;
                 STREAM_STAMP(2);
@@ -905,11 +909,8 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 m.stop = 0;
                 m.next_row = (nxt >= 0) ? nxt / tiles : -1;
                 m.next_tile = (nxt >= 0) ? nxt % tiles : -1;
-                mbar_arrive(&sh.full[s]);              // second arrival: the stage is described
-                if (!early) {
-                    if (c.cls == CLS_EXACT) mbar_arrive(&sh.full[s]);
-                    else issue_copy(row, tile, s);
-                }
+                if (c.cls == CLS_EXACT) mbar_arrive(&sh.full[s]);      // nothing is copied for rows of the exact class
+                else issue_copy(row, tile, s);
             }
             __syncwarp();
             // hit buffer (n + 1) % (NSTAGE + 1) was last used by tile n - NSTAGE, which the consumers have left
