@@ -30,7 +30,7 @@ from paper_2607_20475_b200 import workloads as wl  # noqa: E402
 
 METRIC = "us_per_fused_sample_call"
 # DRAM bytes (read + write) of one call's kernels from the ncu captures summarised under profiles/ (per workload)
-NCU_TRAFFIC = {"c2": 17.80e6, "c3": 144.8e6}
+NCU_TRAFFIC = {"c2": 17.89e6, "c3": 143.0e6}
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -391,9 +391,9 @@ def run_sonic(args, rank, world, local_rank):
             "rows_per_s": rows * world / (us_call * 1e-6),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC.get(name), "peak_source": which, "kernel": "whole call",
-                         "note": "algorithmic bytes of the call / CUDA-event time of the whole call (stream + merge + "
-                                 "exact kernels, overlapped by programmatic dependent launch); the per-kernel split is "
-                                 "in profiles/"},
+                         "note": "algorithmic bytes of the call / CUDA-event time of the whole call (stream, merge and both "
+                                 "launches of the exact kernel, overlapped through a forked side stream and programmatic "
+                                 "dependent launch); the per-kernel split is in profiles/"},
             "cpu_baseline": {"value": cpu_us, "unit": "us", "cores": 1, "kind": "oracle", "sample": cpu_desc},
             "e2e": {"value": job_value(e2e_us, world), "unit": "us", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": launches_per_call * steps,
