@@ -161,3 +161,62 @@ def test_short_lists_per_tile_hit_lists(sonic, oracle, dtype, n_hist, n_bias):
     assert header_error_word(dev) == 0
     ref = oracle.sample(w)
     compare_sample(got, ref, w)
+
+
+def test_many_short_rows_through_the_work_queue(sonic, oracle):
+    # far more rows than resident CTAs, one ragged tile each: every CTA takes a run and then single tiles from the
+    # queue; afterwards the queue counter in the workspace header is back at zero
+    B, V = 1500, 777
+    rng = np.random.default_rng(4242)
+    x = (rng.standard_normal((B, V)) * 3).astype(np.float32)
+    kinds = np.arange(B) % 3
+    mode = np.where(kinds == 0, wl.GREEDY, np.where(kinds == 1, wl.TOP_K | wl.TEMPERATURE, wl.TOP_K | wl.TOP_P)).astype(np.uint32)
+    w = make_sample(x, mode, temperature=np.where(kinds == 1, 0.7, 1.0), top_k=np.where(kinds == 0, 0, 12),
+                    top_p=np.where(kinds == 2, 0.9, 1.0), seed=np.arange(B) + 5)
+    dev = sonic.DeviceSample(w)
+    for _ in range(2):
+        dev.run()
+    got = dev.results()
+    assert header_error_word(dev) == 0
+    import torch
+    assert int(dev.ws[8:12].view(torch.int32).cpu().numpy()[0]) == 0      # header word 2: the work counter
+    ref = oracle.sample(w)
+    compare_sample(got, ref, w)
+
+
+def test_two_host_threads_share_the_device(sonic, oracle):
+    # two threads, each with its own stream and workspace, call into the library at the same time (the calls
+    # enqueue one at a time and share the library's internal side stream)
+    import threading
+    import torch
+    ws = [wl.config1(), wl.config1()]
+    ws[1] = make_sample(np.asarray(ws[1].logits)[::-1].copy(), ws[1].mode[::-1].copy(), temperature=ws[1].temperature[::-1].copy(),
+                        top_k=ws[1].top_k[::-1].copy(), top_p=ws[1].top_p[::-1].copy(), min_p=ws[1].min_p[::-1].copy(),
+                        seed=ws[1].seed[::-1].copy(), offset=ws[1].offset[::-1].copy())
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    devs = []
+    for w, st in zip(ws, streams):
+        with torch.cuda.stream(st):
+            devs.append(sonic.DeviceSample(w))
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(i):
+        try:
+            with torch.cuda.stream(streams[i]):
+                for _ in range(50):
+                    devs[i].run()
+            streams[i].synchronize()
+        except Exception as exc:      # pragma: no cover - reported below
+            errors.append(exc)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors
+    torch.cuda.synchronize()
+    for w, dev in zip(ws, devs):
+        assert header_error_word(dev) == 0
+        compare_sample(dev.results(), oracle.sample(w), w)
