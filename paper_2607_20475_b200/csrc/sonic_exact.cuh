@@ -44,11 +44,13 @@ __device__ __forceinline__ bool tighter(const Cut &a, const Cut &b) {   // a kee
     return a.v > b.v || (a.v == b.v && a.idx < b.idx);
 }
 
+constexpr int ORD_GROUPS = SLICE_MAX / EX_WARPS / 128;     // groups of 128 elements in a warp's run, at most
 struct ExactShared {
     unsigned long long xch[2][CL][XV];
     unsigned long long vals[XV];
     unsigned long long wtot[EX_WARPS];
     unsigned long long wcnt[EX_WARPS];
+    unsigned long long gtot[EX_WARPS][ORD_GROUPS];   // ordered passes: totals of each warp's groups of 128 elements
     unsigned long long red_mass[HBINS / CL];
     unsigned int red_cnt[HBINS / CL];
     unsigned int ucount;
@@ -146,7 +148,8 @@ __device__ void ordered_totals(ExactCtx &x, WF wf, CF cf, OrderedState<T> &st, u
     const int wlo = x.warp * wch;
     T wt = T(0);
     unsigned long long cn = 0;
-    for (int i = wlo + x.lane; i < wlo + wch; i += 128) {      // four independent elements per trip (wch is a multiple of 64)
+    int g = 0;
+    for (int i = wlo + x.lane; i < wlo + wch; i += 128, ++g) {      // four independent elements per trip
         T w4[4];
         unsigned long long c4[4];
 #pragma unroll
@@ -156,14 +159,18 @@ __device__ void ordered_totals(ExactCtx &x, WF wf, CF cf, OrderedState<T> &st, u
             w4[u] = in ? wf(ii) : T(0);
             c4[u] = in ? cf(ii) : 0ull;
         }
+        // the trip's 128 consecutive elements form one group: its total is kept for ordered_find, and the warp
+        // total is the sum of the group totals in order (every lane computes the same values)
+        T ts = (w4[0] + w4[1]) + (w4[2] + w4[3]);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { wt += w4[u]; cn += c4[u]; }
+        for (int off = 16; off > 0; off >>= 1) ts += __shfl_xor_sync(0xFFFFFFFFu, ts, off);
+        if (x.lane == 0) x.sh->gtot[x.warp][g] = *reinterpret_cast<unsigned long long *>(&ts);
+        wt += ts;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) cn += c4[u];
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        wt += __shfl_xor_sync(0xFFFFFFFFu, wt, off);
-        cn += __shfl_xor_sync(0xFFFFFFFFu, cn, off);
-    }
+    for (int off = 16; off > 0; off >>= 1) cn += __shfl_xor_sync(0xFFFFFFFFu, cn, off);
     __syncthreads();
     if (x.lane == 0) { x.sh->wtot[x.warp] = *reinterpret_cast<unsigned long long *>(&wt); x.sh->wcnt[x.warp] = cn; }
     __syncthreads();
@@ -219,28 +226,46 @@ __device__ int ordered_find(ExactCtx &x, T target, WF wf, const OrderedState<T> 
             T run = st.cta_off + st.warp_off;
             int found = -1, last_member = -1;
             T fw = T(0), lw = T(0);
-            for (int i = wlo; i < wlo + wch; i += 32) {
-                const T wv = wf(i + x.lane);
-                T incl = wv;
+            // First pass: skip the groups of 128 elements that end before the target (their totals were left by
+            // ordered_totals).  Should rounding leave it without any positive element, a second pass scans the
+            // whole run.
+            for (int pass = 0; pass < 2 && found < 0 && last_member < 0; ++pass) {
+                int istart = wlo;
+                run = st.cta_off + st.warp_off;
+                if (pass == 0) {
+                    const int ngroups = (wch + 127) / 128;
+                    T acc = run;
+                    for (int gg = 0; gg + 1 < ngroups; ++gg) {      // never past the last group
+                        const T t = *reinterpret_cast<T *>(&x.sh->gtot[x.warp][gg]);
+                        if (acc + t > target) break;
+                        acc += t;
+                        istart += 128;
+                    }
+                    run = acc;
+                }
+                for (int i = istart; i < wlo + wch; i += 32) {
+                    const T wv = wf(i + x.lane);
+                    T incl = wv;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if (x.lane >= o) incl += up;
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                        if (x.lane >= o) incl += up;
+                    }
+                    const unsigned int hit = __ballot_sync(0xFFFFFFFFu, (run + incl > target) && (wv > T(0)));
+                    const unsigned int pos = __ballot_sync(0xFFFFFFFFu, wv > T(0));
+                    if (hit) {
+                        const int l = __ffs(hit) - 1;
+                        found = x.lo + i + l;
+                        fw = __shfl_sync(0xFFFFFFFFu, wv, l);
+                        break;
+                    }
+                    if (pos) {
+                        const int l = 31 - __clz(pos);
+                        last_member = x.lo + i + l;
+                        lw = __shfl_sync(0xFFFFFFFFu, wv, l);
+                    }
+                    run += __shfl_sync(0xFFFFFFFFu, incl, 31);
                 }
-                const unsigned int hit = __ballot_sync(0xFFFFFFFFu, (run + incl > target) && (wv > T(0)));
-                const unsigned int pos = __ballot_sync(0xFFFFFFFFu, wv > T(0));
-                if (hit) {
-                    const int l = __ffs(hit) - 1;
-                    found = x.lo + i + l;
-                    fw = __shfl_sync(0xFFFFFFFFu, wv, l);
-                    break;
-                }
-                if (pos) {
-                    const int l = 31 - __clz(pos);
-                    last_member = x.lo + i + l;
-                    lw = __shfl_sync(0xFFFFFFFFu, wv, l);
-                }
-                run += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
             if (found < 0) { found = last_member; fw = lw; }   // rounding between levels: last positive element
             if (x.lane == 0) { x.sh->flag = found; x.sh->vals[3] = *reinterpret_cast<unsigned long long *>(&fw); }
