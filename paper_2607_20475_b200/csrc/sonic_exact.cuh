@@ -146,10 +146,12 @@ template <typename T, typename WF, typename CF>
 __device__ void ordered_totals(ExactCtx &x, WF wf, CF cf, OrderedState<T> &st, unsigned long long &count_out) {
     const int wch = x.per / EX_WARPS;                    // elements per warp (multiple of 32)
     const int wlo = x.warp * wch;
+    const int lane = x.lane;
+    unsigned long long *gt = x.sh->gtot[x.warp];
     T wt = T(0);
     unsigned long long cn = 0;
     int g = 0;
-    for (int i = wlo + x.lane; i < wlo + wch; i += 128, ++g) {      // four independent elements per trip
+    for (int i = wlo + lane; i < wlo + wch; i += 128, ++g) {      // four independent elements per trip
         T w4[4];
         unsigned long long c4[4];
 #pragma unroll
@@ -164,7 +166,7 @@ __device__ void ordered_totals(ExactCtx &x, WF wf, CF cf, OrderedState<T> &st, u
         T ts = (w4[0] + w4[1]) + (w4[2] + w4[3]);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) ts += __shfl_xor_sync(0xFFFFFFFFu, ts, off);
-        if (x.lane == 0) x.sh->gtot[x.warp][g] = *reinterpret_cast<unsigned long long *>(&ts);
+        if (lane == 0) gt[g] = *reinterpret_cast<unsigned long long *>(&ts);
         wt += ts;
 #pragma unroll
         for (int u = 0; u < 4; ++u) cn += c4[u];
@@ -223,6 +225,7 @@ __device__ int ordered_find(ExactCtx &x, T target, WF wf, const OrderedState<T> 
         }
         if (cross_warp < 0) cross_warp = EX_WARPS - 1;    // rounding between levels
         if (x.warp == cross_warp) {
+            const int lane = x.lane, lo_g = x.lo;
             T run = st.cta_off + st.warp_off;
             int found = -1, last_member = -1;
             T fw = T(0), lw = T(0);
@@ -244,24 +247,24 @@ __device__ int ordered_find(ExactCtx &x, T target, WF wf, const OrderedState<T> 
                     run = acc;
                 }
                 for (int i = istart; i < wlo + wch; i += 32) {
-                    const T wv = wf(i + x.lane);
+                    const T wv = wf(i + lane);
                     T incl = wv;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
                         const T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                        if (x.lane >= o) incl += up;
+                        if (lane >= o) incl += up;
                     }
                     const unsigned int hit = __ballot_sync(0xFFFFFFFFu, (run + incl > target) && (wv > T(0)));
                     const unsigned int pos = __ballot_sync(0xFFFFFFFFu, wv > T(0));
                     if (hit) {
                         const int l = __ffs(hit) - 1;
-                        found = x.lo + i + l;
+                        found = lo_g + i + l;
                         fw = __shfl_sync(0xFFFFFFFFu, wv, l);
                         break;
                     }
                     if (pos) {
                         const int l = 31 - __clz(pos);
-                        last_member = x.lo + i + l;
+                        last_member = lo_g + i + l;
                         lw = __shfl_sync(0xFFFFFFFFu, wv, l);
                     }
                     run += __shfl_sync(0xFFFFFFFFu, incl, 31);
@@ -298,24 +301,31 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
     // that overlap), then added to the histogram
     // The mass of a bin is a 64-bit integer kept as two 32-bit words: the low word takes one atomic add whose
     // returned old value reveals a carry; the high word is touched only on a carry or by weights >= 2^-8.
-    auto add_mass = [&](int b, unsigned long long q) {
+    // local copies of what the element loop reads (the context and the cut arrive by reference: read through them,
+    // every access would go to memory)
+    const uint32_t *keys = x.keys;
+    unsigned int *hcnt = x.hcnt, *hm0 = x.hm0, *hm1 = x.hm1;
+    const int len = x.len, lo_g = x.lo, per = x.per, tid = x.tid, lane = x.lane;
+    const float Mf = x.Mf;
+    const Cut bs = base;
+    auto add_mass = [=](int b, unsigned long long q) {
         const unsigned int lo = (unsigned int)q, hi = (unsigned int)(q >> 32);
         unsigned int carry = 0;
-        if (lo) { const unsigned int old = atomicAdd(&x.hm0[b], lo); carry = (old + lo < old) ? 1u : 0u; }
-        if (hi + carry) atomicAdd(&x.hm1[b], hi + carry);
+        if (lo) { const unsigned int old = atomicAdd(&hm0[b], lo); carry = (old + lo < old) ? 1u : 0u; }
+        if (hi + carry) atomicAdd(&hm1[b], hi + carry);
     };
-    for (int i0 = 0; i0 < x.per; i0 += 4 * EX_THREADS) {
+    for (int i0 = 0; i0 < per; i0 += 4 * EX_THREADS) {
         int bin[4];
         unsigned long long q[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int i = i0 + u * EX_THREADS + x.tid;
+            const int i = i0 + u * EX_THREADS + tid;
             bin[u] = -1; q[u] = 0ull;
-            if (i < x.len) {
-                const uint32_t key = x.keys[i];
-                if (member(base, key, x.lo + i)) {
+            if (i < len) {
+                const uint32_t key = keys[i];
+                if (member(bs, key, lo_g + i)) {
                     bin[u] = digit(key);
-                    if (by_mass && bin[u] >= 0) q[u] = qweight(key, x.Mf);
+                    if (by_mass && bin[u] >= 0) q[u] = qweight(key, Mf);
                 }
             }
         }
@@ -334,12 +344,12 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
                     const unsigned int p2 = __reduce_add_sync(active, (unsigned int)(q[u] >> 40));
                     qs = (unsigned long long)p0 + ((unsigned long long)p1 << 20) + ((unsigned long long)p2 << 40);
                 }
-                if ((int)(__ffs(active) - 1) == x.lane) {
-                    atomicAdd(&x.hcnt[bin[u]], n);
+                if ((int)(__ffs(active) - 1) == lane) {
+                    atomicAdd(&hcnt[bin[u]], n);
                     if (by_mass) add_mass(bin[u], qs);
                 }
             } else {
-                atomicAdd(&x.hcnt[bin[u]], 1u);
+                atomicAdd(&hcnt[bin[u]], 1u);
                 if (by_mass) add_mass(bin[u], q[u]);
             }
         }
@@ -487,13 +497,30 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
                           unsigned long long *sortbuf) {
     unsigned long long target = need, in_bin = 0;
     const float Mf = x.Mf;
-    auto dig_a = [&](uint32_t key) -> int {
+    auto dig_a = [=](uint32_t key) -> int {
         float t = fminf(__fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f), 2047.0f);
         return 2047 - (int)t;
     };
     const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin, sortbuf);
     SONIC_STAMP(4);
-    auto dig_b = [&](uint32_t key) -> int {
+    // A bin is an interval of (M - y), hence of keys.  A conservative key interval (the exact one widened by a
+    // margin that covers the roundings of the digit arithmetic and of this computation) lets the later passes
+    // reject almost every element with two integer compares before the exact digit test.
+    const bool band_ok = (Mf > -CUDART_INF_F) && (Mf < CUDART_INF_F);
+    const float marg = fmaxf(fabsf(Mf), 64.0f) * 9.5367431640625e-07f;            // 2^-20 of the larger magnitude
+    auto key_band = [&](float d_lo, float d_hi, bool open_below, uint32_t &klo, uint32_t &khi) {   // M - y in [d_lo, d_hi)
+        klo = 0u; khi = 0xFFFFFFFFu;
+        if (!band_ok) return;
+        khi = okey((Mf - d_lo) + marg);
+        if (!open_below) klo = okey((Mf - d_hi) - marg);
+    };
+    uint32_t klo_a, khi_a;
+    {
+        const int n = 2047 - a;
+        key_band((float)n * 0.03125f, (float)(n + 1) * 0.03125f, n == 2047, klo_a, khi_a);
+    }
+    auto dig_b = [=](uint32_t key) -> int {
+        if (key < klo_a || key > khi_a) return -1;
         float t = __fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f);
         int aa = (int)fminf(t, 2047.0f);
         if (2047 - aa != a) return -1;
@@ -503,7 +530,15 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     int b = -1;
     if (in_bin > (unsigned long long)GATHER_FAST) b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin, sortbuf);
     SONIC_STAMP(5);
-    auto in_range = [&](uint32_t key) -> bool {
+    uint32_t klo = klo_a, khi = khi_a;
+    if (b >= 0 && a != 0) {                                      // (bin 0 of level 0 is open below: no finer band)
+        const int n = 2047 - a, m = 2047 - b;
+        const float base_d = (float)n + (float)m * 0.00048828125f;              // aa + m / 2048, exact in fp32
+        const float top_d = (m == 2047) ? (float)(n + 1) : base_d + 0.00048828125f;
+        key_band(base_d * 0.03125f, top_d * 0.03125f, false, klo, khi);
+    }
+    auto in_range = [=](uint32_t key) -> bool {
+        if (key < klo || key > khi) return false;
         if (dig_a(key) != a) return false;
         return b < 0 || dig_b(key) == b;
     };
@@ -512,20 +547,24 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         // CTA 0, which sorts them and picks the element that completes the target
         if (x.tid == 0) x.sh->ucount = 0;
         __syncthreads();
-        for (int i0 = 0; i0 < x.per; i0 += 4 * EX_THREADS) {
+        const uint32_t *keys = x.keys;
+        const int len = x.len, lo_g = x.lo, per = x.per, tid = x.tid, lane = x.lane;
+        unsigned int *ucount = &x.sh->ucount;
+        const Cut bs = base;
+        for (int i0 = 0; i0 < per; i0 += 4 * EX_THREADS) {
             uint32_t key[4];
             bool want[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * EX_THREADS + x.tid;
-                key[u] = (i < x.len) ? x.keys[i] : 0u;
-                want[u] = (i < x.len) && member(base, key[u], x.lo + i) && in_range(key[u]);
+                const int i = i0 + u * EX_THREADS + tid;
+                key[u] = (i < len) ? keys[i] : 0u;
+                want[u] = (i < len) && member(bs, key[u], lo_g + i) && in_range(key[u]);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * EX_THREADS + x.tid;
-                const unsigned int pos = warp_append(&x.sh->ucount, want[u], x.lane);
-                if (want[u] && pos < (unsigned int)GATHER_CAP) sortbuf[pos] = ((unsigned long long)key[u] << 32) | (uint32_t)(~(uint32_t)(x.lo + i));
+                const int i = i0 + u * EX_THREADS + tid;
+                const unsigned int pos = warp_append(ucount, want[u], lane);
+                if (want[u] && pos < (unsigned int)GATHER_CAP) sortbuf[pos] = ((unsigned long long)key[u] << 32) | (uint32_t)(~(uint32_t)(lo_g + i));
             }
         }
         __syncthreads();
@@ -591,7 +630,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     for (int pass = 0; pass < 3; ++pass) {
         const int nb = (pass < 2) ? 11 : 10;
         const int shift = 32 - pbits - nb;
-        auto dig_k = [&](uint32_t key) -> int {
+        auto dig_k = [=](uint32_t key) -> int {
             if (pbits && (key >> (32 - pbits)) != prefix) return -1;
             if (!in_range(key)) return -1;
             return (int)((key >> shift) & ((1u << nb) - 1u));
@@ -609,8 +648,11 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     if (r < 1) r = 1;
     if (r > in_bin) r = in_bin;
     const uint32_t v = prefix;
-    auto tie = [&](int i) -> unsigned long long {
-        return (i < x.len && x.keys[i] == v && member(base, v, x.lo + i)) ? 1ull : 0ull;
+    const uint32_t *tkeys = x.keys;
+    const int tlen = x.len, tlo = x.lo;
+    const Cut tbase = base;
+    auto tie = [=](int i) -> unsigned long long {
+        return (i < tlen && tkeys[i] == v && member(tbase, v, tlo + i)) ? 1ull : 0ull;
     };
     OrderedState<unsigned long long> st;
     unsigned long long ntie, wdummy;
@@ -815,11 +857,16 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     // final support: size and mass in one ordered pass, then the draw in index order
     uint32_t a_acc, a_draw;
     draw_cells(P, c, a_acc, a_draw);
-    auto wq = [&](int i) -> unsigned long long {
-        return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? qweight(x.keys[i], x.Mf) : 0ull;
+    // (the weight functions capture copies of what they read: a reference to the context would keep it in memory)
+    const uint32_t *skeys = x.keys;
+    const int slen = x.len, slo = x.lo;
+    const float sMf = x.Mf;
+    const Cut scut = cut;
+    auto wq = [=](int i) -> unsigned long long {
+        return (i < slen && member(scut, skeys[i], slo + i)) ? qweight(skeys[i], sMf) : 0ull;
     };
-    auto inS = [&](int i) -> unsigned long long {
-        return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? 1ull : 0ull;
+    auto inS = [=](int i) -> unsigned long long {
+        return (i < slen && member(scut, skeys[i], slo + i)) ? 1ull : 0ull;
     };
     OrderedState<unsigned long long> stq;
     unsigned long long nS;
@@ -851,17 +898,17 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         SONIC_STAMP(20);
         // residual max(0, p - q) over the support, weights in fp64 (p - q cancels, so the weights must be accurate)
         const double Md = (double)x.Mf;
-        auto wd = [&](int i) -> double {
-            return (i < x.len && member(cut, x.keys[i], x.lo + i)) ? exp((double)unkey(x.keys[i]) - Md) : 0.0;
+        auto wd = [=](int i) -> double {
+            return (i < slen && member(scut, skeys[i], slo + i)) ? exp((double)unkey(skeys[i]) - Md) : 0.0;
         };
         OrderedState<double> std_;
         unsigned long long cdummy;
         ordered_totals<double>(x, wd, inS, std_, cdummy);
         const double Wd = std_.total;
         SONIC_STAMP(21);
-        auto rd = [&](int i) -> double {
-            if (!(i < x.len && member(cut, x.keys[i], x.lo + i))) return 0.0;
-            double r = exp((double)unkey(x.keys[i]) - Md) / Wd - (double)__ldg(q + x.lo + i);
+        auto rd = [=](int i) -> double {
+            if (!(i < slen && member(scut, skeys[i], slo + i))) return 0.0;
+            double r = exp((double)unkey(skeys[i]) - Md) / Wd - (double)__ldg(q + slo + i);
             return r > 0.0 ? r : 0.0;
         };
         OrderedState<double> str;
