@@ -679,6 +679,13 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     x.lo = x.rank * x.per;
     x.len = max(0, min(V - x.lo, x.per));
     cg::this_cluster().sync();                               // every CTA of the cluster is resident before DSMEM traffic
+    if (P.op == OP_VERIFY && c.l < P.K && P.draft_probs) {
+        // verification rows read the draft distribution of their slice twice near the end of the row: ask for it now,
+        // one 128-byte line per thread and trip, so that those reads find it in L2
+        const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)V;
+        for (int i = x.tid * 32; i < x.len; i += EX_THREADS * 32)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(q + x.lo + i));
+    }
     SONIC_STAMP(0);
 #ifdef SONIC_TRACE
     SONIC_STAMP(12);
@@ -906,9 +913,10 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         ordered_totals<double>(x, wd, inS, std_, cdummy);
         const double Wd = std_.total;
         SONIC_STAMP(21);
+        const double inv_Wd = 1.0 / Wd;                        // p = w * (1 / W): one rounding more than w / W, far below the margins
         auto rd = [=](int i) -> double {
             if (!(i < slen && member(scut, skeys[i], slo + i))) return 0.0;
-            double r = exp((double)unkey(skeys[i]) - Md) / Wd - (double)__ldg(q + slo + i);
+            double r = exp((double)unkey(skeys[i]) - Md) * inv_Wd - (double)__ldg(q + slo + i);
             return r > 0.0 ? r : 0.0;
         };
         OrderedState<double> str;
