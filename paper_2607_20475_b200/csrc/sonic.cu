@@ -174,6 +174,12 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
         if ((e = cudaEventRecord(g_join[dev], g_side[dev])) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
     }
 
+    // after the fork every exit joins the side stream again (also the failing ones: the caller's stream, or its
+    // capture, must not be left with a branch that was never joined)
+    auto unwind = [&](int code) {
+        if (fork) cudaStreamWaitEvent(st, g_join[dev], 0);
+        return code;
+    };
     const int grid1 = nitems < sm_count * 3 ? nitems : sm_count * 3;       // persistent: three CTAs per SM
     // a CTA's first request to the work queue: seven eighths of an even share, at least one item
     int chunk = (int)((7ll * nitems) / (8ll * grid1));
@@ -181,7 +187,7 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems, chunk);
     else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems, chunk);
     e = cudaGetLastError();
-    if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
+    if (e != cudaSuccess) return unwind(fail_cuda(e, "stream kernel launch"));
     // the merge kernel and the exact kernel's second round are programmatic dependents: they may begin launching
     // while their predecessor still runs and synchronise on it inside the kernel
     cudaLaunchAttribute pdl;
@@ -196,7 +202,7 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     cfg.blockDim = dim3(MERGE_THREADS);
     cfg.dynamicSmemBytes = MERGE_SMEM;
     e = cudaLaunchKernelEx(&cfg, sonic_merge_kernel, P, tiles);
-    if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
+    if (e != cudaSuccess) return unwind(fail_cuda(e, "merge kernel launch"));
 
     // rows the merge kernel cannot prove are rare: a few clusters suffice for the second round (the full set when
     // this launch also runs the first round)
@@ -208,7 +214,7 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     const int rounds = fork ? 2 : 3;
     if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P, rounds);
     else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P, rounds);
-    if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (second round)");
+    if (e != cudaSuccess) return unwind(fail_cuda(e, "exact kernel launch (second round)"));
 
     // join: everything after this call in the caller's stream sees the first round's rows too
     if (fork && (e = cudaStreamWaitEvent(st, g_join[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
