@@ -444,21 +444,29 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             const int runs = (Pn + 31) >> 5;
             if (key != 0ull) {
                 int rank = lane;
-                for (int r = 0; r < runs; ++r) {
-                    if (r == warp) continue;
-                    const unsigned long long *run = buf + r * 32;
-                    int lo = 0;                                    // number of keys of the run above `key`
+                // four runs at a time: their binary searches are independent chains of shared-memory reads
+                for (int r0 = 0; r0 < runs; r0 += 4) {
+                    const unsigned long long *run[4];
+                    int lo[4];
 #pragma unroll
-                    for (int step = 16; step > 0; step >>= 1)
-                        if (run[lo + step - 1] > key) lo += step;
-                    if (lo < 32 && run[lo] > key) ++lo;            // covers a run whose 32 keys are all above
-                    rank += lo;
+                    for (int u = 0; u < 4; ++u) { run[u] = buf + min(r0 + u, runs - 1) * 32; lo[u] = 0; }
+#pragma unroll
+                    for (int step = 16; step > 0; step >>= 1) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (run[u][lo[u] + step - 1] > key) lo[u] += step;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (lo[u] < 32 && run[u][lo[u]] > key) ++lo[u];        // covers a run whose 32 keys are all above
+                        if (r0 + u < runs && r0 + u != warp) rank += lo[u];     // (lo[u] = number of keys of the run above `key`)
+                    }
                 }
                 dst[rank] = key;
             }
         }
         csync();
-        for (int i = tid; i < Pn; i += THREADS) buf[i] = dst[i];
+        for (int i = tid; i < n; i += THREADS) buf[i] = dst[i];       // only the n best are used from here on
         csync();
     } else {
         const int m = next_pow2(Pn);
