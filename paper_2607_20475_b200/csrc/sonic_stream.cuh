@@ -122,6 +122,7 @@ __device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm 
 #define KERNEL_T1(k) do { } while (0)
 #define STREAM_STAMP(i) do { } while (0)
 #endif
+constexpr int BITONIC_SLACK_SIZE = 2048;       // large n: the threshold search may stop anywhere up to this many keys
 constexpr int RANK_SORT_MAX = 512;            // at most this many candidates: sort by rank counting
 constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
 struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
@@ -306,11 +307,13 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     else return false;
     unsigned long long *sorted = buf;
     int Pn2 = Pn;
-    if (Pn > RANK_SORT_MAX && Pn > n + n / 2 + 64) {
-        // far more proven candidates than needed: search a key threshold that keeps between n and a little more
-        // than n of them (any such threshold keeps the n best), then sort only those.  The upper end is what the
-        // rank-counting sort takes in one go, else the next power of two (the bitonic sort's size).
-        const int want_hi = (n + n / 2 + 16 <= RANK_SORT_MAX) ? n + n / 2 + 16 : next_pow2(n);
+    // How many keys the sort below should get at most: what the rank sort takes in one go when n is small, else a
+    // bitonic size with slack above n (a wide window needs few search passes; sorting twice as many keys costs
+    // less than searching a narrow one).
+    const int want_hi = (n + n / 2 + 16 <= RANK_SORT_MAX) ? n + n / 2 + 16 : max(next_pow2(n), BITONIC_SLACK_SIZE);
+    if (Pn > RANK_SORT_MAX && Pn > want_hi) {
+        // more proven candidates than that: search a key threshold that keeps between n and want_hi of them (any
+        // such threshold keeps the n best), then sort only those
         unsigned long long lo = 0ull, hi = ~0ull;          // count(>= lo) >= n > count(>= hi)
         {
             // start from the range the keys actually span
