@@ -66,6 +66,7 @@ struct ExactCtx {
     int trace;
     unsigned int *tracep;
     float Mf;                                  // largest processed logit
+    float scale, inv_scale;                    // histogram bins per logit unit (a power of two) and its reciprocal
 };
 
 // All CTAs contribute XV values; afterwards every CTA holds all of them.
@@ -484,21 +485,22 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
 }
 
 constexpr int GATHER_CAP = MAX_TOPK;          // elements CTA 0 can sort
-constexpr int GATHER_FAST = 256;              // above this many elements in the crossing bin a second level pays off
+constexpr int GATHER_FAST = 1024;             // above this many elements in the crossing bin a second level pays off
 
 // Selection inside `base`:
 //   by_mass == false: the cut of the `need`-th largest element (1 <= need <= count inside base)
 //   by_mass == true : the cut of the smallest ranking prefix whose mass reaches p * (mass inside base)
-// Levels: two histograms uniform in (M - y) (1/32 then 2^-16 wide), which spread any
-// smooth logit distribution over many bins; then the few elements of the crossing bin
-// are gathered into CTA 0 and sorted.  Bins too crowded for that (massive ties) are
+// Levels: a histogram of 2048 bins uniform in (M - y) whose width (a power of two) is chosen so that the bins just
+// cover the row's finite range, and, if its crossing bin still holds more than GATHER_FAST elements, a second one
+// that splits that bin 2048 ways; they spread any smooth logit distribution over many bins.  Then the elements of
+// the crossing bin are gathered into CTA 0 and sorted.  Bins too crowded for that (massive ties) are
 // resolved by three more levels over the key bits and an ordered tie count.
 __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned long long need, float p,
                           unsigned long long *sortbuf) {
     unsigned long long target = need, in_bin = 0;
-    const float Mf = x.Mf;
+    const float Mf = x.Mf, scale = x.scale, inv_scale = x.inv_scale;
     auto dig_a = [=](uint32_t key) -> int {
-        float t = fminf(__fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f), 2047.0f);
+        float t = fminf(__fmul_rn(__fsub_rn(Mf, unkey(key)), scale), 2047.0f);
         return 2047 - (int)t;
     };
     const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin, sortbuf);
@@ -507,7 +509,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     // margin that covers the roundings of the digit arithmetic and of this computation) lets the later passes
     // reject almost every element with two integer compares before the exact digit test.
     const bool band_ok = (Mf > -CUDART_INF_F) && (Mf < CUDART_INF_F);
-    const float marg = fmaxf(fabsf(Mf), 64.0f) * 9.5367431640625e-07f;            // 2^-20 of the larger magnitude
+    const float marg = fmaxf(fabsf(Mf), 2048.0f * inv_scale) * 9.5367431640625e-07f;   // 2^-20 of the larger magnitude
     auto key_band = [&](float d_lo, float d_hi, bool open_below, uint32_t &klo, uint32_t &khi) {   // M - y in [d_lo, d_hi)
         klo = 0u; khi = 0xFFFFFFFFu;
         if (!band_ok) return;
@@ -517,11 +519,11 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
     uint32_t klo_a, khi_a;
     {
         const int n = 2047 - a;
-        key_band((float)n * 0.03125f, (float)(n + 1) * 0.03125f, n == 2047, klo_a, khi_a);
+        key_band((float)n * inv_scale, (float)(n + 1) * inv_scale, n == 2047, klo_a, khi_a);
     }
     auto dig_b = [=](uint32_t key) -> int {
         if (key < klo_a || key > khi_a) return -1;
-        float t = __fmul_rn(__fsub_rn(Mf, unkey(key)), 32.0f);
+        float t = __fmul_rn(__fsub_rn(Mf, unkey(key)), scale);
         int aa = (int)fminf(t, 2047.0f);
         if (2047 - aa != a) return -1;
         float f = fminf(__fmul_rn(__fsub_rn(t, (float)aa), 2048.0f), 2047.0f);
@@ -535,7 +537,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         const int n = 2047 - a, m = 2047 - b;
         const float base_d = (float)n + (float)m * 0.00048828125f;              // aa + m / 2048, exact in fp32
         const float top_d = (m == 2047) ? (float)(n + 1) : base_d + 0.00048828125f;
-        key_band(base_d * 0.03125f, top_d * 0.03125f, false, klo, khi);
+        key_band(base_d * inv_scale, top_d * inv_scale, false, klo, khi);
     }
     auto in_range = [=](uint32_t key) -> bool {
         if (key < klo || key > khi) return false;
@@ -757,7 +759,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     }
     bad = __syncthreads_or(bad);
     SONIC_STAMP(1);
-    uint32_t kmax = 0;
+    uint32_t kmax = 0, kmin = 0xFFFFFFFFu;      // kmin over the finite elements
     unsigned int nfin32 = 0;
     for (int l0 = x.tid * 4; l0 < x.per; l0 += EX_THREADS * 4) {   // per is a multiple of 1024: whole float4s
         const float4 z4 = *reinterpret_cast<const float4 *>(zf + l0);
@@ -768,27 +770,41 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
             const float y = c.temp ? __fdiv_rn(zz[u], c.tau) : zz[u];
             kk[u] = okey(y);
             kmax = max(kmax, kk[u]);
-            nfin32 += (kk[u] > KEY_NEG_INF && l0 + u < x.len) ? 1u : 0u;
+            const bool fin = (kk[u] > KEY_NEG_INF && l0 + u < x.len);
+            nfin32 += fin ? 1u : 0u;
+            if (fin) kmin = min(kmin, kk[u]);
         }
         *reinterpret_cast<uint4 *>(x.keys + l0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
     }
     unsigned long long nfin = nfin32;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, off));
+    for (int off = 16; off > 0; off >>= 1) {
+        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, off));
+        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, off));
+    }
     nfin = block_sum_u64(x, nfin);
     __syncthreads();
-    if (x.lane == 0) x.sh->wtot[x.warp] = kmax;
+    if (x.lane == 0) { x.sh->wtot[x.warp] = kmax; x.sh->wcnt[x.warp] = kmin; }
     __syncthreads();
-    for (int w = 0; w < EX_WARPS; ++w) kmax = max(kmax, (uint32_t)x.sh->wtot[w]);
+    for (int w = 0; w < EX_WARPS; ++w) { kmax = max(kmax, (uint32_t)x.sh->wtot[w]); kmin = min(kmin, (uint32_t)x.sh->wcnt[w]); }
     unsigned long long all[CL][XV];
     {
-        unsigned long long v[XV] = {kmax, nfin, 0, 0};
+        unsigned long long v[XV] = {kmax, nfin, kmin, 0};
         allgather(x, v, all);
     }
-    uint32_t Mkey = 0;
+    uint32_t Mkey = 0, mkey = 0xFFFFFFFFu;
     unsigned long long Nf = 0;
-    for (int r = 0; r < CL; ++r) { Mkey = max(Mkey, (uint32_t)all[r][0]); Nf += all[r][1]; }
+    for (int r = 0; r < CL; ++r) { Mkey = max(Mkey, (uint32_t)all[r][0]); Nf += all[r][1]; mkey = min(mkey, (uint32_t)all[r][2]); }
     x.Mf = unkey(Mkey);
+    // Histogram resolution: 2048 bins uniform in (M - y) that just cover the row's finite range, the bin width a power
+    // of two (so that scaling is exact); 32 bins per unit when the range is degenerate.
+    {
+        int e = 5;
+        const float spread = (Nf > 0) ? __fsub_rn(x.Mf, unkey(mkey)) : 0.0f;
+        if (spread > 0.0f && spread < CUDART_INF_F) e = max(-10, min(10, ilogbf(2040.0f / spread)));
+        x.scale = ldexpf(1.0f, e);
+        x.inv_scale = ldexpf(1.0f, -e);
+    }
     SONIC_STAMP(2);
     const bool leader = (x.rank == 0 && x.tid == 0);
 
