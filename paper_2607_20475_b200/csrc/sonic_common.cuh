@@ -334,12 +334,11 @@ __device__ __noinline__ void bitonic_sort_desc_cta(unsigned long long *a, int m,
             const unsigned long long o0 = __shfl_xor_sync(0xFFFFFFFFu, x0, j >> 1);
             const unsigned long long o1 = __shfl_xor_sync(0xFFFFFFFFu, x1, j >> 1);
             const bool take_max = (desc == ((e & j) == 0));
-            x0 = take_max ? max(x0, o0) : min(x0, o0);
-            x1 = take_max ? max(x1, o1) : min(x1, o1);
+            // keep mine if it is on the side this lane takes, else the partner's (one comparison per element)
+            x0 = ((x0 > o0) == take_max) ? x0 : o0;
+            x1 = ((x1 > o1) == take_max) ? x1 : o1;
         }
-        const unsigned long long hi = max(x0, x1), lo = min(x0, x1);
-        x0 = desc ? hi : lo;
-        x1 = desc ? lo : hi;
+        if ((x0 > x1) != desc) { const unsigned long long t = x0; x0 = x1; x1 = t; }
     };
 #pragma unroll 1
     for (int base = 0; base < mm; base += 2 * THREADS) {

@@ -999,7 +999,19 @@ sonic_exact_kernel(const KParams P, const int rounds) {
             while (bits) {
                 const int row = (w << 5) + __ffs(bits) - 1;
                 bits &= bits - 1;
-                if (ordinal % ncl == cid) { exact_row<DT>(P, row, x, sortbuf); KERNEL_T1(rounds == 2 ? 3 : 2); }
+                if (ordinal % ncl == cid) {
+#ifdef SONIC_TRACE
+                    const unsigned int tr0 = gtimer_lo();
+#endif
+                    exact_row<DT>(P, row, x, sortbuf);
+                    KERNEL_T1(rounds == 2 ? 3 : 2);
+#ifdef SONIC_TRACE
+                    if (threadIdx.x == 0 && x.rank == 0) {
+                        atomicMax(&P.error[56], ((gtimer_lo() - tr0) << 8) | (unsigned int)(row & 255));    // slowest row: ns << 8 | row
+                        atomicMin(&P.error[57], tr0);                                                   // first row start
+                    }
+#endif
+                }
                 ++ordinal;
             }
         }
