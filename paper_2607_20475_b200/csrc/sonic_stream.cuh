@@ -438,7 +438,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                     const bool up = ((lane & kk) == 0);            // this block of kk sorts descending
                     const bool first = ((lane & jj) == 0);         // the lower lane of the pair
                     const bool take_max = (up == first);
-                    key = take_max ? max(key, o) : min(key, o);
+                    key = ((key > o) == take_max) ? key : o;           // mine if it is on the side this lane takes
                 }
             }
             csync();                                               // every thread has read its key from buf
