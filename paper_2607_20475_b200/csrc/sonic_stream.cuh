@@ -165,20 +165,8 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     const bool strict = c.temp && !complete;            // keys are compared after the temperature division
     const uint32_t tykey = c.temp ? okey(__fdiv_rn(unkey(tkey), c.tau)) : tkey;
     const int total = sh.tcnt[tiles];
-    // candidates are fetched eight per thread at a time (independent loads), then filtered and packed
+    // candidates are fetched eight per lane at a time (independent loads), then filtered and packed
     constexpr int GB = 8;
-    auto fetch = [&](int j0, unsigned long long (&cd)[GB]) {
-#pragma unroll
-        for (int u = 0; u < GB; ++u) {
-            const int j = j0 + u * THREADS + tid;
-            cd[u] = 0ull;
-            if (j < total) {
-                int t = 0;
-                while (sh.tcnt[t + 1] <= j) ++t;
-                cd[u] = __ldcg(P.cand + (size_t)row * CAND_CAP + (size_t)t * cap_t + (j - sh.tcnt[t]));
-            }
-        }
-    };
     // proven candidate -> its key after the temperature division (0 if it is not proven)
     auto proven_key = [&](unsigned long long cd, int j) -> unsigned long long {
         const uint32_t zk = (uint32_t)(cd >> 32);
@@ -246,21 +234,37 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         csync();
         for (int w = 0; w < THREADS / 32; ++w) kmax = max(kmax, red[w]);
         csync();
-        unsigned long long lo = 1ull, hi = kmax + 1ull;              // count(>= lo) >= k > ... count(>= hi) = 0
+        // every proven key is at least (cutoff key << 32): the search starts from the range the keys can span
+        unsigned long long lo = max(1ull, (unsigned long long)(c.temp ? tykey : tkey) << 32), hi = kmax + 1ull;   // count(>= lo) >= k > count(>= hi) = 0
         for (int it = 0; it < 24 && hi - lo > 1ull; ++it) {
             const unsigned long long step = (hi - lo) >> 3;
             unsigned long long th[7];
 #pragma unroll
             for (int q = 0; q < 7; ++q) th[q] = (step > 0) ? lo + step * (q + 1) : min(hi - 1ull, lo + 1ull + q);
             int cnt[7] = {0, 0, 0, 0, 0, 0, 0};
-            for (int j0 = 0; j0 < total; j0 += GB * THREADS) {
-                unsigned long long cd[GB];
-                fetch(j0, cd);
+            // one pass over the candidates, tile-major like the packing pass above
+            for (int ta = warp; ta < tiles; ta += 2 * NW) {
+                const int tb = ta + NW;
+                const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
+                const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
+                const unsigned long long *pa = P.cand + (size_t)row * CAND_CAP + (size_t)ta * cap_t;
+                const unsigned long long *pb = P.cand + (size_t)row * CAND_CAP + (size_t)tb * cap_t;
+                for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
+                    unsigned long long cd[GB];
 #pragma unroll
-                for (int u = 0; u < GB; ++u) {
-                    const unsigned long long out = proven_key(cd[u], j0 + u * THREADS + tid);
+                    for (int u = 0; u < HB; ++u) {
+                        const int j = j0 + u * 32 + lane;
+                        cd[u] = (j < na) ? __ldcg(pa + j) : 0ull;
+                        cd[HB + u] = (j < nb) ? __ldcg(pb + j) : 0ull;
+                    }
 #pragma unroll
-                    for (int q = 0; q < 7; ++q) cnt[q] += (out >= th[q]) ? 1 : 0;
+                    for (int u = 0; u < GB; ++u) {
+                        const int j = j0 + (u % HB) * 32 + lane;
+                        const bool valid = (u < HB) ? (j < na) : (j < nb);
+                        const unsigned long long out = proven_key(cd[u], valid ? 0 : total);
+#pragma unroll
+                        for (int q = 0; q < 7; ++q) cnt[q] += (out >= th[q]) ? 1 : 0;
+                    }
                 }
             }
             int *redi = reinterpret_cast<int *>(sh.scratch);
