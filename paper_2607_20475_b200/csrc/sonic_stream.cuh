@@ -572,6 +572,71 @@ __device__ __forceinline__ int epilogue_truncate(const RowCfg &c, int n, unsigne
     return n;
 }
 
+// The same for one warp and n <= WARP_EPILOGUE_MAX, in registers: a lane holds four consecutive weights, the
+// cumulative sums come from one shuffle scan, the cuts from votes.  Leaves the surviving prefix length in sh.n_p
+// and its total weight in cs[length - 1].
+template <typename SH>
+__device__ __forceinline__ void epilogue_truncate_warp(const RowCfg &c, int n, unsigned long long *buf, SH &sh, int lane) {
+    static_assert(WARP_EPILOGUE_MAX <= 128, "four elements per lane");
+    EpiView v(buf);
+    const double M = (double)unkey((uint32_t)(buf[0] >> 32));
+    double cs[4];
+    double run = 0.0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int j = lane * 4 + u;
+        run += (j < n) ? v.w[j] : 0.0;
+        cs[u] = run;
+    }
+    double incl = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const double excl = incl - run;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) cs[u] += excl;
+    const double Z = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    // first position (ranking order) where a cut falls: 4 * lane + u of the first element that satisfies `hit`
+    auto first_hit = [&](const bool (&hit)[4]) -> int {
+        int mine = 4;
+#pragma unroll
+        for (int u = 3; u >= 0; --u) if (hit[u]) mine = u;
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, mine < 4);
+        if (!m) return -1;
+        const int l = __ffs(m) - 1;
+        return l * 4 + __shfl_sync(0xFFFFFFFFu, mine, l);
+    };
+    int keep = n;
+    if (c.z & M_TOP_P) {
+        const double target = (double)c.p * Z;
+        bool hit[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) hit[u] = (lane * 4 + u < n) && cs[u] >= target;
+        const int j = first_hit(hit);
+        if (j >= 0) keep = min(keep, j + 1);
+    }
+    if (c.z & M_MIN_P) {
+        const double thr = M + log((double)c.theta);
+        bool hit[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = lane * 4 + u;
+            hit[u] = (j < n) && !((double)unkey((uint32_t)(buf[j] >> 32)) >= thr);     // first element below the threshold
+        }
+        const int j = first_hit(hit);
+        if (j >= 0) keep = min(keep, j);
+    }
+    // total weight of the survivors: the cumulative sum at position keep - 1
+    double mine = 0.0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) if (((keep - 1) & 3) == u) mine = cs[u];
+    const double W = __shfl_sync(0xFFFFFFFFu, mine, (keep - 1) >> 2);
+    if (lane == 0) { sh.n_p = keep; v.cs[keep - 1] = W; }     // the tail reads the survivors' total weight from there
+    __syncwarp();
+}
+
 // survivors in vocabulary-index order
 template <int NT, typename Sync>
 __device__ __forceinline__ void epilogue_index_order(int n, unsigned long long *buf, int tid) {
@@ -695,7 +760,7 @@ __device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row,
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
     __syncthreads();
     MERGE_STAMP(4);
-    if (tid < 32) epilogue_truncate<32, WarpSync>(c, n, buf, sh, tid);
+    if (tid < 32) epilogue_truncate_warp(c, n, buf, sh, tid);
     __syncthreads();
     n = sh.n_p;
     MERGE_STAMP(6);
