@@ -716,19 +716,53 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
         use_residual = cs[n - 1] > 0.0;
         csync();
     }
-    if (!use_residual) {
-        for (int j = tid; j < n; j += THREADS) cs[j] = w[(uint32_t)ik[j]];
+    bool picked = false;
+    if constexpr (NT == 32) {
+        if (!use_residual) {
+            // one warp, at most 128 survivors: the index-order cumulative weights stay in registers (a lane holds
+            // four consecutive positions), the drawn position comes from a vote
+            double csr[4];
+            double run = 0.0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = tid * 4 + u;
+                run += (j < n) ? w[(uint32_t)ik[j]] : 0.0;
+                csr[u] = run;
+            }
+            double incl = run;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (tid >= o) incl += up;
+            }
+            const double excl = incl - run;
+            const double target = u_draw * __shfl_sync(0xFFFFFFFFu, incl, 31);
+            int mine = 4;
+#pragma unroll
+            for (int u = 3; u >= 0; --u) if (tid * 4 + u < n && csr[u] + excl > target) mine = u;
+            const unsigned int m = __ballot_sync(0xFFFFFFFFu, mine < 4);
+            int j = n - 1;
+            if (m) { const int l = __ffs(m) - 1; j = l * 4 + __shfl_sync(0xFFFFFFFFu, mine, l); }
+            if (tid == 0) sh.pick = j;
+            picked = true;
+            __syncwarp();
+        }
+    }
+    if (!picked) {
+        if (!use_residual) {
+            for (int j = tid; j < n; j += THREADS) cs[j] = w[(uint32_t)ik[j]];
+            csync();
+            block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
+        }
+        const double R = cs[n - 1];
+        const double target = u_draw * R;
+        if (tid == 0) sh.pick = n - 1;
         csync();
-        block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
+        for (int j = tid; j < n; j += THREADS)
+            if (cs[j] > target && (j == 0 || !(cs[j - 1] > target))) sh.pick = j;
+        csync();
     }
     MERGE_STAMP(8);
-    const double R = cs[n - 1];
-    const double target = u_draw * R;
-    if (tid == 0) sh.pick = n - 1;
-    csync();
-    for (int j = tid; j < n; j += THREADS)
-        if (cs[j] > target && (j == 0 || !(cs[j - 1] > target))) sh.pick = j;
-    csync();
     if (tid == 0) {
         int j = sh.pick;
         int token = (int)(~(uint32_t)(ik[j] >> 32));
