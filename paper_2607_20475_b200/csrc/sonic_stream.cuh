@@ -128,16 +128,16 @@ constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of 
 struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
 
 template <int NT, typename Sync, typename SH>
-__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid);
+__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells);
 template <int THREADS, typename SH>
-__device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid);
+__device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells);
 
 // Row merge for top-k class rows (one CTA per row).  buf is MERGE_CAP 64-bit
 // words of shared memory.  Returns false if the candidates cannot prove the
 // row's answer.
 template <int THREADS, typename Sync>
 __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int tiles,
-                               unsigned long long *buf, MergeShared<THREADS> &sh, int tid) {
+                               unsigned long long *buf, MergeShared<THREADS> &sh, int tid, uint2 cells) {
     Sync csync;
     MERGE_STAMP(0);
     const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
@@ -502,9 +502,9 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     }
     // small supports are finished by one warp without block barriers
     if (n <= WARP_EPILOGUE_MAX) {
-        merge_epilogue_small<THREADS>(P, c, row, n, buf, sh, tid);
+        merge_epilogue_small<THREADS>(P, c, row, n, buf, sh, tid, cells);
     } else {
-        merge_epilogue<THREADS, Sync>(P, c, row, n, buf, sh, tid);
+        merge_epilogue<THREADS, Sync>(P, c, row, n, buf, sh, tid, cells);
     }
     return true;
 }
@@ -598,11 +598,8 @@ __device__ __forceinline__ void epilogue_truncate_warp(const RowCfg &c, int n, u
 #pragma unroll
     for (int u = 0; u < 4; ++u) cs[u] += excl;
     const double Z = __shfl_sync(0xFFFFFFFFu, incl, 31);
-    // first position (ranking order) where a cut falls: 4 * lane + u of the first element that satisfies `hit`
-    auto first_hit = [&](const bool (&hit)[4]) -> int {
-        int mine = 4;
-#pragma unroll
-        for (int u = 3; u >= 0; --u) if (hit[u]) mine = u;
+    // first position (ranking order) where a cut falls, from every lane's first hit among its four (4: none)
+    auto first_hit = [&](int mine) -> int {
         const unsigned int m = __ballot_sync(0xFFFFFFFFu, mine < 4);
         if (!m) return -1;
         const int l = __ffs(m) - 1;
@@ -611,21 +608,21 @@ __device__ __forceinline__ void epilogue_truncate_warp(const RowCfg &c, int n, u
     int keep = n;
     if (c.z & M_TOP_P) {
         const double target = (double)c.p * Z;
-        bool hit[4];
+        int mine = 4;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) hit[u] = (lane * 4 + u < n) && cs[u] >= target;
-        const int j = first_hit(hit);
+        for (int u = 3; u >= 0; --u) if (lane * 4 + u < n && cs[u] >= target) mine = u;
+        const int j = first_hit(mine);
         if (j >= 0) keep = min(keep, j + 1);
     }
     if (c.z & M_MIN_P) {
         const double thr = M + log((double)c.theta);
-        bool hit[4];
+        int mine = 4;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 3; u >= 0; --u) {
             const int j = lane * 4 + u;
-            hit[u] = (j < n) && !((double)unkey((uint32_t)(buf[j] >> 32)) >= thr);     // first element below the threshold
+            if (j < n && !((double)unkey((uint32_t)(buf[j] >> 32)) >= thr)) mine = u;          // first element below the threshold
         }
-        const int j = first_hit(hit);
+        const int j = first_hit(mine);
         if (j >= 0) keep = min(keep, j);
     }
     // total weight of the survivors: the cumulative sum at position keep - 1
@@ -675,7 +672,7 @@ __device__ __forceinline__ void epilogue_index_order(int n, unsigned long long *
 
 // draw, verification, selection and the row's outputs
 template <int NT, typename Sync, typename SH>
-__device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+__device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells) {
     Sync csync;
     constexpr int THREADS = NT;
     EpiView v(buf);
@@ -684,8 +681,7 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
     const double W = cs[n - 1];                 // still the ranking-order cumulative sums here
     csync();
     MERGE_STAMP(7);
-    uint32_t a_acc, a_draw;
-    draw_cells(P, c, a_acc, a_draw);
+    const uint32_t a_acc = cells.x, a_draw = cells.y;      // the row's Philox cells, drawn before the wait on the streaming kernel
     const double u_draw = cell_to_u(a_draw);
     uint32_t flags = 0;
     float p_draft = 0.0f;
@@ -774,7 +770,7 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
 
 
 template <int NT, typename Sync, typename SH>
-__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+__device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells) {
     Sync csync;
     epilogue_weights<NT>(n, buf, tid);
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
@@ -783,13 +779,13 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
     n = epilogue_truncate<NT, Sync>(c, n, buf, sh, tid);
     MERGE_STAMP(6);
     epilogue_index_order<NT, Sync>(n, buf, tid);
-    epilogue_tail<NT, Sync>(P, c, row, n, buf, sh, tid);
+    epilogue_tail<NT, Sync>(P, c, row, n, buf, sh, tid, cells);
 }
 
 // Small supports: the linear parts on warp 0 (warp-level synchronisation only), the weights and the quadratic
 // index ranking on the whole CTA.  Three block barriers in all.
 template <int THREADS, typename SH>
-__device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid) {
+__device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells) {
     epilogue_weights<THREADS>(n, buf, tid);
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
     __syncthreads();
@@ -799,7 +795,7 @@ __device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row,
     n = sh.n_p;
     MERGE_STAMP(6);
     epilogue_index_order<THREADS, BlockSync>(n, buf, tid);
-    if (tid < 32) epilogue_tail<32, WarpSync>(P, c, row, n, buf, sh, tid);
+    if (tid < 32) epilogue_tail<32, WarpSync>(P, c, row, n, buf, sh, tid, cells);
 }
 
 // What the producer hands to the consumers with each stage.
@@ -1297,6 +1293,9 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     KERNEL_T0(1);
     const RowCfg c = load_cfg(P, row);         // inputs only: independent of the streaming kernel
     if (c.cls == CLS_EXACT && row != 0) return;
+    // the row's two uniforms depend on the inputs alone: drawn here, while the streaming kernel may still be running
+    uint2 cells = make_uint2(0u, 0u);
+    if (P.op != OP_TOPK && c.cls == CLS_TOPK) draw_cells(P, c, cells.x, cells.y);
     pdl_wait_primary();                        // tile records and candidates of the streaming kernel
     if (row == 0 && tid == 0) P.error[WS_QUEUE] = 0u;    // the streaming kernel is done with its work counter
     if (c.cls == CLS_EXACT) return;
@@ -1334,7 +1333,7 @@ sonic_merge_kernel(const KParams P, const int tiles) {
         }
         return;
     }
-    const bool ok = merge_topk_row<MERGE_THREADS, BlockSync>(P, c, row, tiles, reinterpret_cast<unsigned long long *>(smem_raw), s_merge, tid);
+    const bool ok = merge_topk_row<MERGE_THREADS, BlockSync>(P, c, row, tiles, reinterpret_cast<unsigned long long *>(smem_raw), s_merge, tid, cells);
     if (tid == 0 && !ok) { rs->status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
     KERNEL_T1(1);
 }
