@@ -626,10 +626,46 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         c.idx = (int)(~(uint32_t)all[0][0]);
         return c;
     }
-    // crowded bin: descend over the key bits of the elements in range
+    // Crowded bin.  With low-precision logits this is almost always ONE value repeated thousands of times: a pass
+    // over the elements in range finds their smallest and largest key, and if the two agree the boundary value is
+    // known.  Otherwise the key bits of the elements in range are descended, 11 + 11 + 10 at a time.
     uint32_t prefix = 0;
     int pbits = 0;
-    for (int pass = 0; pass < 3; ++pass) {
+    {
+        const uint32_t *keys = x.keys;
+        const int len = x.len, lo_g = x.lo, per = x.per, tid = x.tid;
+        const Cut bs = base;
+        uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
+        for (int i0 = 0; i0 < per; i0 += 4 * EX_THREADS) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * EX_THREADS + tid;
+                if (i < len) {
+                    const uint32_t key = keys[i];
+                    if (member(bs, key, lo_g + i) && in_range(key)) { kmn = min(kmn, key); kmx = max(kmx, key); }
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            kmx = max(kmx, __shfl_xor_sync(0xFFFFFFFFu, kmx, off));
+            kmn = min(kmn, __shfl_xor_sync(0xFFFFFFFFu, kmn, off));
+        }
+        // one 64-bit word per warp carries both: the largest key and the complement of the smallest
+        const unsigned long long both = ((unsigned long long)kmx << 32) | (uint32_t)(~kmn);
+        __syncthreads();
+        if (x.lane == 0) x.sh->wtot[x.warp] = both;
+        __syncthreads();
+        unsigned long long hi = 0, lo32 = 0;
+        for (int w = 0; w < EX_WARPS; ++w) { hi = max(hi, x.sh->wtot[w] >> 32); lo32 = max(lo32, x.sh->wtot[w] & 0xFFFFFFFFull); }
+        unsigned long long v[XV] = {hi, lo32, 0, 0};
+        unsigned long long all[CL][XV];
+        allgather(x, v, all);
+        uint32_t gmax = 0, gninv = 0;
+        for (int r = 0; r < CL; ++r) { gmax = max(gmax, (uint32_t)all[r][0]); gninv = max(gninv, (uint32_t)all[r][1]); }
+        if (gmax == (uint32_t)~gninv) { prefix = gmax; pbits = 32; }          // every element in range has this key
+    }
+    for (int pass = 0; pass < 3 && pbits < 32; ++pass) {
         const int nb = (pass < 2) ? 11 : 10;
         const int shift = 32 - pbits - nb;
         auto dig_k = [=](uint32_t key) -> int {
