@@ -529,8 +529,54 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         float f = fminf(__fmul_rn(__fsub_rn(t, (float)aa), 2048.0f), 2047.0f);
         return 2047 - (int)f;
     };
+    // Smallest and largest key among the members of `base` that satisfy `inr` (one pass, one cluster barrier).
+    // With low-precision logits a crowded bin is almost always ONE value repeated thousands of times; when the two
+    // keys agree, the boundary value is known without further levels, gathering or sorting.
+    auto value_span = [&](auto inr, uint32_t &gmin, uint32_t &gmax) {
+        const uint32_t *keys = x.keys;
+        const int len = x.len, lo_g = x.lo, per = x.per, tid = x.tid;
+        const Cut bs = base;
+        uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
+        for (int i0 = 0; i0 < per; i0 += 4 * EX_THREADS) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * EX_THREADS + tid;
+                if (i < len) {
+                    const uint32_t key = keys[i];
+                    if (member(bs, key, lo_g + i) && inr(key)) { kmn = min(kmn, key); kmx = max(kmx, key); }
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            kmx = max(kmx, __shfl_xor_sync(0xFFFFFFFFu, kmx, off));
+            kmn = min(kmn, __shfl_xor_sync(0xFFFFFFFFu, kmn, off));
+        }
+        // one 64-bit word per warp carries both: the largest key and the complement of the smallest
+        const unsigned long long both = ((unsigned long long)kmx << 32) | (uint32_t)(~kmn);
+        __syncthreads();
+        if (x.lane == 0) x.sh->wtot[x.warp] = both;
+        __syncthreads();
+        unsigned long long hi = 0, lo32 = 0;
+        for (int w = 0; w < EX_WARPS; ++w) { hi = max(hi, x.sh->wtot[w] >> 32); lo32 = max(lo32, x.sh->wtot[w] & 0xFFFFFFFFull); }
+        unsigned long long v[XV] = {hi, lo32, 0, 0};
+        unsigned long long all[CL][XV];
+        allgather(x, v, all);
+        uint32_t gninv = 0;
+        gmax = 0;
+        for (int r = 0; r < CL; ++r) { gmax = max(gmax, (uint32_t)all[r][0]); gninv = max(gninv, (uint32_t)all[r][1]); }
+        gmin = ~gninv;
+    };
+    bool single = false;                                          // the crossing bin holds one repeated value...
+    uint32_t single_key = 0;                                      // ...this one
     int b = -1;
-    if (in_bin > (unsigned long long)GATHER_FAST) b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin, sortbuf);
+    if (in_bin > (unsigned long long)GATHER_FAST) {
+        auto in_a = [=](uint32_t key) -> bool { return !(key < klo_a || key > khi_a) && dig_a(key) == a; };
+        uint32_t gmin, gmax;
+        value_span(in_a, gmin, gmax);
+        if (gmin == gmax) { single = true; single_key = gmax; }
+        else b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin, sortbuf);
+    }
     SONIC_STAMP(5);
     uint32_t klo = klo_a, khi = khi_a;
     if (b >= 0 && a != 0) {                                      // (bin 0 of level 0 is open below: no finer band)
@@ -544,7 +590,7 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         if (dig_a(key) != a) return false;
         return b < 0 || dig_b(key) == b;
     };
-    if (in_bin <= (unsigned long long)GATHER_CAP) {
+    if (!single && in_bin <= (unsigned long long)GATHER_CAP) {
         // every CTA packs its elements of the bin into its own list, then the lists are laid end to end in
         // CTA 0, which sorts them and picks the element that completes the target
         if (x.tid == 0) x.sh->ucount = 0;
@@ -626,45 +672,17 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         c.idx = (int)(~(uint32_t)all[0][0]);
         return c;
     }
-    // Crowded bin.  With low-precision logits this is almost always ONE value repeated thousands of times: a pass
-    // over the elements in range finds their smallest and largest key, and if the two agree the boundary value is
-    // known.  Otherwise the key bits of the elements in range are descended, 11 + 11 + 10 at a time.
+    // Crowded bin (or one repeated value, found above).  Once more the smallest and largest key in range are
+    // compared (the range is narrower after a second level); if they still differ, the key bits of the elements in
+    // range are descended, 11 + 11 + 10 at a time.
     uint32_t prefix = 0;
     int pbits = 0;
-    {
-        const uint32_t *keys = x.keys;
-        const int len = x.len, lo_g = x.lo, per = x.per, tid = x.tid;
-        const Cut bs = base;
-        uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
-        for (int i0 = 0; i0 < per; i0 += 4 * EX_THREADS) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * EX_THREADS + tid;
-                if (i < len) {
-                    const uint32_t key = keys[i];
-                    if (member(bs, key, lo_g + i) && in_range(key)) { kmn = min(kmn, key); kmx = max(kmx, key); }
-                }
-            }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            kmx = max(kmx, __shfl_xor_sync(0xFFFFFFFFu, kmx, off));
-            kmn = min(kmn, __shfl_xor_sync(0xFFFFFFFFu, kmn, off));
-        }
-        // one 64-bit word per warp carries both: the largest key and the complement of the smallest
-        const unsigned long long both = ((unsigned long long)kmx << 32) | (uint32_t)(~kmn);
-        __syncthreads();
-        if (x.lane == 0) x.sh->wtot[x.warp] = both;
-        __syncthreads();
-        unsigned long long hi = 0, lo32 = 0;
-        for (int w = 0; w < EX_WARPS; ++w) { hi = max(hi, x.sh->wtot[w] >> 32); lo32 = max(lo32, x.sh->wtot[w] & 0xFFFFFFFFull); }
-        unsigned long long v[XV] = {hi, lo32, 0, 0};
-        unsigned long long all[CL][XV];
-        allgather(x, v, all);
-        uint32_t gmax = 0, gninv = 0;
-        for (int r = 0; r < CL; ++r) { gmax = max(gmax, (uint32_t)all[r][0]); gninv = max(gninv, (uint32_t)all[r][1]); }
-        if (gmax == (uint32_t)~gninv) { prefix = gmax; pbits = 32; }          // every element in range has this key
+    if (!single) {
+        uint32_t gmin, gmax;
+        value_span(in_range, gmin, gmax);
+        if (gmin == gmax) { single = true; single_key = gmax; }
     }
+    if (single) { prefix = single_key; pbits = 32; }
     for (int pass = 0; pass < 3 && pbits < 32; ++pass) {
         const int nb = (pass < 2) ? 11 : 10;
         const int shift = 32 - pbits - nb;
