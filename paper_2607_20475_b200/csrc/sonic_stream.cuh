@@ -122,7 +122,6 @@ __device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm 
 #define KERNEL_T1(k) do { } while (0)
 #define STREAM_STAMP(i) do { } while (0)
 #endif
-constexpr int BITONIC_SLACK_SIZE = 2048;       // large n: the threshold search may stop anywhere up to this many keys
 constexpr int RANK_SORT_MAX = 512;            // at most this many candidates: sort by rank counting
 constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
 struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
@@ -311,29 +310,103 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     else return false;
     unsigned long long *sorted = buf;
     int Pn2 = Pn;
-    // How many keys the sort below should get at most: what the rank sort takes in one go when n is small, else a
-    // bitonic size with slack above n (a wide window needs few search passes; sorting twice as many keys costs
-    // less than searching a narrow one).
-    const int want_hi = (n + n / 2 + 16 <= RANK_SORT_MAX) ? n + n / 2 + 16 : max(next_pow2(n), BITONIC_SLACK_SIZE);
+    // How many keys the sort below should get at most: what the rank sort takes in one go when n is small, else the
+    // bitonic size that leaves the threshold search a window of at least 16 ranks above n (for the largest n the
+    // next size up would cost more than searching a narrow window).
+    int want_hi = (n + n / 2 + 16 <= RANK_SORT_MAX) ? n + n / 2 + 16 : next_pow2(n + 16);
+    if (want_hi > MERGE_CAP / 2) want_hi = next_pow2(n);
     if (Pn > RANK_SORT_MAX && Pn > want_hi) {
         // more proven candidates than that: search a key threshold that keeps between n and want_hi of them (any
         // such threshold keeps the n best), then sort only those
         unsigned long long lo = 0ull, hi = ~0ull;          // count(>= lo) >= n > count(>= hi)
+        bool tight = false;
         {
-            // start from the range the keys actually span
-            unsigned long long mn = ~0ull, mx = 0ull;
-            for (int i = tid; i < Pn; i += THREADS) { mn = min(mn, buf[i]); mx = max(mx, buf[i]); }
+            // First bracket from the data itself: 31 of the keys, sorted, split the candidates into 32 buckets of
+            // about equal population wherever the keys crowd; one counting pass then places n within one bucket.
+            unsigned long long *sth = reinterpret_cast<unsigned long long *>(sh.scratch);          // [32] ascending, last = sentinel
+            int *hist = reinterpret_cast<int *>(sh.scratch + 32);                                  // [32]
+            unsigned long long *res = reinterpret_cast<unsigned long long *>(sh.scratch + 64);     // lo, hi, count(>= lo), count(>= hi)
+            if (tid < 32) {
+                unsigned long long k = (tid < 31) ? buf[(int)(((long long)(tid + 1) * Pn) >> 5)] : ~0ull;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                mn = min(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
-                mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+                for (int kk = 2; kk <= 32; kk <<= 1) {
+#pragma unroll
+                    for (int jj = kk >> 1; jj > 0; jj >>= 1) {
+                        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, k, jj);
+                        const bool take_min = (((tid & kk) == 0) == ((tid & jj) == 0));
+                        k = ((k < o) == take_min) ? k : o;
+                    }
+                }
+                sth[tid] = k;
+                hist[tid] = 0;
             }
-            unsigned long long *red = reinterpret_cast<unsigned long long *>(sh.scratch);
-            if ((tid & 31) == 0) { red[tid >> 5] = mn; red[THREADS / 32 + (tid >> 5)] = mx; }
             csync();
-            for (int w = 0; w < THREADS / 32; ++w) { mn = min(mn, red[w]); mx = max(mx, red[THREADS / 32 + w]); }
+            for (int i = tid; i < Pn; i += THREADS) {
+                const unsigned long long key = buf[i];
+                int bkt = 0;                                   // number of sampled keys <= key
+#pragma unroll
+                for (int step = 16; step > 0; step >>= 1)
+                    if (bkt + step <= 31 && sth[bkt + step - 1] <= key) bkt += step;
+                atomicAdd(&hist[bkt], 1);
+            }
             csync();
-            lo = mn; hi = mx + 1ull;
+            if (tid < 32) {
+                int suf = hist[tid];                           // -> number of keys in buckets >= tid
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int dn = __shfl_down_sync(0xFFFFFFFFu, suf, o);
+                    if (tid + o < 32) suf += dn;
+                }
+                // keys >= sth[q] are those of buckets q + 1 and above: the largest such q that still keeps n
+                const unsigned int okm = __ballot_sync(0xFFFFFFFFu, tid >= 1 && suf >= n);
+                if (okm) {
+                    const int l = 31 - __clz(okm);
+                    const int cnt = __shfl_sync(0xFFFFFFFFu, suf, l);
+                    const int above = (l < 31) ? __shfl_sync(0xFFFFFFFFu, suf, (l + 1) & 31) : 0;     // keys >= hi
+                    if (tid == 0) { res[0] = sth[l - 1]; res[1] = sth[l]; res[2] = (unsigned long long)cnt; res[3] = (unsigned long long)above; }
+                } else {
+                    const int above = __shfl_sync(0xFFFFFFFFu, suf, 1);
+                    if (tid == 0) { res[0] = 0ull; res[1] = sth[0]; res[2] = (unsigned long long)Pn; res[3] = (unsigned long long)above; }
+                }
+            }
+            csync();
+            lo = res[0]; hi = res[1];
+            const int cnt_lo = (int)res[2], cnt_hi = (int)res[3];
+            tight = cnt_lo <= want_hi;
+            csync();
+            // The bucket [lo, hi) holds the boundary.  If it is small, its keys are collected and ranked, which gives
+            // the threshold that keeps exactly n (no search over key space, whose passes multiply when equal values
+            // differ only in their index bits).
+            const int in_bucket = cnt_lo - cnt_hi, need_here = n - cnt_hi;         // 1 <= need_here <= in_bucket
+            if (!tight && in_bucket <= THREADS) {
+                unsigned long long *list = reinterpret_cast<unsigned long long *>(sh.scratch);         // [THREADS]
+                if (tid == 0) sh.count = 0;
+                csync();
+                for (int i0 = 0; i0 < Pn; i0 += THREADS) {
+                    const int i = i0 + tid;
+                    const unsigned long long key = (i < Pn) ? buf[i] : 0ull;
+                    const bool inb = (i < Pn) && key >= lo && key < hi;
+                    const unsigned int mk = __ballot_sync(0xFFFFFFFFu, inb);
+                    int base = 0;
+                    if ((tid & 31) == 0 && mk) base = atomicAdd(&sh.count, __popc(mk));
+                    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                    if (inb) list[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
+                }
+                csync();
+                unsigned long long found = 0ull;
+                if (tid < in_bucket) {
+                    const unsigned long long key = list[tid];
+                    int rank = 0;
+                    for (int j = 0; j < in_bucket; ++j) rank += (list[j] > key) ? 1 : 0;
+                    if (rank == need_here - 1) found = key;
+                }
+                csync();
+                if (found) list[0] = found;                     // exactly one thread (keys are distinct)
+                csync();
+                lo = list[0];
+                tight = true;                                   // count(>= lo) == n
+                csync();
+            }
         }
         MERGE_STAMP(11);
         // eight-way search: seven interior thresholds per pass.  The warps add their counts into one of two sets
@@ -343,7 +416,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         if (tid < 16) tot2[tid] = 0;
         csync();
         int pass = 0;
-        for (int it = 0; it < 24 && hi - lo > 1ull; ++it, ++pass) {
+        for (int it = 0; it < 24 && !tight && hi - lo > 1ull; ++it, ++pass) {
             const unsigned long long step = (hi - lo) >> 3;
             unsigned long long th[7];
 #pragma unroll

@@ -220,3 +220,29 @@ def test_two_host_threads_share_the_device(sonic, oracle):
     for w, dev in zip(ws, devs):
         assert header_error_word(dev) == 0
         compare_sample(dev.results(), oracle.sample(w), w)
+
+
+@pytest.mark.parametrize("dtype", [wl.DTYPE_F32, wl.DTYPE_BF16])
+def test_threshold_search_with_heavy_ties(sonic, oracle, dtype):
+    # coarse-grained logits (a few dozen distinct values, so equal values differ only in their index) with k from
+    # just above the small-sort limit to the largest the streaming path takes: the merge kernel has to cut the
+    # candidate list inside a run of equal values
+    V = 100000
+    rng = np.random.default_rng(90210)
+    ks = [513, 600, 777, 1000, 1023, 1025, 1500, 2047, 2048, 2049, 3000, 4095, 4096]
+    x = (np.round(rng.standard_normal((len(ks), V)) * 4) / 4).astype(np.float32)
+    x[1::2] = np.round(rng.standard_normal((len(ks[1::2]), V)) * 64).astype(np.float32) / 64
+    w = make_sample(x, [wl.TOP_K | wl.TEMPERATURE] * len(ks), dtype=dtype, temperature=[0.9] * len(ks), top_k=ks,
+                    seed=np.arange(len(ks)) + 31, offset=np.arange(len(ks)))
+    dev = sonic.DeviceSample(w)
+    dev.run()
+    got = dev.results()
+    assert header_error_word(dev) == 0
+    compare_sample(got, oracle.sample(w), w)
+    tw = wl.TopKWorkload(name="ties", B=len(ks), V=V, dtype=dtype, logits=w.logits)
+    rv, ri = oracle.topk(tw.logits_f32(), 4096)
+    for k in (513, 1000, 2049, 4096):
+        dk = sonic.DeviceTopK(tw, k)
+        dk.run()
+        gv, gi = dk.results()
+        compare_topk(gv, gi, rv[:, :k].copy(), ri[:, :k].copy())
