@@ -952,14 +952,16 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     SONIC_STAMP(10);
     const unsigned long long mul = 2ull * a_draw + 1ull;               // u = mul / 2^25
     const unsigned long long T = (__umul64hi(Wq, mul) << 39) | ((Wq * mul) >> 25);
-    unsigned long long qt = 0;
-    int token = ordered_find<unsigned long long>(x, T, wq, stq, qt);
-    double token_prob = (double)qt / (double)Wq;
+    // A position that carries a draft token needs a draw from p only if the draft is rejected AND the residual is
+    // empty; every other row draws from p (below).
+    const bool draft_pos = (P.op == OP_VERIFY && c.l < P.K);
+    bool plain_draw = !draft_pos;
+    int token = -1;
     SONIC_STAMP(11);
 
     uint32_t flags = F_FALLBACK;
     float p_draft = 0.0f;
-    if (P.op == OP_VERIFY && c.l < P.K) {
+    if (draft_pos) {
         const int d = P.draft_tokens[(size_t)c.b * P.K + c.l];
         const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)V;
         unsigned long long v[XV] = {0, 0, 0, 0};
@@ -969,34 +971,51 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         for (int r = 0; r < CL; ++r) if (all[r][0]) qd = all[r][0] - 1ull;
         double Pd = (double)qd / (double)Wq;
         double Q = (d >= 0 && d < V) ? (double)__ldg(q + d) : 0.0;
-        bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);
+        const bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);      // the same value in every CTA
         p_draft = (float)Pd;
-        if (accept) flags |= F_ACCEPT;
         SONIC_STAMP(20);
-        // residual max(0, p - q) over the support, weights in fp64 (p - q cancels, so the weights must be accurate)
-        const double Md = (double)x.Mf;
-        auto wd = [=](int i) -> double {
-            return (i < slen && member(scut, skeys[i], slo + i)) ? exp((double)unkey(skeys[i]) - Md) : 0.0;
-        };
-        OrderedState<double> std_;
-        unsigned long long cdummy;
-        ordered_totals<double>(x, wd, inS, std_, cdummy);
-        const double Wd = std_.total;
-        SONIC_STAMP(21);
-        const double inv_Wd = 1.0 / Wd;                        // p = w * (1 / W): one rounding more than w / W, far below the margins
-        auto rd = [=](int i) -> double {
-            if (!(i < slen && member(scut, skeys[i], slo + i))) return 0.0;
-            double r = exp((double)unkey(skeys[i]) - Md) * inv_Wd - (double)__ldg(q + slo + i);
-            return r > 0.0 ? r : 0.0;
-        };
-        OrderedState<double> str;
-        ordered_totals<double>(x, rd, inS, str, cdummy);
-        if (str.total > 0.0) {
-            double rw;
-            const int t2 = ordered_find<double>(x, cell_to_u(a_draw) * str.total, rd, str, rw);
-            if (t2 >= 0) token = t2;           // (verification rows report p(d), not the probability of this token)
+        if (accept) {
+            // the request moves on with the draft token: neither the residual nor a draw of this position is read
+            flags |= F_ACCEPT;
+            token = d;
+        } else {
+            // residual max(0, p - q) over the support, weights in fp64 (p - q cancels, so the weights must be accurate)
+            const double Md = (double)x.Mf;
+            auto wd = [=](int i) -> double {
+                return (i < slen && member(scut, skeys[i], slo + i)) ? exp((double)unkey(skeys[i]) - Md) : 0.0;
+            };
+            OrderedState<double> std_;
+            unsigned long long cdummy;
+            ordered_totals<double>(x, wd, inS, std_, cdummy);
+            const double Wd = std_.total;
+            SONIC_STAMP(21);
+            const double inv_Wd = 1.0 / Wd;                        // p = w * (1 / W): one rounding more than w / W, far below the margins
+            auto rd = [=](int i) -> double {
+                if (!(i < slen && member(scut, skeys[i], slo + i))) return 0.0;
+                double r = exp((double)unkey(skeys[i]) - Md) * inv_Wd - (double)__ldg(q + slo + i);
+                return r > 0.0 ? r : 0.0;
+            };
+            OrderedState<double> str;
+            ordered_totals<double>(x, rd, inS, str, cdummy);
+            if (str.total > 0.0) {
+                double rw;
+                token = ordered_find<double>(x, cell_to_u(a_draw) * str.total, rd, str, rw);
+            }
+            if (token < 0) {
+                // empty residual (p <= q on the whole support, by rounding): draw from p itself; the ordered totals
+                // of the fixed-point weights were overwritten by the passes above
+                unsigned long long ndummy;
+                ordered_totals<unsigned long long>(x, wq, inS, stq, ndummy);
+                plain_draw = true;
+            }
+            SONIC_STAMP(22);
         }
-        SONIC_STAMP(22);
+    }
+    double token_prob = 0.0;
+    if (plain_draw) {
+        unsigned long long qt = 0;
+        token = ordered_find<unsigned long long>(x, T, wq, stq, qt);
+        token_prob = (double)qt / (double)Wq;
     }
     if (leader) {
         emit_row(P, c, row, token, (float)token_prob, flags, (int)nS, p_draft);

@@ -774,16 +774,18 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
         p_draft = (float)Pd;
         if (accept) flags |= F_ACCEPT;
         csync();
-        // residual max(0, p - q) over the support, in index order
-        for (int j = tid; j < n; j += THREADS) {
-            int idx = (int)(~(uint32_t)(ik[j] >> 32));
-            double r = w[(uint32_t)ik[j]] / W - (double)__ldg(q + idx);
-            cs[j] = r > 0.0 ? r : 0.0;
+        if (!accept) {        // (an accepted position's own token is never read: the request moves on with the draft)
+            // residual max(0, p - q) over the support, in index order
+            for (int j = tid; j < n; j += THREADS) {
+                int idx = (int)(~(uint32_t)(ik[j] >> 32));
+                double r = w[(uint32_t)ik[j]] / W - (double)__ldg(q + idx);
+                cs[j] = r > 0.0 ? r : 0.0;
+            }
+            csync();
+            block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
+            use_residual = cs[n - 1] > 0.0;
+            csync();
         }
-        csync();
-        block_inclusive_scan<THREADS, Sync>(cs, n, sh.scratch, tid);
-        use_residual = cs[n - 1] > 0.0;
-        csync();
     }
     bool picked = false;
     if constexpr (NT == 32) {
