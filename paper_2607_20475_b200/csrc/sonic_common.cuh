@@ -49,6 +49,8 @@ constexpr int CLS_TOPK = 1;                   // streaming path, candidates + me
 constexpr int CLS_EXACT = 2;                  // full-vocabulary exact path only
 
 constexpr int WS_QUEUE = 2;                    // workspace header word: the stream kernel's work counter (zero between calls)
+constexpr int WS_EXACT_TICKET = 3;             // workspace header word: next row ordinal of the exact kernel's first round (zero between calls)
+constexpr int WS_EXACT_LEFT = 6;               // workspace header word: clusters of that round that have run out of rows (zero between calls)
 constexpr int WS_FAILED_ROWS = 1;              // workspace header word: rows of the current call the merge kernel could not prove
 constexpr uint32_t ST_FAILED = 0x1;           // streaming path could not prove the row
 constexpr uint32_t ST_BADID = 0x2;            // a list id was out of range

@@ -55,6 +55,7 @@ struct ExactShared {
     unsigned int red_cnt[HBINS / CL];
     unsigned int ucount;
     int flag;
+    int ticket;                                      // first round: the ordinal of the cluster's next row
 };
 
 struct ExactCtx {
@@ -1043,8 +1044,9 @@ sonic_exact_kernel(const KParams P, const int rounds) {
     // Two rounds, launched separately (`rounds` is the set this launch runs).  Round 0: the rows that belong to
     // this path by class, known from the inputs alone, so this launch runs beside the streaming and merge
     // kernels.  Round 1, a programmatic dependent of the merge kernel: the rows that kernel could not prove.  In
-    // each round every CTA marks the rows of ALL requests and the marked rows are dealt round-robin to the
-    // clusters (all CTAs derive the same list).
+    // each round every CTA marks the rows of ALL requests (all CTAs derive the same list).  Round 0 hands the
+    // marked rows out one at a time from a counter in the workspace header (rows differ a lot in length: a
+    // verification row whose draft is rejected takes two more passes), round 1 deals its few rows round-robin.
     KERNEL_T0(rounds == 2 ? 3 : 2);
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;
@@ -1066,27 +1068,49 @@ sonic_exact_kernel(const KParams P, const int rounds) {
             if (mine) atomicOr(&need[row >> 5], 1u << (row & 31));
         }
         __syncthreads();
-        int ordinal = 0;
-        for (int w = 0; w < nwords; ++w) {
-            uint32_t bits = need[w];
-            while (bits) {
-                const int row = (w << 5) + __ffs(bits) - 1;
-                bits &= bits - 1;
-                if (ordinal % ncl == cid) {
-#ifdef SONIC_TRACE
-                    const unsigned int tr0 = gtimer_lo();
-#endif
-                    exact_row<DT>(P, row, x, sortbuf);
-                    KERNEL_T1(rounds == 2 ? 3 : 2);
-#ifdef SONIC_TRACE
-                    if (threadIdx.x == 0 && x.rank == 0) {
-                        atomicMax(&P.error[56], ((gtimer_lo() - tr0) << 8) | (unsigned int)(row & 255));    // slowest row: ns << 8 | row
-                        atomicMin(&P.error[57], tr0);                                                   // first row start
-                    }
-#endif
+        int nmarked = 0;
+        for (int w = 0; w < nwords; ++w) nmarked += __popc(need[w]);
+        if (nmarked == 0) continue;                                  // (round 0: the counter is never touched)
+        int next_static = cid;
+        for (;;) {
+            int t;
+            if (round == 0) {
+                // the cluster's first thread draws the ordinal and leaves it in every CTA's shared memory
+                if (x.rank == 0 && x.tid == 0) {
+                    const int drawn = (int)atomicAdd(&P.error[WS_EXACT_TICKET], 1u);
+                    for (int r = 0; r < CL; ++r) *cg::this_cluster().map_shared_rank(&x.sh->ticket, r) = drawn;
                 }
-                ++ordinal;
+                cg::this_cluster().sync();
+                t = x.sh->ticket;                 // (the next write comes after the barriers of the row, or never)
+            } else {
+                t = next_static;
+                next_static += ncl;
             }
+            if (t >= nmarked) break;
+            int row = -1, seen = 0;
+            for (int w = 0; w < nwords && row < 0; ++w) {
+                const uint32_t bits = need[w];
+                const int c = __popc(bits);
+                if (t < seen + c) row = (w << 5) + (int)__fns(bits, 0, t - seen + 1);
+                seen += c;
+            }
+#ifdef SONIC_TRACE
+            const unsigned int tr0 = gtimer_lo();
+#endif
+            exact_row<DT>(P, row, x, sortbuf);
+            KERNEL_T1(rounds == 2 ? 3 : 2);
+#ifdef SONIC_TRACE
+            if (threadIdx.x == 0 && x.rank == 0) {
+                atomicMax(&P.error[56], ((gtimer_lo() - tr0) << 8) | (unsigned int)(row & 255));    // slowest row: ns << 8 | row
+                atomicMin(&P.error[57], tr0);                                                   // first row start
+            }
+#endif
+        }
+        // round 0: the last cluster to run out of rows puts both counters back to zero for the next call (every
+        // cluster has drawn its final ordinal by then)
+        if (round == 0 && x.rank == 0 && x.tid == 0) {
+            const unsigned int left = atomicAdd(&P.error[WS_EXACT_LEFT], 1u);
+            if (left == (unsigned int)(ncl - 1)) { P.error[WS_EXACT_TICKET] = 0u; P.error[WS_EXACT_LEFT] = 0u; }
         }
     }
 }

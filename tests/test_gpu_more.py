@@ -246,3 +246,24 @@ def test_threshold_search_with_heavy_ties(sonic, oracle, dtype):
         dk.run()
         gv, gi = dk.results()
         compare_topk(gv, gi, rv[:, :k].copy(), ri[:, :k].copy())
+
+
+def test_exact_row_counters_return_to_zero(sonic, oracle):
+    # more exact-class rows than clusters (top-k off on every stochastic request, K + 1 positions each): the rows are
+    # handed out from a counter in the workspace header, which the last cluster puts back to zero; replays must
+    # therefore give the same answers and leave header words 3 and 6 at zero
+    import torch
+    vw = wl.config4(B=12, K=3, V=20000)
+    vw.sample.top_k[:] = 0
+    vw.sample.mode[:] = (vw.sample.mode & ~np.uint32(wl.TOP_K)).astype(np.uint32)
+    dev = sonic.DeviceVerify(vw)
+    dev.run()
+    first = dev.results()
+    for _ in range(3):
+        dev.run()
+    again = dev.results()
+    for key in first:
+        assert np.array_equal(first[key], again[key]), key
+    hdr = dev.ws[:32].view(torch.int32).cpu().numpy()
+    assert hdr[0] == 0 and hdr[3] == 0 and hdr[6] == 0
+    compare_verify(again, oracle.verify(vw), vw)
