@@ -1087,11 +1087,18 @@ sonic_exact_kernel(const KParams P, const int rounds) {
                 next_static += ncl;
             }
             if (t >= nmarked) break;
+            // ordinal among the marked rows in row order.  Verification, first round: a request's K + 1 positions are
+            // marked together, and the positions that carry a draft (the long rows when the draft is rejected) go first
+            int ord = t;
+            if (round == 0 && P.op == OP_VERIFY && P.K > 0) {
+                const int K1 = P.K + 1, ndraft = (nmarked / K1) * P.K;
+                ord = (t < ndraft) ? (t / P.K) * K1 + (t % P.K) : (t - ndraft) * K1 + P.K;
+            }
             int row = -1, seen = 0;
             for (int w = 0; w < nwords && row < 0; ++w) {
                 const uint32_t bits = need[w];
                 const int c = __popc(bits);
-                if (t < seen + c) row = (w << 5) + (int)__fns(bits, 0, t - seen + 1);
+                if (ord < seen + c) row = (w << 5) + (int)__fns(bits, 0, ord - seen + 1);
                 seen += c;
             }
 #ifdef SONIC_TRACE
