@@ -14,6 +14,8 @@ namespace sonic {
 // Verification epilogue: the K+1 positions of a request were resolved
 // independently (accept flag, correction token); this scans them in order.
 __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
+    KERNEL_T0(5);
+    KERNEL_T1(5);
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const int K = P.K;

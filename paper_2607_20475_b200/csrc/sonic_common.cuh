@@ -136,6 +136,14 @@ __device__ __forceinline__ float unkey(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
 }
 
+// z / tau in IEEE round-to-nearest for a finite tau > 0.  Infinities and NaN (masked or padded entries) pass through
+// unchanged without entering the division's slow path, which the whole warp would otherwise wait for.
+__device__ __forceinline__ float div_tau(float z, float tau) {
+    const bool special = !(fabsf(z) < CUDART_INF_F);
+    const float q = __fdiv_rn(special ? 1.0f : z, tau);
+    return special ? z : q;
+}
+
 // Number of groups G per warp tile whose maxima bound the tile cutoff (a power of two,
 // 2..32, or 64 with half-lane groups).  For position-independent data a warp tile's
 // cutoff exceeds t with probability (1 - exp(-x))^G, x = (elements above t per group),
@@ -144,7 +152,15 @@ __device__ __forceinline__ float unkey(uint32_t k) {
 //     P(G) = V * (G / 1024) * -ln(1 - Nw^(-1/G))
 // elements.  Pick the smallest G whose P(G) clears k with a margin that covers the
 // spread of T, and give up (-1: exact kernel) if that needs more than the merge can sort.
+// The proof itself fails when some warp tile has an element of the row's top k in every
+// group: with x_k = k * (1024 / G) / V elements of the top k per group that happens with
+// probability about Nw * (1 - exp(-x_k))^G per row; G must also keep this below 1e-3 (four
+// groups would otherwise send one row in three hundred to the exact kernel at k = 64,
+// V = 2^18, and such a row costs more than the whole call does without it).
 // G = 0 means "keep every finite element" (vocabularies the merge can sort whole).
+#ifndef SONIC_LG_FAIL_MAX
+#define SONIC_LG_FAIL_MAX -9.97f          // log2(1e-3)
+#endif
 __device__ __forceinline__ int pick_groups(int k, int V) {
     if (V <= MERGE_CAP) return 0;
     const float nw = (float)((V + WARP_TILE - 1) / WARP_TILE);
@@ -155,7 +171,9 @@ __device__ __forceinline__ int pick_groups(int k, int V) {
         // the proven count scatters around the estimate (about 15 % at G = 16, far more at G = 2)
         const float need = (float)k * (G >= 16 ? 1.7f : 1.0f + 6.0f * rsqrtf((float)G)) + 30.0f;
         // above MERGE_CAP the merge first narrows the candidates with a key floor; the tiles' slots bound the rest
-        if (est >= need) return (est <= 0.5f * (float)CAND_CAP) ? G : -1;
+        const float xk = (float)k * ((float)WARP_TILE / (float)G) / (float)V;
+        const float lg_fail = lg + (float)G * __log2f(1.0f - __expf(-xk));        // log2 of the failure probability
+        if (est >= need && lg_fail <= SONIC_LG_FAIL_MAX) return (est <= 0.5f * (float)CAND_CAP) ? G : -1;
     }
     return -1;
 }

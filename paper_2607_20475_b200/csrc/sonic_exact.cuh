@@ -822,7 +822,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         uint32_t kk[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float y = c.temp ? __fdiv_rn(zz[u], c.tau) : zz[u];
+            const float y = c.temp ? div_tau(zz[u], c.tau) : zz[u];
             kk[u] = okey(y);
             kmax = max(kmax, kk[u]);
             const bool fin = (kk[u] > KEY_NEG_INF && l0 + u < x.len);
@@ -1055,7 +1055,7 @@ sonic_exact_kernel(const KParams P, const int rounds) {
         if (!((rounds >> round) & 1)) continue;
         if (round == 1) {
             pdl_wait_primary();
-            if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u) return;     // the merge kernel proved every row: nothing to scan
+            if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u) { KERNEL_T1(3); return; }     // the merge kernel proved every row: nothing to scan
         }
         __syncthreads();
         for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;

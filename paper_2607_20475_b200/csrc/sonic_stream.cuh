@@ -131,6 +131,54 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
 template <int THREADS, typename SH>
 __device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells);
 
+// Ranks of at most THREADS distinct non-zero keys held one per thread in list[0, n): every warp sorts its 32 keys
+// with shuffles and writes them back as a descending run, then a key's rank is its place in its own run plus, for
+// every other run, the number of keys there above it (a binary search in the sorted run; 0 pads the last run).
+// Returns the thread's key after the warp sort (0 = padding) and leaves its rank in `rank`.  Two block barriers.
+template <int THREADS, typename Sync>
+__device__ __forceinline__ unsigned long long rank_keys(unsigned long long *list, int n, int tid, int &rank) {
+    Sync csync;
+    const int lane = tid & 31, warp = tid >> 5;
+    unsigned long long key = (tid < n) ? list[tid] : 0ull;
+#pragma unroll
+    for (int kk = 2; kk <= 32; kk <<= 1) {
+#pragma unroll
+        for (int jj = kk >> 1; jj > 0; jj >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
+            const bool up = ((lane & kk) == 0);            // this block of kk sorts descending
+            const bool first = ((lane & jj) == 0);         // the lower lane of the pair
+            const bool take_max = (up == first);
+            key = ((key > o) == take_max) ? key : o;           // mine if it is on the side this lane takes
+        }
+    }
+    csync();                                               // every thread has read its key from the list
+    list[tid] = key;                                       // sorted runs of 32 (descending), in place
+    csync();
+    const int runs = (n + 31) >> 5;
+    rank = lane;
+    if (key != 0ull) {
+        // four runs at a time: their binary searches are independent chains of shared-memory reads
+        for (int r0 = 0; r0 < runs; r0 += 4) {
+            const unsigned long long *run[4];
+            int lo[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { run[u] = list + min(r0 + u, runs - 1) * 32; lo[u] = 0; }
+#pragma unroll
+            for (int step = 16; step > 0; step >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (run[u][lo[u] + step - 1] > key) lo[u] += step;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (lo[u] < 32 && run[u][lo[u]] > key) ++lo[u];        // covers a run whose 32 keys are all above
+                if (r0 + u < runs && r0 + u != warp) rank += lo[u];     // (lo[u] = number of keys of the run above `key`)
+            }
+        }
+    }
+    return key;
+}
+
 // Row merge for top-k class rows (one CTA per row).  buf is MERGE_CAP 64-bit
 // words of shared memory.  Returns false if the candidates cannot prove the
 // row's answer.
@@ -162,7 +210,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     const unsigned int tkey = sh.tkey;
     const bool complete = (tkey == KEY_NEG_INF);
     const bool strict = c.temp && !complete;            // keys are compared after the temperature division
-    const uint32_t tykey = c.temp ? okey(__fdiv_rn(unkey(tkey), c.tau)) : tkey;
+    const uint32_t tykey = c.temp ? okey(div_tau(unkey(tkey), c.tau)) : tkey;
     const int total = sh.tcnt[tiles];
     // candidates are fetched eight per lane at a time (independent loads), then filtered and packed
     constexpr int GB = 8;
@@ -170,7 +218,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     auto proven_key = [&](unsigned long long cd, int j) -> unsigned long long {
         const uint32_t zk = (uint32_t)(cd >> 32);
         uint32_t yk = zk;
-        if (c.temp) yk = okey(__fdiv_rn(unkey(zk), c.tau));
+        if (c.temp) yk = okey(div_tau(unkey(zk), c.tau));
         const bool keep = (j < total) && (zk >= tkey) && !(strict && yk <= tykey);
         return keep ? (((unsigned long long)yk << 32) | (uint32_t)cd) : 0ull;
     };
@@ -222,7 +270,9 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 }
             }
         }
+        MERGE_STAMP(17);
         csync();
+        MERGE_STAMP(18);
         if (attempt == 1 || sh.count <= MERGE_CAP || sh.count < c.k) break;
         // More proven candidates than the buffer holds (large k): find a key floor that keeps between k and
         // MERGE_CAP of them by an eight-way search over the candidates in global memory, then pack again.
@@ -341,6 +391,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 hist[tid] = 0;
             }
             csync();
+            MERGE_STAMP(13);
             for (int i = tid; i < Pn; i += THREADS) {
                 const unsigned long long key = buf[i];
                 int bkt = 0;                                   // number of sampled keys <= key
@@ -350,6 +401,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 atomicAdd(&hist[bkt], 1);
             }
             csync();
+            MERGE_STAMP(14);
             if (tid < 32) {
                 int suf = hist[tid];                           // -> number of keys in buckets >= tid
 #pragma unroll
@@ -374,6 +426,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             const int cnt_lo = (int)res[2], cnt_hi = (int)res[3];
             tight = cnt_lo <= want_hi;
             csync();
+            MERGE_STAMP(15);
             // The bucket [lo, hi) holds the boundary.  If it is small, its keys are collected and ranked, which gives
             // the threshold that keeps exactly n (no search over key space, whose passes multiply when equal values
             // differ only in their index bits).
@@ -393,15 +446,11 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                     if (inb) list[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
                 }
                 csync();
-                unsigned long long found = 0ull;
-                if (tid < in_bucket) {
-                    const unsigned long long key = list[tid];
-                    int rank = 0;
-                    for (int j = 0; j < in_bucket; ++j) rank += (list[j] > key) ? 1 : 0;
-                    if (rank == need_here - 1) found = key;
-                }
+                MERGE_STAMP(16);
+                int rank;
+                const unsigned long long key = rank_keys<THREADS, Sync>(list, in_bucket, tid, rank);
                 csync();
-                if (found) list[0] = found;                     // exactly one thread (keys are distinct)
+                if (key != 0ull && rank == need_here - 1) list[0] = key;      // exactly one thread (keys are distinct)
                 csync();
                 lo = list[0];
                 tight = true;                                   // count(>= lo) == n
@@ -505,45 +554,9 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         static_assert(RANK_SORT_MAX <= THREADS, "one candidate per thread");
         unsigned long long *dst = buf + MERGE_CAP / 2;
         {
-            const int lane = tid & 31, warp = tid >> 5;
-            unsigned long long key = (tid < Pn) ? buf[tid] : 0ull;
-#pragma unroll
-            for (int kk = 2; kk <= 32; kk <<= 1) {
-#pragma unroll
-                for (int jj = kk >> 1; jj > 0; jj >>= 1) {
-                    const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
-                    const bool up = ((lane & kk) == 0);            // this block of kk sorts descending
-                    const bool first = ((lane & jj) == 0);         // the lower lane of the pair
-                    const bool take_max = (up == first);
-                    key = ((key > o) == take_max) ? key : o;           // mine if it is on the side this lane takes
-                }
-            }
-            csync();                                               // every thread has read its key from buf
-            buf[tid] = key;                                        // sorted runs of 32 (descending), in place
-            csync();
-            const int runs = (Pn + 31) >> 5;
-            if (key != 0ull) {
-                int rank = lane;
-                // four runs at a time: their binary searches are independent chains of shared-memory reads
-                for (int r0 = 0; r0 < runs; r0 += 4) {
-                    const unsigned long long *run[4];
-                    int lo[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) { run[u] = buf + min(r0 + u, runs - 1) * 32; lo[u] = 0; }
-#pragma unroll
-                    for (int step = 16; step > 0; step >>= 1) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (run[u][lo[u] + step - 1] > key) lo[u] += step;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (lo[u] < 32 && run[u][lo[u]] > key) ++lo[u];        // covers a run whose 32 keys are all above
-                        if (r0 + u < runs && r0 + u != warp) rank += lo[u];     // (lo[u] = number of keys of the run above `key`)
-                    }
-                }
-                dst[rank] = key;
-            }
+            int rank;
+            const unsigned long long key = rank_keys<THREADS, Sync>(buf, Pn, tid, rank);
+            if (key != 0ull) dst[rank] = key;
         }
         csync();
         for (int i = tid; i < n; i += THREADS) buf[i] = dst[i];       // only the n best are used from here on
@@ -1241,7 +1254,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             }
             if (c.div_all) {
 #pragma unroll
-                for (int q = 0; q < EPL; ++q) e[q] = __fdiv_rn(e[q], c.tau);
+                for (int q = 0; q < EPL; ++q) e[q] = div_tau(e[q], c.tau);
             }
 
             // per-vector maxima, half maxima, lane maximum
@@ -1338,7 +1351,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                             float v;
                             if (DT == 0 || patched) v = ptile[li];
                             else v = __uint_as_float((uint32_t)reinterpret_cast<const unsigned short *>(stage)[li] << 16);
-                            if (c.div_all) v = __fdiv_rn(v, c.tau);
+                            if (c.div_all) v = div_tau(v, c.tau);
                             *dst++ = ((unsigned long long)okey(v) << 32) | (uint32_t)(~(uint32_t)(tile_base + li));
                         }
                     }
