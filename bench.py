@@ -117,7 +117,8 @@ class ClockSampler:
 
 
 def oracle_time(name: str, w, budget_s: float):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns (us per call, description)."""
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns (us per call, description,
+    rows of the sample, rows of the sample whose decision margin is below 1e-6)."""
     from oracle import oracle
     import copy as _copy
     if name == "c4":
@@ -128,21 +129,23 @@ def oracle_time(name: str, w, budget_s: float):
         sub.sample = _slice_sample(vw.sample, nreq, rows=nreq * (vw.K + 1))
         sub.draft_tokens = vw.draft_tokens[:nreq]
         sub.draft_probs = vw.draft_probs[:nreq]
-        t0 = time.perf_counter(); oracle.verify(sub); dt = time.perf_counter() - t0
+        t0 = time.perf_counter(); ref = oracle.verify(sub); dt = time.perf_counter() - t0
+        near = int((ref["margin"] < 1e-6).sum())
         reps = max(1, int(budget_s / max(dt, 1e-3)) - 1)
         t0 = time.perf_counter()
         for _ in range(reps):
             oracle.verify(sub)
         dt = (time.perf_counter() - t0) / reps if reps else dt
-        return dt * vw.B / nreq * 1e6, f"{nreq} of {vw.B} requests x {reps} repetitions, scaled to the full batch"
+        return dt * vw.B / nreq * 1e6, f"{nreq} of {vw.B} requests x {reps} repetitions, scaled to the full batch", nreq, near
     n = max(1, min(w.B, 8))
     sub = _slice_sample(w, n, rows=n)
     t0 = time.perf_counter(); oracle.sample(sub); dt = time.perf_counter() - t0
     per_row = dt / n
     n2 = int(max(1, min(w.B, budget_s / max(per_row, 1e-6))))
     sub = _slice_sample(w, n2, rows=n2)
-    t0 = time.perf_counter(); oracle.sample(sub); dt = time.perf_counter() - t0
-    return dt * w.B / n2 * 1e6, f"first {n2} of {w.B} rows, one pass, scaled to the full batch"
+    t0 = time.perf_counter(); ref = oracle.sample(sub); dt = time.perf_counter() - t0
+    near = int((ref["margin"] < 1e-6).sum())
+    return dt * w.B / n2 * 1e6, f"first {n2} of {w.B} rows, one pass, scaled to the full batch", n2, near
 
 
 def _slice_sample(w, n, rows):
@@ -185,7 +188,7 @@ def run_reference(args, rank, world):
     times = []
     desc = ""
     for i in range(args.warmup + args.steps):
-        us, desc = oracle_time(name, w, budget_s=max(0.05, budget))
+        us, desc, _, _ = oracle_time(name, w, budget_s=max(0.05, budget))
         if i >= args.warmup:
             times.append(us)
     us = float(np.mean(times))
@@ -241,6 +244,46 @@ def time_graph_steps(graph_full, per_graph, graph_rem, rem, steps):
     end.record()
     torch.cuda.synchronize()
     return start.elapsed_time(end) / 1000.0
+
+
+def time_graph_min(graph, per_graph, reps=12):
+    """Fastest replay of the graph, per call (CUDA events around every replay)."""
+    import torch
+    best = float("inf")
+    for _ in range(reps):
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        graph.replay()
+        e.record()
+        torch.cuda.synchronize()
+        best = min(best, s.elapsed_time(e) * 1000.0 / per_graph)
+    return best
+
+
+def time_warm_l2(dev, calls=8, reps=12):
+    """The same call back to back on ONE input copy (the input stays in L2 when it fits): us per call."""
+    import torch
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(calls):
+            dev.run()
+    for _ in range(3):
+        g.replay()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s.record()
+    for _ in range(reps):
+        g.replay()
+    e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e) * 1000.0 / (calls * reps)
+
+
+def fallback_rows(name, devs):
+    """Rows (requests for c4) per call, over the input copies, that report the exact kernel (diagnostic flag bit 2)."""
+    per_copy = [int((d.results()["flags"][:(d.vw.B if name == "c4" else None)] & 4).astype(bool).sum()) for d in devs]
+    return {"mean_per_call": float(np.mean(per_copy)), "max_per_call": int(max(per_copy)),
+            "unit": "requests" if name == "c4" else "rows"}
 
 
 def measure_floor(calls=64, reps=20):
@@ -369,6 +412,9 @@ def run_sonic(args, rank, world, local_rank):
     e2e_us, h2d, d2h = e2e_measure(name, devs[0], steps=min(steps, 40))
     e2e_us = max_over_ranks(e2e_us, world, "cuda")
     floor_us = measure_floor() if rank == 0 else None
+    min_us = time_graph_min(g_full, per_graph) if rank == 0 else None
+    warm_us = time_warm_l2(devs[0]) if rank == 0 else None
+    fb = fallback_rows(name, devs) if rank == 0 else None
 
     extra = {}
     if rank == 0 and args.also:
@@ -381,7 +427,7 @@ def run_sonic(args, rank, world, local_rank):
         rows = B * (w0.K + 1) if name == "c4" else B
         achieved = bytes_call / (us_call * 1e-6) / 1e9
         launches_per_call = 5 if name == "c4" else 4     # exact (first round), stream, merge, exact (second round) [, verify combine]
-        cpu_us, cpu_desc = oracle_time(name, w0, budget_s=15.0)
+        cpu_us, cpu_desc, cpu_rows, cpu_near = oracle_time(name, w0, budget_s=15.0)
         out = {
             "metric": METRIC, "value": job_value(us_call, world), "unit": "us", "n_gpus": world, "steps": steps,
             "warmup": max(3, args.warmup), "ms_per_step": us_call / 1000.0, "higher_is_better": False,
@@ -398,6 +444,12 @@ def run_sonic(args, rank, world, local_rank):
             "e2e": {"value": job_value(e2e_us, world), "unit": "us", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": launches_per_call * steps,
             "empty_graph_node_us": floor_us,
+            "us_per_call_min": min_us,
+            "warm_l2": {"us_per_call": warm_us, "input_fits_l2": bool(bytes_call < L2_BYTES),
+                        "note": "one input copy replayed back to back"},
+            "rows": {"per_call": rows, "exact_kernel": fb,
+                     "near_margin": {"count": cpu_near, "of": cpu_rows, "unit": fb["unit"],
+                                     "note": "decision margin below 1e-6 in the oracle, on the cpu_baseline sample"}},
             "clocks": clocks,
             "also": extra,
         }
@@ -466,6 +518,44 @@ def quick_measure(name, binding, reps=30):
             "copies": copies}
 
 
+def run_sweep():
+    """Throughput sweep beyond the five configurations (one GPU): fused sample call on B rows of vocabulary V, all
+    rows low-entropy ("spiked") or high-entropy ("flat"), fp32 and bf16.  Prints one JSON line with the table."""
+    import torch
+    from paper_2607_20475_b200 import binding
+    binding.lib()
+    peak, which = peaks()
+    table = []
+    for dtype, dname in ((wl.DTYPE_F32, "f32"), (wl.DTYPE_BF16, "bf16")):
+        for V in (1 << 15, 1 << 16, 1 << 17, 1 << 18):
+            for B in (1, 8, 64, 256):
+                for regime in ("spiked", "flat"):
+                    nbytes = B * V * (2 if dtype == wl.DTYPE_BF16 else 4)
+                    copies = int(min(16, max(2, np.ceil(2.0 * L2_BYTES / nbytes))))
+                    ws = binding.new_workspace(B)
+                    devs = [binding.DeviceSample(wl.sweep_case(B, V, dtype, regime, c), ws=ws) for c in range(copies)]
+                    g = capture(devs, copies)
+                    for _ in range(3):
+                        g.replay()
+                    reps = int(max(5, min(200, 2000 // copies)))
+                    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda.synchronize()
+                    s.record()
+                    for _ in range(reps):
+                        g.replay()
+                    e.record()
+                    torch.cuda.synchronize()
+                    us = s.elapsed_time(e) * 1000.0 / (reps * copies)
+                    fb = int(np.mean([int((d.results()["flags"] & 4).astype(bool).sum()) for d in devs]))
+                    table.append({"dtype": dname, "V": V, "B": B, "rows": regime, "us_per_call": round(us, 2),
+                                  "gbs": round(nbytes / us / 1e3, 1), "frac": round(nbytes / us / 1e3 / peak, 4),
+                                  "cold": bool(copies * nbytes > 2 * L2_BYTES), "exact_rows": fb})
+                    del devs, g, ws
+                    torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "fused sample call, temperature 0.8, top-k 50, top-p 0.9", "peak_gbs": peak,
+                      "peak_source": which, "table": table}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -473,6 +563,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="sonic", choices=["sonic", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4"])
+    ap.add_argument("--sweep", action="store_true", help="time the V x B x entropy x dtype sweep instead (one GPU)")
     ap.add_argument("--also", default="c1,c3,c4,c5k1,c5k64", help="other configurations to time briefly (comma separated, '' for none)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -484,6 +575,10 @@ def main():
         if args.warmup == 16:
             args.warmup = 1
         run_reference(args, rank, world)
+        return
+    if args.sweep:
+        if rank == 0:
+            run_sweep()
         return
     run_sonic(args, rank, world, local_rank)
 

@@ -389,3 +389,21 @@ def config5(regime: str, B: int = 256, V: int = 262144, dtype: int = DTYPE_F32,
             raise ValueError(regime)
     logits = f32_to_bf16_bits(x) if dtype == DTYPE_BF16 else x
     return TopKWorkload(name=f"c5-{regime}", B=B, V=V, dtype=dtype, logits=logits, meta={"regime": regime})
+
+
+def sweep_case(B: int, V: int, dtype: int, regime: str, copy: int = 0) -> SampleWorkload:
+    """Throughput-sweep input beyond the five configurations: B stochastic rows, all "spiked" (N(0,1) with +10 on
+    three ids: low entropy) or all "flat" (N(0,1): high entropy), temperature 0.8, top-k 50, top-p 0.9."""
+    rng = np.random.default_rng(BASE_SEED + 700 + 31 * copy + (0 if regime == "spiked" else 1))
+    x = rng.standard_normal((B, V)).astype(np.float32)
+    if regime == "spiked":
+        for r in range(B):
+            x[r, rng.choice(V, size=3, replace=False)] += np.float32(10.0)
+    d = _defaults(B)
+    d["mode"][:] = TEMPERATURE | TOP_K | TOP_P
+    d["temperature"][:] = 0.8
+    d["top_k"][:] = 50
+    d["top_p"][:] = 0.9
+    d["offset"][:] = np.arange(B)
+    lg = f32_to_bf16_bits(x) if dtype == DTYPE_BF16 else x
+    return SampleWorkload(name=f"sweep-{regime}", B=B, V=V, dtype=dtype, logits=lg, **d)
