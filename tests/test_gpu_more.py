@@ -267,3 +267,26 @@ def test_exact_row_counters_return_to_zero(sonic, oracle):
     hdr = dev.ws[:32].view(torch.int32).cpu().numpy()
     assert hdr[0] == 0 and hdr[3] == 0 and hdr[6] == 0
     compare_verify(again, oracle.verify(vw), vw)
+
+
+def test_thousands_of_exact_rows_share_the_row_counter(sonic, oracle):
+    # far more exact-class rows than clusters, short rows with a ragged slice per CTA: every cluster draws rows from
+    # the counter until it runs dry; rows of the streaming classes are interleaved
+    B, V = 3000, 300
+    rng = np.random.default_rng(5150)
+    x = (rng.standard_normal((B, V)) * 2).astype(np.float32)
+    kinds = np.arange(B) % 4
+    mode = np.select([kinds == 0, kinds == 1, kinds == 2], [wl.TOP_P | wl.TEMPERATURE, wl.MIN_P, wl.GREEDY],
+                     wl.TOP_K | wl.TOP_P).astype(np.uint32)
+    w = make_sample(x, mode, temperature=np.where(kinds == 0, 0.8, 1.0), top_k=np.where(kinds == 3, 7, 0),
+                    top_p=np.where(kinds % 3 == 0, 0.85, 1.0), min_p=np.where(kinds == 1, 0.03, 0.0),
+                    seed=np.arange(B) + 17, offset=np.arange(B) * 3)
+    dev = sonic.DeviceSample(w)
+    for _ in range(2):
+        dev.run()
+    got = dev.results()
+    import torch
+    hdr = dev.ws[:32].view(torch.int32).cpu().numpy()
+    assert hdr[0] == 0 and hdr[2] == 0 and hdr[3] == 0 and hdr[6] == 0
+    compare_sample(got, oracle.sample(w), w)
+    assert all(got["flags"][r] & 4 for r in range(B) if kinds[r] in (0, 1))
