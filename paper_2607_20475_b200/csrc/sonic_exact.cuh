@@ -1070,14 +1070,18 @@ sonic_exact_kernel(const KParams P, const int rounds) {
         __syncthreads();
         int nmarked = 0;
         for (int w = 0; w < nwords; ++w) nmarked += __popc(need[w]);
-        if (nmarked == 0) continue;                                  // (round 0: the counter is never touched)
+        if (nmarked == 0) continue;                                  // (round 0: the counters are never touched)
         int next_static = cid;
+        bool first = true;
         for (;;) {
             int t;
-            if (round == 0) {
+            if (round == 0 && first) {
+                t = cid;                          // a cluster's first row needs no draw: the counter hands out ncl, ncl + 1, ...
+                first = false;
+            } else if (round == 0) {
                 // the cluster's first thread draws the ordinal and leaves it in every CTA's shared memory
                 if (x.rank == 0 && x.tid == 0) {
-                    const int drawn = (int)atomicAdd(&P.error[WS_EXACT_TICKET], 1u);
+                    const int drawn = ncl + (int)atomicAdd(&P.error[WS_EXACT_TICKET], 1u);
                     for (int r = 0; r < CL; ++r) *cg::this_cluster().map_shared_rank(&x.sh->ticket, r) = drawn;
                 }
                 cg::this_cluster().sync();
