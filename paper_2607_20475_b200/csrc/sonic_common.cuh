@@ -122,6 +122,7 @@ struct RowCfg {
     float alpha, beta, gamma;
     int hist_len, bias_len;
     int cls, G;            // path class; groups per warp tile (0 = keep every finite element)
+    bool tile_min;         // the tile cutoff is the smallest warp cutoff (tile mode of pick_groups), not the largest
     bool bad;              // parameter outside its domain
     bool temp;             // temperature bit
     bool div_all;          // streaming path divides every element (greedy with temperature)
@@ -144,36 +145,50 @@ __device__ __forceinline__ float div_tau(float z, float tau) {
     return special ? z : q;
 }
 
-// Number of groups G per warp tile whose maxima bound the tile cutoff (a power of two,
-// 2..32, or 64 with half-lane groups).  For position-independent data a warp tile's
-// cutoff exceeds t with probability (1 - exp(-x))^G, x = (elements above t per group),
-// so the row-wide cutoff T (the largest over Nw warp tiles) sits where
-// 1 - exp(-x) = Nw^(-1/G), and the proven prefix holds about
-//     P(G) = V * (G / 1024) * -ln(1 - Nw^(-1/G))
-// elements.  Pick the smallest G whose P(G) clears k with a margin that covers the
-// spread of T, and give up (-1: exact kernel) if that needs more than the merge can sort.
-// The proof itself fails when some warp tile has an element of the row's top k in every
-// group: with x_k = k * (1024 / G) / V elements of the top k per group that happens with
-// probability about Nw * (1 - exp(-x_k))^G per row; G must also keep this below 1e-3 (four
-// groups would otherwise send one row in three hundred to the exact kernel at k = 64,
-// V = 2^18, and such a row costs more than the whole call does without it).
-// G = 0 means "keep every finite element" (vocabularies the merge can sort whole).
+// Which group maxima bound a tile's cutoff.  A warp tile (1024 elements) is cut into G groups (a power of
+// two, 1..32, or 64 with half-lane groups) and the cutoff of a block is the smallest of its group maxima, so
+// at least one element per group lies at or above it.  Two kinds of block:
+//   warp mode: block = warp tile (G groups); the tile cutoff is the LARGEST of its eight warp cutoffs;
+//   tile mode: block = the whole 8192-element tile (8 G groups); the tile cutoff is the SMALLEST warp cutoff.
+// The row-wide cutoff T is the largest tile cutoff either way.  For position-independent data a block of m
+// groups has a cutoff above t with probability (1 - exp(-x))^m, x = (elements above t per group), so with
+// Nb blocks in the row T sits where 1 - exp(-x) = Nb^(-1/m), and the proven prefix holds about
+//     P = V * (G / 1024) * -ln(1 - Nb^(-1/m))
+// elements.  A minimum over more groups concentrates better: at V = 2^18 tile mode with G = 1 proves
+// 245 elements on average (94 at worst in 400 simulated rows) where warp mode with G = 4 proves 265 (63 at
+// worst) and G = 8 proves 1330.  The candidates are tried in the order of their P (warp 2, tile 1, warp 4,
+// tile 2, warp 8, tile 4, warp 16, tile 8, warp 32, warp 64) and the first one is taken whose P clears k
+// with a margin that covers the spread of T and whose proof fails rarely enough: the proof fails when
+// some block has an element of the row's top k in every group; with x_k = k * (1024 / G) / V elements
+// of the top k per group that happens with probability about Nb * (1 - exp(-x_k))^m per row, which must
+// stay below 1e-3 (warp mode with four groups would send one row in three hundred to the exact kernel at
+// k = 64, V = 2^18, and such a row costs more than the whole call does without it).  Tile mode stops at
+// G = 8: a minimum over more groups now and then falls so low that the tile overflows its candidate slot.
+// Returns G, plus PICK_TILE_MODE in tile mode; 0 means "keep every finite element" (vocabularies the
+// merge can sort whole); -1 hands the row to the exact kernel.
 #ifndef SONIC_LG_FAIL_MAX
 #define SONIC_LG_FAIL_MAX -9.97f          // log2(1e-3)
 #endif
+constexpr int PICK_TILE_MODE = 0x100;
 __device__ __forceinline__ int pick_groups(int k, int V) {
     if (V <= MERGE_CAP) return 0;
-    const float nw = (float)((V + WARP_TILE - 1) / WARP_TILE);
-    const float lg = __log2f(nw);
-    for (int G = 2; G <= 64; G <<= 1) {
-        const float r = exp2f(-lg / (float)G);                       // Nw^(-1/G)
+    const float lg_nw = __log2f((float)((V + WARP_TILE - 1) / WARP_TILE));
+    const float lg_nt = __log2f((float)((V + CTA_TILE - 1) / CTA_TILE));
+    for (int step = 0; step < 11; ++step) {
+        const bool tile = (step & 1) != 0;
+        if (tile && step > 7) continue;
+        const int G = tile ? (1 << (step >> 1)) : (2 << (step >> 1));
+        const float m = (float)(tile ? G * (CTA_TILE / WARP_TILE) : G);              // groups per block
+        const float lg = tile ? lg_nt : lg_nw;                                      // log2 of the blocks per row
+        const float r = exp2f(-lg / m);                                             // Nb^(-1/m)
         const float est = (float)V * ((float)G / (float)WARP_TILE) * -__logf(1.0f - r);
-        // the proven count scatters around the estimate (about 15 % at G = 16, far more at G = 2)
-        const float need = (float)k * (G >= 16 ? 1.7f : 1.0f + 6.0f * rsqrtf((float)G)) + 30.0f;
+        // the proven count scatters around the estimate (about 15 % at 16 groups, far more at 2)
+        const float need = (float)k * (m >= 16.0f ? 1.7f : 1.0f + 6.0f * rsqrtf(m)) + 30.0f;
         // above MERGE_CAP the merge first narrows the candidates with a key floor; the tiles' slots bound the rest
         const float xk = (float)k * ((float)WARP_TILE / (float)G) / (float)V;
-        const float lg_fail = lg + (float)G * __log2f(1.0f - __expf(-xk));        // log2 of the failure probability
-        if (est >= need && lg_fail <= SONIC_LG_FAIL_MAX) return (est <= 0.5f * (float)CAND_CAP) ? G : -1;
+        const float lg_fail = lg + m * __log2f(1.0f - __expf(-xk));                 // log2 of the failure probability
+        if (est >= need && lg_fail <= SONIC_LG_FAIL_MAX)
+            return (est <= 0.5f * (float)CAND_CAP) ? (G | (tile ? PICK_TILE_MODE : 0)) : -1;
     }
     return -1;
 }
@@ -245,6 +260,7 @@ __device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const C
     if (c.k < 0) c.k = 0;
     c.div_all = false;
     c.G = 0;
+    c.tile_min = false;
     if (greedy || (P.op == OP_TOPK && c.k == 1)) {
         c.cls = CLS_GREEDY;
         c.div_all = c.temp;
@@ -258,7 +274,7 @@ __device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const C
                 G = pick_groups(c.k, P.V);
                 if (memo_k) { *memo_k = c.k; *memo_G = G; }
             }
-            if (G >= 0) { c.cls = CLS_TOPK; c.G = G; }
+            if (G >= 0) { c.cls = CLS_TOPK; c.G = G & (PICK_TILE_MODE - 1); c.tile_min = (G & PICK_TILE_MODE) != 0; }
         }
     }
     return c;

@@ -1296,26 +1296,44 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                     rec->best = b;
                 }
             } else {
-                // tile cutoff: minimum over G groups of the group maximum, then the largest over the eight warp tiles
+                // warp cutoff: minimum over G groups of the group maximum.  Tile cutoff: the largest of the eight
+                // warp cutoffs (warp mode) or the smallest (tile mode: a minimum over all 8 G groups of the tile).
+                // In tile mode a group without a finite element (masked, or past the row's end) does not take
+                // part: it would drag the cutoff to -inf and the tile would emit everything it has.
                 float g;
                 const int G = c.G;
+                const bool tmin = c.tile_min;
                 if (G == 0) {
                     g = -CUDART_INF_F;
                 } else {
                     const int L = (G >= 32) ? 1 : (32 / G);           // lanes per group
-                    g = (G == 64) ? fminf(h0, h1) : lm;
+                    if (G == 64) {
+                        const float a0 = (tmin && h0 == -CUDART_INF_F) ? CUDART_INF_F : h0;
+                        const float a1 = (tmin && h1 == -CUDART_INF_F) ? CUDART_INF_F : h1;
+                        g = fminf(a0, a1);
+                    } else {
+                        g = lm;
+                    }
 #pragma unroll
                     for (int off = 1; off < 32; off <<= 1) {
+                        if (tmin && off == L && g == -CUDART_INF_F) g = CUDART_INF_F;
                         const float o = __shfl_xor_sync(0xFFFFFFFFu, g, off);
                         g = (off < L) ? fmaxf(g, o) : fminf(g, o);
                     }
+                    if (tmin && g == -CUDART_INF_F) g = CUDART_INF_F;   // G = 1: the warp tile is the group
                 }
                 if (lane == 0) sh.tw[s][warp] = g;
                 if (tid == 0) sh.ncand[s] = 0;
                 csync();
                 float t = sh.tw[s][0];
+                if (tmin) {
 #pragma unroll
-                for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, sh.tw[s][w]);
+                    for (int w = 1; w < STREAM_WARPS; ++w) t = fminf(t, sh.tw[s][w]);
+                    if (t == CUDART_INF_F) t = -CUDART_INF_F;          // no finite element in the tile: nothing to emit
+                } else {
+#pragma unroll
+                    for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, sh.tw[s][w]);
+                }
                 // every finite element >= t goes to the tile's candidate slot; a warp reserves its share of the
                 // slot with one shared-memory atomic and adds it to the tile record (no second barrier).
                 // Most warps hold no candidate at all and leave after one vote.  The others mark their
