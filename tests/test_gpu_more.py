@@ -290,3 +290,37 @@ def test_thousands_of_exact_rows_share_the_row_counter(sonic, oracle):
     assert hdr[0] == 0 and hdr[2] == 0 and hdr[3] == 0 and hdr[6] == 0
     compare_sample(got, oracle.sample(w), w)
     assert all(got["flags"][r] & 4 for r in range(B) if kinds[r] in (0, 1))
+
+
+@pytest.mark.parametrize("V", [262144, 200003, 128256, 100001])
+def test_tile_cutoffs_ragged_rows_sparse_masks_and_empty_tiles(sonic, oracle, V):
+    # small and medium k take their tile cutoff as the smallest group maximum of the whole tile; groups with no
+    # finite element (past a ragged row's end, masked out, a whole tile masked) must not drag it down: every row
+    # has to agree with the oracle, and the dense rows and small k be finished by the streaming path (no exact-kernel flag)
+    rng = np.random.default_rng(V)
+    ks = [8, 20, 50, 64, 200, 256, 600, 1000]
+    B = 2 * len(ks)
+    x = rng.standard_normal((B, V)).astype(np.float32)
+    allowed = np.ones((B, V), dtype=bool)
+    for r in range(len(ks), B):
+        allowed[r] = rng.random(V) < 0.05                 # sparse: many groups of 128 hold no allowed id
+        allowed[r, 3 * 8192:5 * 8192] = False             # two whole tiles masked
+        allowed[r, 8192 + 1024:8192 + 4096] = False       # three warp tiles of one tile masked
+    mode = [wl.TOP_K | wl.TEMPERATURE] * len(ks) + [wl.TOP_K | wl.TEMPERATURE | wl.GRAMMAR] * len(ks)
+    w = make_sample(x, mode, temperature=rng.uniform(0.6, 1.4, B), top_k=ks + ks, bitmask=pack_bits(allowed),
+                    seed=np.arange(B) + 5, offset=np.arange(B))
+    dev = sonic.DeviceSample(w)
+    dev.run()
+    got = dev.results()
+    compare_sample(got, oracle.sample(w), w)
+    # (the sparse rows with a large k may legitimately miss their proof: few finite elements per group)
+    must_stream = [r for r in range(B) if r < len(ks) or w.top_k[r] <= 64]
+    assert not (got["flags"][must_stream] & 4).any(), np.nonzero(got["flags"] & 4)[0]
+    assert header_error_word(dev) == 0
+    tw = wl.TopKWorkload(name="ragged", B=B, V=V, dtype=wl.DTYPE_F32, logits=np.where(allowed, x, -np.inf).astype(np.float32))
+    rv, ri = oracle.topk(tw.logits_f32(), 1024)
+    for k in (8, 64, 256, 1024):
+        d = sonic.DeviceTopK(tw, k)
+        d.run()
+        gv, gi = d.results()
+        compare_topk(gv, gi, rv[:, :k].copy(), ri[:, :k].copy())
