@@ -148,18 +148,55 @@ def oracle_time(name: str, w, budget_s: float):
     return dt * w.B / n2 * 1e6, f"first {n2} of {w.B} rows, one pass, scaled to the full batch", n2, near
 
 
-def _slice_sample(w, n, rows):
+def _slice_sample(w, n, rows, start=0):
     import copy as _copy
     s = _copy.copy(w)
     s.B = n
-    s.logits = w.logits[:rows]
+    s.logits = w.logits[start:start + rows]
     for f in ("mode", "temperature", "top_k", "top_p", "min_p", "rep_penalty", "freq_penalty", "pres_penalty", "seed",
               "offset", "hist_ids", "hist_counts", "hist_len", "bias_ids", "bias_vals", "bias_len"):
         v = getattr(w, f)
-        setattr(s, f, None if v is None else v[:n])
+        setattr(s, f, None if v is None else v[start:start + n])
     if w.bitmask is not None:
-        s.bitmask = w.bitmask[:rows]
+        s.bitmask = w.bitmask[start:start + rows]
     return s
+
+
+def oracle_time_all_cores(name: str, w, budget_s: float):
+    """The same oracle with the rows of a singular-mode workload dealt to one thread per host core (the C routine
+    releases the interpreter lock).  Returns (us per call scaled to the full batch, threads, description) or None."""
+    if name == "c4":
+        return None
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import oracle
+    cores = len(os.sched_getaffinity(0))
+    t0 = time.perf_counter(); oracle.sample(_slice_sample(w, 1, 1)); per_row = time.perf_counter() - t0
+    per_thread = int(max(1, min(w.B // max(1, cores), budget_s / max(per_row, 1e-6))))
+    threads = min(cores, max(1, w.B // per_thread))
+    parts = [_slice_sample(w, per_thread, per_thread, start=i * per_thread) for i in range(threads)]
+    with ThreadPoolExecutor(threads) as pool:
+        t0 = time.perf_counter()
+        list(pool.map(oracle.sample, parts))
+        dt = time.perf_counter() - t0
+    rows = per_thread * threads
+    return dt * w.B / rows * 1e6, threads, f"{rows} of {w.B} rows, {per_thread} per thread, one pass, scaled to the full batch"
+
+
+def read_probe(gib: float = 1.0, reps: int = 10):
+    """Read-only streaming rate of this GPU (the path is read-dominated, the measured peak is a copy): a library
+    reduction over a buffer far larger than L2, best of `reps`, CUDA events.  A second denominator, not the target."""
+    import torch
+    x = torch.empty(int(gib * (1 << 30)) // 4, dtype=torch.float32, device="cuda").fill_(1.0)
+    best = float("inf")
+    for _ in range(3):
+        x.sum()
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); x.sum(); e1.record(); torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) * 1e-3)
+    gbs = x.numel() * 4 / best / 1e9
+    del x
+    return {"gbs": gbs, "bytes": int(gib * (1 << 30)), "how": "torch.sum over fp32, best of %d, CUDA events" % reps}
 
 
 def config_dict(name, w0, copies=None, bytes_call=None, world=1):
@@ -428,6 +465,8 @@ def run_sonic(args, rank, world, local_rank):
         achieved = bytes_call / (us_call * 1e-6) / 1e9
         launches_per_call = 5 if name == "c4" else 4     # exact (first round), stream, merge, exact (second round) [, verify combine]
         cpu_us, cpu_desc, cpu_rows, cpu_near = oracle_time(name, w0, budget_s=15.0)
+        cpu_all = oracle_time_all_cores(name, w0, budget_s=6.0)
+        probe = read_probe()
         out = {
             "metric": METRIC, "value": job_value(us_call, world), "unit": "us", "n_gpus": world, "steps": steps,
             "warmup": max(3, args.warmup), "ms_per_step": us_call / 1000.0, "higher_is_better": False,
@@ -441,6 +480,9 @@ def run_sonic(args, rank, world, local_rank):
                                  "launches of the exact kernel, overlapped through a forked side stream and programmatic "
                                  "dependent launch); the per-kernel split is in profiles/"},
             "cpu_baseline": {"value": cpu_us, "unit": "us", "cores": 1, "kind": "oracle", "sample": cpu_desc},
+            "cpu_baseline_all_cores": None if cpu_all is None else
+                {"value": cpu_all[0], "unit": "us", "cores": cpu_all[1], "kind": "oracle", "sample": cpu_all[2]},
+            "read_probe": dict(probe, frac_of_read_probe=achieved / probe["gbs"]),
             "e2e": {"value": job_value(e2e_us, world), "unit": "us", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": launches_per_call * steps,
             "empty_graph_node_us": floor_us,
