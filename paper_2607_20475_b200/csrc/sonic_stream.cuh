@@ -189,23 +189,28 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     MERGE_STAMP(0);
     const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
     const TileRec *rec = P.tiles + (size_t)row * MAX_TILES;
-    // tile records: one thread per tile, then a serial prefix over at most 32 entries
-    if (tid == 0) { sh.count = 0; sh.tkey = 0; sh.found = 0; }
-    csync();
-    if (tid < tiles) {
-        const unsigned int cnt = __ldcg(&rec[tid].cnt);
-        P.tiles[(size_t)row * MAX_TILES + tid].cnt = 0u;           // the streaming kernel accumulates into it
-        sh.tcnt[tid + 1] = (int)cnt;
-        atomicMax(&sh.tkey, __ldcg(&rec[tid].tkey));
-        if (cnt > (unsigned int)cap_t) sh.found = 1;     // a tile overflowed its slot
+    // tile records: the first warp takes one tile per lane; prefix of the counts and the largest cutoff by shuffles
+    static_assert(MAX_TILES <= 32, "one tile record per lane of the first warp");
+    if (tid < 32) {
+        unsigned int cnt = 0u, tk = 0u;
+        if (tid < tiles) {
+            cnt = __ldcg(&rec[tid].cnt);
+            tk = __ldcg(&rec[tid].tkey);
+            P.tiles[(size_t)row * MAX_TILES + tid].cnt = 0u;       // the streaming kernel accumulates into it
+        }
+        const bool over = __any_sync(0xFFFFFFFFu, cnt > (unsigned int)cap_t);     // a tile overflowed its slot
+        int incl = (int)cnt;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (tid >= off) incl += o;
+        }
+        tk = __reduce_max_sync(0xFFFFFFFFu, tk);
+        sh.tcnt[tid + 1] = incl;                                   // lanes past the last tile repeat the total
+        if (tid == 0) { sh.tcnt[0] = 0; sh.count = 0; sh.tkey = tk; sh.found = over ? 1 : 0; }
     }
     csync();
     if (sh.found) return false;
-    if (tid == 0) {
-        sh.tcnt[0] = 0;
-        for (int t = 0; t < tiles; ++t) sh.tcnt[t + 1] += sh.tcnt[t];
-    }
-    csync();
     MERGE_STAMP(1);
     const unsigned int tkey = sh.tkey;
     const bool complete = (tkey == KEY_NEG_INF);
@@ -235,6 +240,24 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
             const unsigned long long *pa = P.cand + (size_t)row * CAND_CAP + (size_t)ta * cap_t;
             const unsigned long long *pb = P.cand + (size_t)row * CAND_CAP + (size_t)tb * cap_t;
+            if (max(na, nb) <= 32) {
+                // small k: a tile brings a dozen candidates, one per lane
+                const unsigned long long ca = (lane < na) ? __ldcg(pa + lane) : 0ull;
+                const unsigned long long cb = (lane < nb) ? __ldcg(pb + lane) : 0ull;
+                const unsigned long long oa = proven_key(ca, lane < na ? 0 : total);
+                const unsigned long long ob = proven_key(cb, lane < nb ? 0 : total);
+                kmax = max(kmax, max(oa, ob));
+                const unsigned int ma = __ballot_sync(0xFFFFFFFFu, oa >= floor_key);
+                const unsigned int mb = __ballot_sync(0xFFFFFFFFu, ob >= floor_key);
+                const int nk = __popc(ma) + __popc(mb);
+                int base = 0;
+                if (lane == 0 && nk) base = atomicAdd(&sh.count, nk);
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                const unsigned int below = (1u << lane) - 1u;
+                if (oa >= floor_key) { const int pos = base + __popc(ma & below); if (pos < MERGE_CAP) buf[pos] = oa; }
+                if (ob >= floor_key) { const int pos = base + __popc(ma) + __popc(mb & below); if (pos < MERGE_CAP) buf[pos] = ob; }
+                continue;
+            }
             for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
                 unsigned long long cd[GB];
 #pragma unroll
