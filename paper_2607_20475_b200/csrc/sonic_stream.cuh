@@ -1364,17 +1364,32 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 // candidate is neither masked nor past the row's end, so the tile holds its value).
                 const float t2 = fmaxf(t, -CUDART_MAX_NORMAL_F);           // e >= t2  <=>  e >= t and e is not -inf
                 if (__any_sync(0xFFFFFFFFu, lm >= t2)) {
+                    // a half of the lanes' elements without a candidate anywhere in the warp is skipped by one vote
                     unsigned int cm = 0;
+                    if (__any_sync(0xFFFFFFFFu, h0 >= t2)) {
 #pragma unroll
-                    for (int q = 0; q < EPL; ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
-                    const int cnt = __popc(cm);
-                    int incl = cnt;
-#pragma unroll
-                    for (int off = 1; off < 32; off <<= 1) {
-                        const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                        if (lane >= off) incl += o;
+                        for (int q = 0; q < EPL / 2; ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
                     }
-                    const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                    if (__any_sync(0xFFFFFFFFu, h1 >= t2)) {
+#pragma unroll
+                        for (int q = EPL / 2; q < EPL; ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
+                    }
+                    const int cnt = __popc(cm);
+                    int incl, total;
+                    if (!__any_sync(0xFFFFFFFFu, cnt > 1)) {
+                        // the usual case, at most one candidate per lane: positions from one vote
+                        const unsigned int has = __ballot_sync(0xFFFFFFFFu, cnt > 0);
+                        incl = __popc(has & (0xFFFFFFFFu >> (31 - lane)));
+                        total = __popc(has);
+                    } else {
+                        incl = cnt;
+#pragma unroll
+                        for (int off = 1; off < 32; off <<= 1) {
+                            const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                            if (lane >= off) incl += o;
+                        }
+                        total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                    }
                     unsigned int base = 0;
                     if (lane == 0) {
                         base = atomicAdd(&sh.ncand[s], (unsigned int)total);
