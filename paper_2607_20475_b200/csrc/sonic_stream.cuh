@@ -909,6 +909,18 @@ __device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row,
     if (tid < 32) epilogue_tail<32, WarpSync>(P, c, row, n, buf, sh, tid, cells);
 }
 
+// Smallest of a warp tile's group maxima, L lanes per group (g: the lane's own maximum, or with half-lane groups
+// the smaller of its two).  In tile mode a group without a finite element counts as +inf, i.e. takes no part.
+template <int L>
+__device__ __forceinline__ float warp_cutoff(float g, bool tile_mode) {
+#pragma unroll
+    for (int off = 1; off < L; off <<= 1) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, off));
+    if (tile_mode && g == -CUDART_INF_F) g = CUDART_INF_F;
+#pragma unroll
+    for (int off = L; off < 32; off <<= 1) g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, off));
+    return g;
+}
+
 // What the producer hands to the consumers with each stage.
 struct StageMeta {
     RowCfg cfg;
@@ -929,7 +941,7 @@ struct StreamShared {
     unsigned long long empty[NSTAGE];          // consumers -> producer: stage free (one arrival per consumer warp)
     StageMeta meta[NSTAGE];
     // per-stage scratch of the consumer warps (a fast warp may already be on the next tile, in the other stage)
-    float tw[NSTAGE][STREAM_WARPS];
+    alignas(16) float tw[NSTAGE][STREAM_WARPS];
     unsigned int ncand[NSTAGE];
     unsigned long long best[NSTAGE][STREAM_WARPS];
     // hit lists: one buffer more than stages, so that the producer fills the next tile's while both stages are busy
@@ -1326,36 +1338,33 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 float g;
                 const int G = c.G;
                 const bool tmin = c.tile_min;
-                if (G == 0) {
-                    g = -CUDART_INF_F;
-                } else {
-                    const int L = (G >= 32) ? 1 : (32 / G);           // lanes per group
-                    if (G == 64) {
-                        const float a0 = (tmin && h0 == -CUDART_INF_F) ? CUDART_INF_F : h0;
-                        const float a1 = (tmin && h1 == -CUDART_INF_F) ? CUDART_INF_F : h1;
-                        g = fminf(a0, a1);
-                    } else {
-                        g = lm;
-                    }
-#pragma unroll
-                    for (int off = 1; off < 32; off <<= 1) {
-                        if (tmin && off == L && g == -CUDART_INF_F) g = CUDART_INF_F;
-                        const float o = __shfl_xor_sync(0xFFFFFFFFu, g, off);
-                        g = (off < L) ? fmaxf(g, o) : fminf(g, o);
-                    }
-                    if (tmin && g == -CUDART_INF_F) g = CUDART_INF_F;   // G = 1: the warp tile is the group
+                switch (G) {                                   // (one straight-line butterfly per group count)
+                case 0: g = -CUDART_INF_F; break;
+                case 1: g = warp_cutoff<32>(lm, tmin); break;
+                case 2: g = warp_cutoff<16>(lm, tmin); break;
+                case 4: g = warp_cutoff<8>(lm, tmin); break;
+                case 8: g = warp_cutoff<4>(lm, tmin); break;
+                case 16: g = warp_cutoff<2>(lm, tmin); break;
+                case 32: g = warp_cutoff<1>(lm, tmin); break;
+                default: {                                     // 64: half-lane groups
+                    const float a0 = (tmin && h0 == -CUDART_INF_F) ? CUDART_INF_F : h0;
+                    const float a1 = (tmin && h1 == -CUDART_INF_F) ? CUDART_INF_F : h1;
+                    g = warp_cutoff<1>(fminf(a0, a1), false);
+                    break;
+                }
                 }
                 if (lane == 0) sh.tw[s][warp] = g;
                 if (tid == 0) sh.ncand[s] = 0;
                 csync();
-                float t = sh.tw[s][0];
+                static_assert(STREAM_WARPS == 8, "the eight warp cutoffs are read as two 128-bit words");
+                const float4 ta = *reinterpret_cast<const float4 *>(&sh.tw[s][0]);
+                const float4 tb = *reinterpret_cast<const float4 *>(&sh.tw[s][4]);
+                float t;
                 if (tmin) {
-#pragma unroll
-                    for (int w = 1; w < STREAM_WARPS; ++w) t = fminf(t, sh.tw[s][w]);
+                    t = fminf(fminf(fminf(ta.x, ta.y), fminf(ta.z, ta.w)), fminf(fminf(tb.x, tb.y), fminf(tb.z, tb.w)));
                     if (t == CUDART_INF_F) t = -CUDART_INF_F;          // no finite element in the tile: nothing to emit
                 } else {
-#pragma unroll
-                    for (int w = 1; w < STREAM_WARPS; ++w) t = fmaxf(t, sh.tw[s][w]);
+                    t = fmaxf(fmaxf(fmaxf(ta.x, ta.y), fmaxf(ta.z, ta.w)), fmaxf(fmaxf(tb.x, tb.y), fmaxf(tb.z, tb.w)));
                 }
                 // every finite element >= t goes to the tile's candidate slot; a warp reserves its share of the
                 // slot with one shared-memory atomic and adds it to the tile record (no second barrier).
