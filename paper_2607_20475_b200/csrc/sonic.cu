@@ -186,8 +186,8 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     // a CTA's first request to the work queue: seven eighths of an even share, at least one item
     int chunk = (int)((7ll * nitems) / (8ll * grid1));
     chunk = chunk < 1 ? 1 : chunk;
-    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems, chunk);
-    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems, chunk);
+    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems, chunk, (int)(CAND_CAP / (unsigned)tiles));
+    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems, chunk, (int)(CAND_CAP / (unsigned)tiles));
     e = cudaGetLastError();
     if (e != cudaSuccess) return unwind(fail_cuda(e, "stream kernel launch"));
     // the merge kernel and the exact kernel's second round are programmatic dependents: they may begin launching

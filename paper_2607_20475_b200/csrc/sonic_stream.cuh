@@ -951,7 +951,7 @@ struct StreamShared {
 
 template <int DT>
 __global__ void __launch_bounds__(STREAM_CTA_THREADS, 3)
-sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const int chunk) {
+sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const int chunk, const int cap_t) {     // cap_t: candidate slots per tile, CAND_CAP / tiles
     constexpr int VEC = VecTraits<DT>::VEC, NV = VecTraits<DT>::NV, NSTAGE = VecTraits<DT>::NSTAGE;
     constexpr int ELT = VecTraits<DT>::ELT;
     constexpr int STAGE_BYTES = CTA_TILE * ELT;
@@ -1314,9 +1314,16 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 if (wm > -CUDART_INF_F) {
                     int best = 0x7FFFFFFF;
                     if (lm == wm) {
+                        // slots ascend: the last write is the lowest; a match in the lane's first half wins
+                        if (h0 == wm) {
 #pragma unroll
-                        for (int q = EPL - 1; q >= 0; --q)
-                            if (e[q] == wm) best = slot_index<DT>(wbase, lane, q);   // slots ascend: the last write is the lowest
+                            for (int q = EPL / 2 - 1; q >= 0; --q)
+                                if (e[q] == wm) best = slot_index<DT>(wbase, lane, q);
+                        } else {
+#pragma unroll
+                            for (int q = EPL - 1; q >= EPL / 2; --q)
+                                if (e[q] == wm) best = slot_index<DT>(wbase, lane, q);
+                        }
                     }
 #pragma unroll
                     for (int off = 16; off > 0; off >>= 1) best = min(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
@@ -1405,7 +1412,6 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                         atomicAdd(&rec->cnt, (unsigned int)total);      // zero before the call; the merge kernel clears it
                     }
                     base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                    const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
                     if ((int)base + total <= cap_t) {
                         unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + (size_t)tile * cap_t + base + (incl - cnt);
                         const int lbase = warp * WARP_TILE + lane * VEC;
