@@ -30,7 +30,7 @@ from paper_2607_20475_b200 import workloads as wl  # noqa: E402
 
 METRIC = "us_per_fused_sample_call"
 # DRAM bytes (read + write) of one call's kernels from the ncu captures summarised under profiles/ (per workload)
-NCU_TRAFFIC = {"c2": 17.84e6, "c3": 143.4e6}
+NCU_TRAFFIC = {"c2": 17.93e6, "c3": 143.1e6}
 L2_BYTES = 126 * 1024 * 1024
 
 

@@ -1301,9 +1301,14 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 for (int q = 1; q < VEC; ++q) m = fmaxf(m, e[j * VEC + q]);
                 mv[j] = m;
             }
-            float h0 = mv[0], h1 = mv[NV / 2];
+            float qm[4];                               // maxima of the lane's four quarters (8 elements each)
 #pragma unroll
-            for (int j = 1; j < NV / 2; ++j) { h0 = fmaxf(h0, mv[j]); h1 = fmaxf(h1, mv[NV / 2 + j]); }
+            for (int i = 0; i < 4; ++i) {
+                qm[i] = mv[i * (NV / 4)];
+#pragma unroll
+                for (int j = 1; j < NV / 4; ++j) qm[i] = fmaxf(qm[i], mv[i * (NV / 4) + j]);
+            }
+            const float h0 = fmaxf(qm[0], qm[1]), h1 = fmaxf(qm[2], qm[3]);
             const float lm = fmaxf(h0, h1);
 
             if (c.cls == CLS_GREEDY) {
@@ -1380,15 +1385,14 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 // candidate is neither masked nor past the row's end, so the tile holds its value).
                 const float t2 = fmaxf(t, -CUDART_MAX_NORMAL_F);           // e >= t2  <=>  e >= t and e is not -inf
                 if (__any_sync(0xFFFFFFFFu, lm >= t2)) {
-                    // a half of the lanes' elements without a candidate anywhere in the warp is skipped by one vote
+                    // a quarter of the lanes' elements without a candidate anywhere in the warp is skipped by one vote
                     unsigned int cm = 0;
-                    if (__any_sync(0xFFFFFFFFu, h0 >= t2)) {
 #pragma unroll
-                        for (int q = 0; q < EPL / 2; ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
-                    }
-                    if (__any_sync(0xFFFFFFFFu, h1 >= t2)) {
+                    for (int i = 0; i < 4; ++i) {
+                        if (__any_sync(0xFFFFFFFFu, qm[i] >= t2)) {
 #pragma unroll
-                        for (int q = EPL / 2; q < EPL; ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
+                            for (int q = i * (EPL / 4); q < (i + 1) * (EPL / 4); ++q) cm |= (e[q] >= t2) ? (1u << q) : 0u;
+                        }
                     }
                     const int cnt = __popc(cm);
                     int incl, total;
