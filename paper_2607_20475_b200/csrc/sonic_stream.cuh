@@ -1319,15 +1319,16 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 if (wm > -CUDART_INF_F) {
                     int best = 0x7FFFFFFF;
                     if (lm == wm) {
-                        // slots ascend: the last write is the lowest; a match in the lane's first half wins
-                        if (h0 == wm) {
+                        // slots ascend: the last write is the lowest; only the first quarter that holds the maximum is searched
+                        bool found = false;
 #pragma unroll
-                            for (int q = EPL / 2 - 1; q >= 0; --q)
-                                if (e[q] == wm) best = slot_index<DT>(wbase, lane, q);
-                        } else {
+                        for (int i = 0; i < 4; ++i) {
+                            if (!found && qm[i] == wm) {
+                                found = true;
 #pragma unroll
-                            for (int q = EPL - 1; q >= EPL / 2; --q)
-                                if (e[q] == wm) best = slot_index<DT>(wbase, lane, q);
+                                for (int q = (i + 1) * (EPL / 4) - 1; q >= i * (EPL / 4); --q)
+                                    if (e[q] == wm) best = slot_index<DT>(wbase, lane, q);
+                            }
                         }
                     }
 #pragma unroll
