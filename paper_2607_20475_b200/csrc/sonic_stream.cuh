@@ -1,26 +1,30 @@
-// Streaming kernel: reads every logit of the rows it owns exactly once, applies
-// the logit-processing prologue, and reduces each 8192-element tile either to
-// an argmax (greedy rows) or to the complete set of elements above a tile
-// cutoff (top-k rows), written to the tile's own slot of the workspace without
-// atomics.  The CTA that finishes a row's last tile merges the row (global
-// top-k, truncation epilogue, token selection) while the others keep streaming.
-// The two halves correspond to the paper's Algorithms "Stage 1: Tile-Local
-// Reduction Kernel" and "Stage 2: Cross-Tile Merge and Selection Kernel"; the
-// selection itself is ours.
+// Streaming kernel and merge kernel.
 //
-// Structure: persistent CTAs (two per SM), each a producer warp plus eight
-// consumer warps.  The producer walks the CTA's tiles, resolves each tile's row
-// configuration and issues one bulk-TMA copy (cp.async.bulk, completion on an
-// mbarrier) of the tile's logits into a ring of shared-memory stages, several
-// tiles ahead of the consumers, so HBM requests stay in flight while the
-// consumers compute.  Every mbarrier wait is bounded: on expiry the kernel
-// records an error in the workspace header and returns.
+// The streaming kernel reads every logit of the rows of the streaming classes
+// exactly once, applies the logit-processing prologue, and reduces each
+// 8192-element tile either to an argmax (greedy rows) or to the complete set of
+// elements at or above a tile cutoff (top-k rows), written to the tile's own
+// slot of the workspace.  The merge kernel, a programmatic dependent launch with
+// one CTA per row, combines a row's tile records and finishes the row (global
+// top-k, truncation epilogue, token selection) or flags it for the exact kernel.
+// The two correspond to the paper's Algorithms "Stage 1: Tile-Local Reduction
+// Kernel" and "Stage 2: Cross-Tile Merge and Selection Kernel"; the selection
+// itself is ours.
 //
-// Exactness: a tile's cutoff t is the minimum of G group maxima, so at least G
-// of its elements are >= t, and the tile emits EVERY finite element >= t.  With
-// T the largest cutoff of the row, the emitted elements >= T are exactly the
-// row's elements >= T.  If there are at least k of them the row's top-k is
-// their top-k; otherwise the row is handed to the exact kernel.
+// Structure of the streaming kernel: persistent CTAs (three per SM), each a
+// producer warp plus eight consumer warps.  The producer takes tiles from a work
+// queue, resolves each tile's row configuration and issues one bulk-TMA copy
+// (cp.async.bulk, completion on an mbarrier) of the tile's logits into a ring of
+// two shared-memory stages, one tile ahead of the consumers, so HBM requests
+// stay in flight while the consumers compute.  Every mbarrier wait is bounded:
+// on expiry the kernel records an error in the workspace header and returns.
+//
+// Exactness: a tile's cutoff t is a minimum of group maxima (of the G groups of
+// one warp tile, or of all 8 G groups of the tile), so the tile holds elements
+// >= t, and it emits EVERY finite element >= t.  With T the largest cutoff of
+// the row, the emitted elements >= T are exactly the row's elements >= T.  If
+// there are at least k of them the row's top-k is their top-k; otherwise the row
+// is handed to the exact kernel.
 #pragma once
 #include "sonic_common.cuh"
 
