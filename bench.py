@@ -249,11 +249,11 @@ def build_device_copies(name, copies, binding):
         w = make_workload(name, copy=c)
         if name == "c4":
             if ws is None:
-                ws = binding.new_workspace(w.B * (w.K + 1))
+                ws = binding.new_workspace(w.B * (w.K + 1), w.V)
             devs.append(binding.DeviceVerify(w, ws=ws))
         else:
             if ws is None:
-                ws = binding.new_workspace(w.B)
+                ws = binding.new_workspace(w.B, w.V)
             devs.append(binding.DeviceSample(w, ws=ws))
     torch.cuda.synchronize()
     return devs
@@ -404,7 +404,7 @@ def job_value(us_per_call_per_replica: float, world: int) -> float:
 def run_sonic(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
-    from paper_2607_20475_b200 import binding
+    from paper_2607_20475_b200 import harness as binding
 
     torch.cuda.set_device(local_rank)
     if world > 1:
@@ -508,7 +508,7 @@ def quick_topk(k, binding, reps=10):
     """sonic_topk on the c5 'normal' regime (B=256, V=262144, fp32), two input copies (> 2x L2), one k."""
     import torch
     tw = wl.config5("normal")
-    ws = binding.new_workspace(tw.B)
+    ws = binding.new_workspace(tw.B, tw.V)
     devs = [binding.DeviceTopK(tw, k, ws=ws), binding.DeviceTopK(tw, k, ws=ws)]
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
@@ -564,7 +564,7 @@ def run_sweep():
     """Throughput sweep beyond the five configurations (one GPU): fused sample call on B rows of vocabulary V, all
     rows low-entropy ("spiked") or high-entropy ("flat"), fp32 and bf16.  Prints one JSON line with the table."""
     import torch
-    from paper_2607_20475_b200 import binding
+    from paper_2607_20475_b200 import harness as binding
     binding.lib()
     peak, which = peaks()
     table = []
@@ -574,7 +574,7 @@ def run_sweep():
                 for regime in ("spiked", "flat"):
                     nbytes = B * V * (2 if dtype == wl.DTYPE_BF16 else 4)
                     copies = int(min(16, max(2, np.ceil(2.0 * L2_BYTES / nbytes))))
-                    ws = binding.new_workspace(B)
+                    ws = binding.new_workspace(B, V)
                     devs = [binding.DeviceSample(wl.sweep_case(B, V, dtype, regime, c), ws=ws) for c in range(copies)]
                     g = capture(devs, copies)
                     for _ in range(3):

@@ -17,6 +17,9 @@
  *   0x040 greedy selection      0x080 top-k                0x100 top-p
  *   0x200 min-p                 0x400 top-k log-probabilities (reserved, ignored)
  * A parameter array may be NULL when no request sets the bit that reads it.
+ * Parameter domains: tau > 0 finite; k >= 0; p, theta in (0, 1]; rep_penalty alpha > 0 finite (the paper states
+ * alpha >= 1), freq_penalty and pres_penalty finite (the paper states >= 0), bias values finite; a set bit with a
+ * parameter outside its domain gives SONIC_FLAG_BADPARAM for that row.
  */
 #ifndef SONIC_H
 #define SONIC_H
@@ -43,25 +46,29 @@ extern "C" {
 /* per-row output flags */
 #define SONIC_FLAG_NO_TOKEN  0x1u   /* no finite processed logit: token is -1 */
 #define SONIC_FLAG_BADPARAM  0x2u   /* tau <= 0, p or theta outside (0,1], k < 0, list id out of range: token is -1 */
-#define SONIC_FLAG_FALLBACK  0x4u   /* diagnostic: the row took the exact full-vocabulary path */
+#define SONIC_FLAG_FALLBACK  0x4u   /* diagnostic: the row was finished by the cluster kernel (top-k beyond the streaming
+                                       path, or a row no other path could finish) */
+#define SONIC_FLAG_DENSE     0x8u   /* diagnostic: top-k off, the row was finished by the full-vocabulary histogram passes */
+#define SONIC_FLAG_TIMEOUT   0x10u  /* a bounded wait inside the streaming kernel expired: token is -1 (see sonic_workspace_init) */
 
-/* Bytes of workspace needed for calls over at most max_rows logit rows
- * (B for sonic_sample / sonic_topk, B*(K+1) for sonic_verify).  Pure host arithmetic. */
-size_t sonic_workspace_bytes(int max_rows);
+/* Bytes of workspace that serve every call over at most max_rows logit rows (B for sonic_sample / sonic_topk,
+ * B*(K+1) for sonic_verify) of at most max_vocab entries each.  max_topk is accepted for forward compatibility
+ * (the candidate slots are sized for every supported k) and ignored.  Pure host arithmetic.
+ * Per row: 1.3 KB of control words, 8 bytes per candidate slot (min(32768, V rounded up to 8192)), and for the rows
+ * with top-k off 4 bytes per vocabulary entry (the processed logits as ordered keys) plus 48 KB of histogram and list. */
+size_t sonic_workspace_bytes(int max_rows, int max_vocab, int max_topk);
 
-/* Zeroes the control words of a workspace once after allocation (a memset
- * enqueued on `stream`, a cudaStream_t passed as void*).  The kernels restore
- * those words at the end of every call, so replays need no re-initialisation.
- * Two calls that use the same workspace must not overlap on the device.
+/* Zeroes the workspace header (the first 512 bytes: work counters and the sticky error word) once after allocation
+ * (a memset enqueued on `stream`, a cudaStream_t passed as void*).  The kernels put the counters back to zero
+ * at the end of every call and initialise every other word they read themselves, so replays need no
+ * re-initialisation and one workspace serves calls of different shapes.  Two calls that use the same workspace
+ * must not overlap on the device.
  *
- * Streams: sonic_sample, sonic_verify and sonic_topk enqueue one of their kernels
- * (the exact path's rows that are known from the inputs alone) on an internal
- * per-device stream that is forked from `stream` at the start of the call and
- * joined to it before the call returns, so that kernel runs beside the others;
- * work enqueued on `stream` after the call is ordered after all of it, and under
- * stream capture the internal stream is captured with `stream`.  The internal
- * stream and two events are created by the first such call on a device (before
- * any capture is begun); calls on one device enqueue one at a time (a host mutex). */
+ * Error word: 32-bit word 0 of the workspace is sticky; bit 0 is set when a bounded wait of the streaming kernel
+ * (a tile copy that never completed) ran out.  Every row of such a call, and of later calls on that workspace,
+ * reports SONIC_FLAG_TIMEOUT with token -1 until the workspace is initialised again with this function.
+ *
+ * Streams: every kernel of a call is enqueued on the caller's `stream`; the library creates no stream or event. */
 int sonic_workspace_init(void *workspace, size_t bytes, void *stream);
 
 /*
@@ -154,8 +161,8 @@ int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, 
  * per call; larger B is rejected with SONIC_ESHAPE.  The scratch memory is a fixed array
  * of about 2.1 MB inside the library image (SONIC_STATIC_MAX_ROWS rows of candidate
  * slots and control words); every GPU that loads the library holds it until the process
- * exits.  The function calls no cudaMalloc, cudaFree or other allocating routine, and it
- * creates no stream or event: all of its kernels go to `stream`.
+ * exits.  The function calls no cudaMalloc, cudaFree or other allocating routine, and
+ * all of its kernels go to `stream`.
  *
  * The first call on each device resolves the array's device address and configures the
  * kernels; that first call should come before any stream capture is begun.  All calls on a device share

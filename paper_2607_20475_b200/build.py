@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsonic.so")
 SOURCES = ["sonic.cu"]
-HEADERS = ["sonic_common.cuh", "sonic_stream.cuh", "sonic_exact.cuh", "../../include/sonic.h"]
+HEADERS = ["sonic_common.cuh", "sonic_dense.cuh", "sonic_stream.cuh", "sonic_exact.cuh", "../../include/sonic.h"]
 
 
 def _stale() -> bool:

@@ -6,6 +6,7 @@
 
 #include "../../include/sonic.h"
 #include "sonic_common.cuh"
+#include "sonic_dense.cuh"
 #include "sonic_stream.cuh"
 #include "sonic_exact.cuh"
 
@@ -43,12 +44,14 @@ __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
     P.out_flags[b] = flags;
 }
 
-constexpr size_t WS_HEADER = 256;
+constexpr size_t WS_HEADER = WS_HEADER_WORDS * 4;
 constexpr int MERGE_SMEM = MERGE_CAP * 8;
 constexpr int STREAM_SMEM_F32 = VecTraits<0>::NSTAGE * CTA_TILE * 4 + (int)sizeof(StreamShared<0>);
 constexpr int STREAM_SMEM_BF16 = VecTraits<1>::NSTAGE * CTA_TILE * 2 + CTA_TILE * 4 + (int)sizeof(StreamShared<1>);
-constexpr int SECOND_ROUND_CLUSTERS = 4;      // clusters of the exact kernel's second launch (rows the merge kernel failed)
+constexpr int EXACT_CLUSTERS = 4;             // clusters of the cluster kernel (its rows are rare)
 constexpr int EXACT_SMEM = SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8 + 8192;
+static_assert(MERGE_SMEM >= DENSE_DYN_SMEM, "stage 2 of the histogram path runs in the merge kernel's shared memory");
+static_assert(DENSE_THREADS == MERGE_THREADS, "stage 2 of the histogram path runs in the merge kernel's CTAs");
 
 static thread_local char g_err[256] = "";
 
@@ -61,23 +64,46 @@ static int fail_cuda(cudaError_t e, const char *what) {
     return SONIC_ECUDA;
 }
 
-constexpr size_t WS_ROW_CTRL = sizeof(RowState) + sizeof(PosResult) + sizeof(TileRec) * MAX_TILES;
-constexpr size_t WS_ROW = WS_ROW_CTRL + (size_t)CAND_CAP * 8;
+// Workspace layout.  Only the header (WS_HEADER bytes at offset 0) is shared by all calls and must be zero between
+// them; everything behind it is laid out for the shape of the call at hand (rows, V, whether the histogram path
+// can be taken) and initialised by the call's own kernels, so one workspace serves calls of any shape that fits.
+struct Layout {
+    size_t rs, pr, tiles, cand, drow, dtile, dlist, rlist, hist, members, ykeys, total;
+    unsigned int cand_stride;
+    int ytiles;
+};
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+static Layout layout_for(long long rows, int V, bool dense) {
+    Layout L;
+    memset(&L, 0, sizeof(L));
+    const int tiles = (V + CTA_TILE - 1) / CTA_TILE;
+    const size_t slots = (size_t)tiles * CTA_TILE < CAND_CAP ? (size_t)tiles * CTA_TILE : CAND_CAP;
+    L.cand_stride = (unsigned int)slots;
+    L.ytiles = tiles;
+    size_t off = WS_HEADER;
+    L.rs = off;    off = align256(off + (size_t)rows * sizeof(RowState));
+    L.pr = off;    off = align256(off + (size_t)rows * sizeof(PosResult));
+    L.tiles = off; off = align256(off + (size_t)rows * sizeof(TileRec) * MAX_TILES);
+    L.cand = off;  off = align256(off + (size_t)rows * slots * 8);
+    if (dense) {
+        L.drow = off;    off = align256(off + (size_t)rows * sizeof(DenseRow));
+        L.dtile = off;   off = align256(off + (size_t)rows * sizeof(DenseTile) * MAX_TILES);
+        L.dlist = off;   off = align256(off + (size_t)rows * 4);
+        L.rlist = off;   off = align256(off + (size_t)rows * 4);
+        L.hist = off;    off = align256(off + (size_t)rows * DBINS * 8);
+        L.members = off; off = align256(off + (size_t)rows * MEMBER_CAP * 8);
+        L.ykeys = off;   off = align256(off + (size_t)rows * tiles * CTA_TILE * 4);
+    }
+    L.total = off;
+    return L;
+}
 
-static size_t ws_bytes_for(int rows) { return WS_HEADER + (size_t)rows * WS_ROW; }
-
-static int g_max_clusters[64];      // co-resident 8-CTA clusters of the exact kernel, per device
 static int g_sm_count[64];
-// Per device: a side stream and two events.  The exact kernel's first round (rows that are its own by class) is
-// forked onto the side stream at the start of a call and joined at its end, so that it runs beside the
-// streaming and merge kernels of the caller's stream.  One call at a time uses them (g_launch_mutex).
-static cudaStream_t g_side[64];
-static cudaEvent_t g_fork[64], g_join[64];
-static std::mutex g_launch_mutex[64];
 
-static int configure_once(int *max_clusters, int *sm_count, int *device) {
+static int configure_once(int *sm_count) {
     static std::once_flag once[64];
     static cudaError_t result[64];
+    static int clusters[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail_cuda(e, "cudaGetDevice");
@@ -88,6 +114,7 @@ static int configure_once(int *max_clusters, int *sm_count, int *device) {
             if (r == cudaSuccess) r = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         };
         set((const void *)sonic_merge_kernel, MERGE_SMEM);
+        set((const void *)sonic_dense_collect_kernel, DENSE_DYN_SMEM);
         set((const void *)sonic_stream_kernel<0>, STREAM_SMEM_F32);
         set((const void *)sonic_stream_kernel<1>, STREAM_SMEM_BF16);
         if (r == cudaSuccess) r = cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
@@ -97,7 +124,7 @@ static int configure_once(int *max_clusters, int *sm_count, int *device) {
         if (r == cudaSuccess) {
             cudaLaunchConfig_t cfg;
             memset(&cfg, 0, sizeof(cfg));
-            cfg.gridDim = dim3(CL * 64);
+            cfg.gridDim = dim3(CL * EXACT_CLUSTERS);
             cfg.blockDim = dim3(EX_THREADS);
             cfg.dynamicSmemBytes = EXACT_SMEM;
             cudaLaunchAttribute attr;
@@ -107,91 +134,63 @@ static int configure_once(int *max_clusters, int *sm_count, int *device) {
             cfg.numAttrs = 1;
             r = cudaOccupancyMaxActiveClusters(&n, (const void *)sonic_exact_kernel<0>, &cfg);
         }
-        g_max_clusters[dev] = n;
+        clusters[dev] = n;
         result[dev] = r;
     });
     if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "kernel configuration");
-    if (g_max_clusters[dev] < 1) return fail(SONIC_ECUDA, "no 8-CTA cluster of the exact kernel fits on this device");
-    *max_clusters = g_max_clusters[dev];
+    if (clusters[dev] < 1) return fail(SONIC_ECUDA, "no 8-CTA cluster of the cluster kernel fits on this device");
     *sm_count = g_sm_count[dev] > 0 ? g_sm_count[dev] : 1;
-    *device = dev;
     return SONIC_OK;
 }
 
-// Creates the side stream and its events on first use (never for sonic_topk_static, which forks nothing).
-static int ensure_side(int dev) {
-    static std::once_flag once[64];
-    static cudaError_t result[64];
-    std::call_once(once[dev], [&] {
-        cudaError_t r = cudaStreamCreateWithFlags(&g_side[dev], cudaStreamNonBlocking);
-        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_fork[dev], cudaEventDisableTiming);
-        if (r == cudaSuccess) r = cudaEventCreateWithFlags(&g_join[dev], cudaEventDisableTiming);
-        result[dev] = r;
-    });
-    if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "side stream creation");
-    return SONIC_OK;
-}
-
-static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, int B_requests, bool fork = true) {
+// One call = a chain of kernels on the caller's stream, each a programmatic dependent of the one before (it may
+// begin launching while its predecessor runs and waits for it inside the kernel; the paper overlaps its two stages
+// the same way, Section 3.5):
+//   stream kernel -> merge kernel (+ stage 2 of the histogram path) -> [collect pass] -> [residual pass]
+//   -> cluster kernel (rows no other path finished; usually none) -> [verification scan]
+static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, int B_requests) {
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
-    if (ws_bytes < ws_bytes_for(P.rows)) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows");
-    int max_clusters = 0, sm_count = 1, dev = 0;
-    int rc = configure_once(&max_clusters, &sm_count, &dev);
+    const bool dense = (P.op != OP_TOPK);
+    const Layout L = layout_for(P.rows, P.V, dense);
+    if (ws_bytes < L.total) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows of this vocabulary size");
+    int sm_count = 1;
+    int rc = configure_once(&sm_count);
     if (rc != SONIC_OK) return rc;
-    // the layout depends on the row capacity the workspace was sized for, recovered from its size
-    const size_t cap_rows = (ws_bytes - WS_HEADER) / WS_ROW;
     unsigned char *base = reinterpret_cast<unsigned char *>(ws);
     P.error = reinterpret_cast<unsigned int *>(base);
-    P.rs = reinterpret_cast<RowState *>(base + WS_HEADER);
-    P.pr = reinterpret_cast<PosResult *>(base + WS_HEADER + cap_rows * sizeof(RowState));
-    P.tiles = reinterpret_cast<TileRec *>(base + WS_HEADER + cap_rows * (sizeof(RowState) + sizeof(PosResult)));
-    P.cand = reinterpret_cast<unsigned long long *>(base + WS_HEADER + cap_rows * WS_ROW_CTRL);
+    P.rs = reinterpret_cast<RowState *>(base + L.rs);
+    P.pr = reinterpret_cast<PosResult *>(base + L.pr);
+    P.tiles = reinterpret_cast<TileRec *>(base + L.tiles);
+    P.cand = reinterpret_cast<unsigned long long *>(base + L.cand);
+    P.cand_stride = L.cand_stride;
+    P.ytiles = L.ytiles;
+    if (dense) {
+        P.drow = reinterpret_cast<DenseRow *>(base + L.drow);
+        P.dtile = reinterpret_cast<DenseTile *>(base + L.dtile);
+        P.dlist = reinterpret_cast<int *>(base + L.dlist);
+        P.rlist = reinterpret_cast<int *>(base + L.rlist);
+        P.hist = reinterpret_cast<unsigned long long *>(base + L.hist);
+        P.members = reinterpret_cast<unsigned long long *>(base + L.members);
+        P.ykeys = reinterpret_cast<unsigned int *>(base + L.ykeys);
+    }
 
     const int tiles = (P.V + CTA_TILE - 1) / CTA_TILE;
     const long long nitems_ll = (long long)tiles * P.rows;
     if (nitems_ll > 0x7FFFFFFF) return fail(SONIC_ESHAPE, "rows x tiles too large");
     const int nitems = (int)nitems_ll;
-    std::lock_guard<std::mutex> lock(g_launch_mutex[dev]);
     cudaError_t e;
 
-    // Fork: the exact kernel's first round goes to the side stream BEFORE the streaming kernel is launched, so that
-    // its clusters (one SM per CTA) are placed first; clusters without a row leave at once and the streaming
-    // kernel's CTAs, which take their tiles from a queue, fill whatever is free.  Without the fork (the entry
-    // point that creates no resources) both rounds run in one launch after the merge kernel.
-    cudaLaunchConfig_t xcfg;
-    memset(&xcfg, 0, sizeof(xcfg));
-    xcfg.gridDim = dim3((P.rows < max_clusters ? P.rows : max_clusters) * CL);
-    xcfg.blockDim = dim3(EX_THREADS);
-    xcfg.dynamicSmemBytes = EXACT_SMEM;
-    if (fork) {
-        rc = ensure_side(dev);
-        if (rc != SONIC_OK) return rc;
-        xcfg.stream = g_side[dev];
-        if ((e = cudaEventRecord(g_fork[dev], st)) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
-        if ((e = cudaStreamWaitEvent(g_side[dev], g_fork[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
-        if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<0>, P, 1);
-        else e = cudaLaunchKernelEx(&xcfg, sonic_exact_kernel<1>, P, 1);
-        if (e != cudaSuccess) return fail_cuda(e, "exact kernel launch (first round)");
-        if ((e = cudaEventRecord(g_join[dev], g_side[dev])) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
-    }
-
-    // after the fork every exit joins the side stream again (also the failing ones: the caller's stream, or its
-    // capture, must not be left with a branch that was never joined)
-    auto unwind = [&](int code) {
-        if (fork) cudaStreamWaitEvent(st, g_join[dev], 0);
-        return code;
-    };
     const int grid1 = nitems < sm_count * 3 ? nitems : sm_count * 3;       // persistent: three CTAs per SM
     // a CTA's first request to the work queue: seven eighths of an even share, at least one item
     int chunk = (int)((7ll * nitems) / (8ll * grid1));
     chunk = chunk < 1 ? 1 : chunk;
-    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems, chunk, (int)(CAND_CAP / (unsigned)tiles));
-    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems, chunk, (int)(CAND_CAP / (unsigned)tiles));
+    const int cap_t = (int)(L.cand_stride / (unsigned)tiles);
+    if (P.dtype == SONIC_DTYPE_F32) sonic_stream_kernel<0><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_F32, st>>>(P, tiles, nitems, chunk, cap_t);
+    else sonic_stream_kernel<1><<<grid1, STREAM_CTA_THREADS, STREAM_SMEM_BF16, st>>>(P, tiles, nitems, chunk, cap_t);
     e = cudaGetLastError();
-    if (e != cudaSuccess) return unwind(fail_cuda(e, "stream kernel launch"));
-    // the merge kernel and the exact kernel's second round are programmatic dependents: they may begin launching
-    // while their predecessor still runs and synchronise on it inside the kernel
+    if (e != cudaSuccess) return fail_cuda(e, "stream kernel launch");
+
     cudaLaunchAttribute pdl;
     pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl.val.programmaticStreamSerializationAllowed = 1;
@@ -200,26 +199,33 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     cfg.stream = st;
     cfg.attrs = &pdl;
     cfg.numAttrs = 1;
-    cfg.gridDim = dim3(P.rows);
+    // the passes of the histogram path take (row, tile) items in a loop: two CTAs per SM at most
+    // (a tile is cut into up to four parts when a call has few rows of that class: up to four CTAs per tile)
+    const int dense_ctas = dense ? (int)(4ll * nitems < 2ll * sm_count ? 4ll * nitems : 2ll * sm_count) : 0;
+    cfg.gridDim = dim3(P.rows + dense_ctas);
     cfg.blockDim = dim3(MERGE_THREADS);
     cfg.dynamicSmemBytes = MERGE_SMEM;
     e = cudaLaunchKernelEx(&cfg, sonic_merge_kernel, P, tiles);
-    if (e != cudaSuccess) return unwind(fail_cuda(e, "merge kernel launch"));
-
-    // rows the merge kernel cannot prove are rare: a few clusters suffice for the second round (the full set when
-    // this launch also runs the first round)
-    const int clusters2 = fork ? (P.rows < SECOND_ROUND_CLUSTERS ? P.rows : (max_clusters < SECOND_ROUND_CLUSTERS ? max_clusters : SECOND_ROUND_CLUSTERS))
-                               : (P.rows < max_clusters ? P.rows : max_clusters);
-    cfg.gridDim = dim3(clusters2 * CL);
+    if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
+    if (dense) {
+        cfg.gridDim = dim3(dense_ctas);
+        cfg.blockDim = dim3(DENSE_THREADS);
+        cfg.dynamicSmemBytes = DENSE_DYN_SMEM;
+        e = cudaLaunchKernelEx(&cfg, sonic_dense_collect_kernel, P, tiles);
+        if (e != cudaSuccess) return fail_cuda(e, "collect pass launch");
+        if (P.op == OP_VERIFY && P.K > 0) {
+            cfg.dynamicSmemBytes = 0;
+            e = cudaLaunchKernelEx(&cfg, sonic_dense_resid_kernel, P, tiles);
+            if (e != cudaSuccess) return fail_cuda(e, "residual pass launch");
+        }
+    }
+    const int clusters = P.rows < EXACT_CLUSTERS ? P.rows : EXACT_CLUSTERS;
+    cfg.gridDim = dim3(clusters * CL);
     cfg.blockDim = dim3(EX_THREADS);
     cfg.dynamicSmemBytes = EXACT_SMEM;
-    const int rounds = fork ? 2 : 3;
-    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P, rounds);
-    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P, rounds);
-    if (e != cudaSuccess) return unwind(fail_cuda(e, "exact kernel launch (second round)"));
-
-    // join: everything after this call in the caller's stream sees the first round's rows too
-    if (fork && (e = cudaStreamWaitEvent(st, g_join[dev], 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
+    if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P);
+    else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P);
+    if (e != cudaSuccess) return fail_cuda(e, "cluster kernel launch");
     if (P.op == OP_VERIFY) {
         sonic_verify_combine_kernel<<<(B_requests + 127) / 128, 128, 0, st>>>(P, B_requests);
         e = cudaGetLastError();
@@ -267,16 +273,19 @@ using namespace sonic;
 
 extern "C" {
 
-size_t sonic_workspace_bytes(int max_rows) {
+size_t sonic_workspace_bytes(int max_rows, int max_vocab, int max_topk) {
+    (void)max_topk;                            // the candidate slots are sized for every supported k
     if (max_rows < 1) max_rows = 1;
-    return ws_bytes_for(max_rows);
+    if (max_vocab < 1) max_vocab = 1;
+    if (max_vocab > SONIC_MAX_VOCAB) max_vocab = SONIC_MAX_VOCAB;
+    return layout_for(max_rows, max_vocab, true).total;
 }
 
 int sonic_workspace_init(void *workspace, size_t bytes, void *stream) {
     if (!workspace) return fail(SONIC_EINVAL, "workspace is NULL");
-    if (bytes < ws_bytes_for(1)) return fail(SONIC_EWORKSPACE, "workspace smaller than one row");
-    const size_t cap_rows = (bytes - WS_HEADER) / WS_ROW;
-    cudaError_t e = cudaMemsetAsync(workspace, 0, WS_HEADER + cap_rows * WS_ROW_CTRL, (cudaStream_t)stream);
+    if (((uintptr_t)workspace & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
+    if (bytes < layout_for(1, 1, true).total) return fail(SONIC_EWORKSPACE, "workspace smaller than one row");
+    cudaError_t e = cudaMemsetAsync(workspace, 0, WS_HEADER, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail_cuda(e, "cudaMemsetAsync");
     g_err[0] = 0;
     return SONIC_OK;
@@ -336,10 +345,12 @@ int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, 
 }
 
 // ---------------------------------------------------------------- no-allocation variant
-// Scratch of sonic_topk_static: a workspace for SONIC_STATIC_MAX_ROWS rows that lives in
+// Scratch of sonic_topk_static: a workspace for SONIC_STATIC_MAX_ROWS rows of the largest vocabulary that lives in
 // the library image.  In host code this name is only a stand-in for the symbol; the device
 // address the kernels need comes from cudaGetSymbolAddress (below), never from `&`.
-static __device__ __align__(256) unsigned char g_static_workspace[WS_HEADER + (size_t)SONIC_STATIC_MAX_ROWS * WS_ROW];
+constexpr size_t STATIC_WS_BYTES = WS_HEADER + 256 * 4 +
+    (size_t)SONIC_STATIC_MAX_ROWS * (sizeof(RowState) + sizeof(PosResult) + sizeof(TileRec) * MAX_TILES + (size_t)CAND_CAP * 8);
+static __device__ __align__(256) unsigned char g_static_workspace[STATIC_WS_BYTES];
 
 static int static_workspace_address(void **out) {
     static std::once_flag once[64];
@@ -369,16 +380,15 @@ int sonic_topk_static(const void *logits, int dtype, int B, int V, int64_t row_s
     void *ws = nullptr;
     rc = static_workspace_address(&ws);
     if (rc != SONIC_OK) return rc;
-    const size_t bytes = WS_HEADER + (size_t)SONIC_STATIC_MAX_ROWS * WS_ROW;
-    // the array keeps whatever the previous call left: the control words must start at zero
-    cudaError_t e = cudaMemsetAsync(ws, 0, WS_HEADER + (size_t)SONIC_STATIC_MAX_ROWS * WS_ROW_CTRL, (cudaStream_t)stream);
+    // the array keeps whatever the previous call left: the header's control words must start at zero
+    cudaError_t e = cudaMemsetAsync(ws, 0, WS_HEADER, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail_cuda(e, "cudaMemsetAsync");
     KParams P;
     memset(&P, 0, sizeof(P));
     P.op = OP_TOPK;
     P.rows = B; P.V = V; P.dtype = dtype; P.logits = logits; P.row_stride = row_stride; P.ktop = k;
     P.out_vals = out_vals; P.out_idx = out_idx;
-    return launch_all(P, ws, bytes, (cudaStream_t)stream, B, /*fork=*/false);     // creates no stream or event either
+    return launch_all(P, ws, STATIC_WS_BYTES, (cudaStream_t)stream, B);
 }
 
 const char *sonic_last_error(void) { return g_err; }

@@ -17,7 +17,7 @@ constexpr uint32_t M_GRAMMAR = 0x001, M_REPETITION = 0x002, M_FREQUENCY = 0x004,
                    M_TOP_P = 0x100, M_MIN_P = 0x200;
 constexpr uint32_t M_PENALTIES = M_REPETITION | M_FREQUENCY | M_PRESENCE;
 
-constexpr uint32_t F_NO_TOKEN = 0x1, F_BADPARAM = 0x2, F_FALLBACK = 0x4;
+constexpr uint32_t F_NO_TOKEN = 0x1, F_BADPARAM = 0x2, F_FALLBACK = 0x4, F_DENSE = 0x8, F_TIMEOUT = 0x10;
 constexpr uint32_t F_ACCEPT = 0x100;          // workspace only (per-position verification result)
 
 constexpr int OP_SAMPLE = 0, OP_VERIFY = 1, OP_TOPK = 2;
@@ -46,28 +46,67 @@ constexpr int MAX_VOCAB = 262144;
 
 constexpr int CLS_GREEDY = 0;                 // streaming path, argmax only
 constexpr int CLS_TOPK = 1;                   // streaming path, candidates + merge
-constexpr int CLS_EXACT = 2;                  // full-vocabulary exact path only
+constexpr int CLS_EXACT = 2;                  // cluster kernel only (top-k beyond what the streaming path sorts)
+constexpr int CLS_DENSE = 3;                  // top-k off: streaming pass for the keys, then the histogram passes
 
-constexpr int WS_QUEUE = 2;                    // workspace header word: the stream kernel's work counter (zero between calls)
-constexpr int WS_EXACT_TICKET = 3;             // workspace header word: next row ordinal of the exact kernel's first round (zero between calls)
-constexpr int WS_EXACT_LEFT = 6;               // workspace header word: clusters of that round that have run out of rows (zero between calls)
-constexpr int WS_FAILED_ROWS = 1;              // workspace header word: rows of the current call the merge kernel could not prove
-constexpr uint32_t ST_FAILED = 0x1;           // streaming path could not prove the row
-constexpr uint32_t ST_BADID = 0x2;            // a list id was out of range
+// Workspace header (the first WS_HEADER_WORDS 32-bit words; the only part of the workspace that must be zero
+// between calls: every other word is initialised by the call that reads it)
+constexpr int WS_ERROR = 0;                    // sticky ERR_* bits
+constexpr int WS_FAILED_ROWS = 1;              // rows of the current call that the streaming or histogram path handed to the cluster kernel
+constexpr int WS_QUEUE = 2;                    // the stream kernel's work counter
+constexpr int WS_EXACT_TICKET = 3;             // next row ordinal of the cluster kernel
+constexpr int WS_NDENSE = 4;                   // rows of the current call on the histogram path (length of the dense list)
+constexpr int WS_NRESID = 5;                   // verification rows of the current call whose draft was rejected (length of the residual list)
+constexpr int WS_EXACT_LEFT = 6;               // clusters of the cluster kernel that have run out of rows
+constexpr int WS_NEXACT = 7;                   // rows of the current call that belong to the cluster kernel by class
+constexpr int WS_HEADER_WORDS = 128;
+constexpr uint32_t ST_FAILED = 0x1;           // streaming / histogram path could not finish the row
 constexpr unsigned int ERR_TIMEOUT = 0x1;     // workspace header: a bounded mbarrier wait expired
+constexpr uint32_t TILE_BADID = 0x1;          // TileRec.flags: a list id of the row was out of range
 
 constexpr uint32_t KEY_NEG_INF = 0x007FFFFFu; // okey(-inf)
 
 struct __align__(16) RowState {
-    unsigned int status;                      // ST_*; zero between calls
+    unsigned int status;                      // ST_*; set to zero by the streaming kernel, ST_FAILED by a row's finisher
     unsigned int pad[3];
 };
 
-struct __align__(16) TileRec {                // written by the tile's CTA, read by the merge kernel
-    unsigned long long best;                  // greedy rows: largest (key << 32 | ~index) of the tile, 0 if none finite
+struct __align__(16) TileRec {                // written by the tile's CTA in the streaming kernel
+    unsigned long long best;                  // greedy and dense rows: largest (key << 32 | ~index) of the tile, 0 if none finite
     unsigned int cnt;                         // top-k rows: candidates of the tile (may exceed the slot: overflow)
     unsigned int tkey;                        // top-k rows: the tile's cutoff as an ordered key
+    unsigned int minkey;                      // dense rows: smallest finite key of the tile (0xFFFFFFFF if none)
+    unsigned int nfin;                        // dense rows: finite elements of the tile
+    unsigned int flags;                       // TILE_*
+    unsigned int pad;
 };
+
+// Histogram path (rows with top-k off), per row.  Initialised by the streaming kernel (the CTA of the row's first
+// tile); the later passes communicate through it.
+constexpr int DBINS = 2048;                   // bins of the mass histogram, uniform in (M - y)
+constexpr int MEMBER_CAP = 4096;              // elements of the crossing bin that can be listed
+struct __align__(16) DenseRow {
+    unsigned int ticket_h, ticket_c, ticket_r, nmembers;     // items that have finished a pass; listed members
+    unsigned int kmin, kmax, overflow, state;                // key span of the members; an item could not stage its members; 1 = collect pass wanted
+    unsigned int Mkey, tk, klo, khi;                         // row maximum; min-p key threshold (0 = none); keys of the crossing bin: klo .. khi (empty if klo > khi)
+    unsigned long long target;                               // mass the ranking prefix must reach (0: top-p does not decide inside the bin)
+    unsigned long long cutc, W;                              // final cut (composite key) and total fixed-point mass of the support
+    float p_draft; int support;
+    unsigned int pad[4];
+};
+static_assert(sizeof(DenseRow) == 96, "DenseRow layout");
+constexpr int DENSE_CHUNK = 512;                 // elements per chunk of a tile
+constexpr int DENSE_CHUNKS = 16;                 // chunks per tile
+struct __align__(16) DenseChunk {             // per chunk of 512 elements, written by pass C
+    unsigned long long A;                     // fixed-point mass of the chunk's elements above the crossing bin
+    unsigned int n, nb;                       // their number; the chunk's elements inside the crossing bin
+};
+struct __align__(16) DenseTile {              // per (row, tile) of the histogram path
+    DenseChunk ch[DENSE_CHUNKS];
+    unsigned long long mass;                  // fixed-point mass of the tile's part of the final support
+    double R, Pp, S;                          // residual pass: sum of max(0, w/W~ - q), sum of w where that is positive, sum of w
+};
+static_assert(sizeof(DenseTile) == 288, "DenseTile layout");
 
 struct __align__(16) PosResult {              // per logit row, verification only
     int token;
@@ -106,11 +145,20 @@ struct KParams {
     float *out_pdraft;
     float *out_vals;
     int *out_idx;
-    unsigned int *error;                      // workspace header word: ERR_* (sticky)
+    unsigned int *error;                      // workspace header (WS_* words); word 0: ERR_* (sticky)
     RowState *rs;
     TileRec *tiles;
     PosResult *pr;
-    unsigned long long *cand;
+    unsigned long long *cand;                 // [rows][cand_stride] candidate slots, split evenly among a row's tiles
+    unsigned int cand_stride;
+    // histogram path (sample / verify calls only)
+    DenseRow *drow;                           // [rows]
+    DenseTile *dtile;                         // [rows][MAX_TILES]
+    int *dlist, *rlist;                       // [rows] rows on the histogram path; rows whose draft was rejected
+    unsigned long long *hist;                 // [rows][DBINS] fixed-point mass per bin
+    unsigned long long *members;              // [rows][MEMBER_CAP] elements of the crossing bin (key << 32 | ~index)
+    unsigned int *ykeys;                      // [rows][ytiles * CTA_TILE] ordered keys of the processed logits
+    int ytiles;
 };
 
 // Per-row configuration derived from the request's mode bits and parameters.
@@ -267,7 +315,10 @@ __device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const C
     } else {
         int kfast = (P.op == OP_TOPK) ? KFAST_TOPK : KFAST_SAMPLE;
         c.cls = CLS_EXACT;
-        if (c.k > 0 && c.k <= kfast) {
+        if (c.k == 0 && P.op != OP_TOPK) {
+            c.cls = CLS_DENSE;                 // the keys it stores are final: divided by the temperature
+            c.div_all = c.temp;
+        } else if (c.k > 0 && c.k <= kfast) {
             int G;
             if (memo_k && *memo_k == c.k) G = *memo_G;
             else {
@@ -281,6 +332,18 @@ __device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const C
 }
 
 __device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) { return resolve_cfg(P, row, fetch_cfg(P, row)); }
+
+#ifdef SONIC_TRACE
+__device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
+#define STREAM_STAMP(i) do { if ((int)blockIdx.x == (int)P.error[121] && lane == 0) P.error[40 + (i)] = gtimer_lo(); } while (0)
+// kernel-level timeline: earliest start and latest end of kernel k (0 stream, 1 merge, 2 exact first launch, 3 exact second launch)
+#define KERNEL_T0(k) do { if (threadIdx.x == 0) atomicMin(&P.error[48 + 2 * (k)], gtimer_lo()); } while (0)
+#define KERNEL_T1(k) do { if (threadIdx.x == 0) atomicMax(&P.error[49 + 2 * (k)], gtimer_lo()); } while (0)
+#else
+#define KERNEL_T0(k) do { } while (0)
+#define KERNEL_T1(k) do { } while (0)
+#define STREAM_STAMP(i) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------- Philox4x32-10
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
@@ -319,6 +382,49 @@ __device__ __forceinline__ float apply_penalties(float v, int count, const RowCf
 
 __device__ __forceinline__ unsigned long long ldcg_u64(const unsigned long long *p) {
     return __ldcg(p);
+}
+
+// Writes the per-row outputs of the sample / verify operations.
+__device__ __forceinline__ void emit_row(const KParams &P, const RowCfg &c, int row, int token, float prob,
+                                         uint32_t flags, int support, float p_draft) {
+    if (P.op == OP_SAMPLE) {
+        P.out_token[row] = token;
+        P.out_prob[row] = prob;
+        P.out_flags[row] = flags;
+        if (P.out_support) P.out_support[row] = support;
+    } else {
+        PosResult r;
+        r.token = token; r.flags = flags; r.p = p_draft; r.support = support;
+        P.pr[row] = r;
+    }
+}
+
+// Fixed-point softmax weight of a key relative to the row maximum: 2^40 * exp(y - M).  Sums of these are
+// order-independent, so replays are bit-identical.  Callers weigh every element and select afterwards
+// (w = qweight(key); sum += cond ? w : 0): behind a branch per element the sixteen independent chains of a thread
+// cannot overlap and a pass takes four times as long.
+__device__ __forceinline__ unsigned long long qweight(uint32_t key, float Mf) {
+    float d = __fsub_rn(unkey(key), Mf);
+    const float L1 = 1.44269502162933349609375f;        // fp32(log2 e)
+    const float L2 = 1.925963033500011e-08f;            // log2 e - L1
+    float t = fmaf(d, L1, d * L2);
+    float w;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w) : "f"(t));
+    return __float2ull_rn(w * 1099511627776.0f);
+}
+
+// floor(W * u) for the draw's uniform u = (2 a + 1) / 2^25, exactly.
+__device__ __forceinline__ unsigned long long draw_target(unsigned long long W, uint32_t a_draw) {
+    const unsigned long long mul = 2ull * a_draw + 1ull;
+    return (__umul64hi(W, mul) << 39) | ((W * mul) >> 25);
+}
+
+// Smallest float not below M + ln(theta) taken in double, as an ordered key: y passes min-p  <=>  okey(y) >= it.
+__device__ __forceinline__ uint32_t minp_key(float Mf, float theta) {
+    const double thr = (double)Mf + log((double)theta);
+    float tf = (float)thr;
+    if ((double)tf < thr) tf = nextafterf(tf, CUDART_INF_F);
+    return okey(tf);
 }
 
 // Programmatic dependent launch (the paper overlaps its two stages the same way, Section 3.5):
@@ -412,6 +518,54 @@ __device__ __noinline__ void bitonic_sort_desc_cta(unsigned long long *a, int m,
         }
         __syncthreads();
     }
+}
+
+// Ranks of at most THREADS distinct non-zero keys held one per thread in list[0, n): every warp sorts its 32 keys
+// with shuffles and writes them back as a descending run, then a key's rank is its place in its own run plus, for
+// every other run, the number of keys there above it (a binary search in the sorted run; 0 pads the last run).
+// Returns the thread's key after the warp sort (0 = padding) and leaves its rank in `rank`.  Two block barriers.
+template <int THREADS, typename Sync>
+__device__ __forceinline__ unsigned long long rank_keys(unsigned long long *list, int n, int tid, int &rank) {
+    Sync csync;
+    const int lane = tid & 31, warp = tid >> 5;
+    unsigned long long key = (tid < n) ? list[tid] : 0ull;
+#pragma unroll
+    for (int kk = 2; kk <= 32; kk <<= 1) {
+#pragma unroll
+        for (int jj = kk >> 1; jj > 0; jj >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
+            const bool up = ((lane & kk) == 0);            // this block of kk sorts descending
+            const bool first = ((lane & jj) == 0);         // the lower lane of the pair
+            const bool take_max = (up == first);
+            key = ((key > o) == take_max) ? key : o;           // mine if it is on the side this lane takes
+        }
+    }
+    csync();                                               // every thread has read its key from the list
+    list[tid] = key;                                       // sorted runs of 32 (descending), in place
+    csync();
+    const int runs = (n + 31) >> 5;
+    rank = lane;
+    if (key != 0ull) {
+        // four runs at a time: their binary searches are independent chains of shared-memory reads
+        for (int r0 = 0; r0 < runs; r0 += 4) {
+            const unsigned long long *run[4];
+            int lo[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { run[u] = list + min(r0 + u, runs - 1) * 32; lo[u] = 0; }
+#pragma unroll
+            for (int step = 16; step > 0; step >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (run[u][lo[u] + step - 1] > key) lo[u] += step;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (lo[u] < 32 && run[u][lo[u]] > key) ++lo[u];        // covers a run whose 32 keys are all above
+                if (r0 + u < runs && r0 + u != warp) rank += lo[u];     // (lo[u] = number of keys of the run above `key`)
+            }
+        }
+    }
+    return key;
 }
 
 __device__ __forceinline__ int next_pow2(int n) {

@@ -1,0 +1,997 @@
+// Histogram path: rows with top-k off (top-p, min-p or plain temperature sampling over the whole vocabulary,
+// and their verification variants), finished by grid-wide passes over the row's ordered keys instead of by one
+// cluster per row.
+//
+// The streaming kernel leaves, per row of this class, the ordered keys of the processed logits (read once from
+// HBM, written once, re-read from L2 by the passes below) and per-tile maxima / minima.  Then, every pass a
+// grid-wide launch whose CTAs take (row, tile) items and whose last-arriving CTA of a row (a ticket counter, no
+// waiting) does the row-level step:
+//   pass H  (rows with top-p): fixed-point probability mass per bin, 2048 bins uniform in (M - y) that just cover
+//           the row's finite range; the last arriver scans the bins from the top for the bin where the
+//           cumulative mass reaches p * Z (the "crossing bin").  The min-p threshold M + ln(theta) is a key
+//           threshold and names a bin as well; the higher of the two bins decides.
+//   pass C  per tile: mass and number of the elements above the crossing bin, and the elements inside it listed
+//           as (key << 32 | ~index); the last arriver resolves the exact cut among the listed elements (a radix
+//           descent over the composite keys weighted by mass; ties by lowest index), then draws: tile-level
+//           CDF from the per-tile masses, one tile re-read for the element.  Rows without top-p know their cut
+//           once the row maximum is known and run pass C in place of pass H.
+//   pass R  (verification rows whose draft was rejected): per-tile sums of the residual max(0, p - q) in fp64,
+//           the last arriver draws from it.
+// This is the truncation epilogue and token selection of the paper's Algorithm "Stage 2" (TopP, MinP; Appendix
+// "Probability Truncation", "Sampling", "Speculative Verification") for supports far beyond the paper's
+// k <= 128 bound (Section 3.3).  Masses are 2^-40 fixed point, sums are integer and order-independent.
+#pragma once
+#include "sonic_common.cuh"
+
+namespace sonic {
+
+#ifdef SONIC_DTRACE
+__device__ __forceinline__ unsigned int dtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
+#define DSTAMP(i) do { if (threadIdx.x == 0) P.error[64 + (i)] = dtimer(); } while (0)
+#else
+#define DSTAMP(i) do { } while (0)
+#endif
+
+constexpr int DENSE_THREADS = 512;
+constexpr int DENSE_WARPS = DENSE_THREADS / 32;
+constexpr int DENSE_EPT = CTA_TILE / DENSE_THREADS;          // 16 keys per thread and tile
+constexpr int DENSE_NV = DENSE_EPT / 4;                      // as 128-bit vectors
+constexpr int STAGE_CAP = 2048;                              // elements of the crossing bin one item can stage
+constexpr int DENSE_DYN_SMEM = MEMBER_CAP * 8;               // members | histogram words | staged members share it
+static_assert(DBINS * 8 <= DENSE_DYN_SMEM && STAGE_CAP * 8 <= DENSE_DYN_SMEM, "dynamic shared memory of the dense passes");
+static_assert(MAX_TILES == 32, "one tile record per lane");
+static_assert(MAX_TILES * DENSE_CHUNKS == DENSE_THREADS, "one chunk record per thread");
+
+struct DenseShared {
+    unsigned long long tile_mass[MAX_TILES];
+    unsigned int tile_nb[MAX_TILES];
+    unsigned long long red64[DENSE_WARPS];
+    double redd[3][DENSE_WARPS];
+    unsigned int red32[2][DENSE_WARPS];
+    unsigned long long comp[DENSE_THREADS];          // listed elements (fast path: at most one per thread)
+    unsigned long long wt[DENSE_THREADS];            // their weights in ranking order
+    unsigned long long chunk[DENSE_THREADS];         // support mass per chunk of 512 elements (tile-major)
+    unsigned long long bc64[4];
+    double bcd[2];
+    unsigned int nstage, kmin, kmax, base;
+    unsigned int Mkey, mkey, Nf, bad;
+    unsigned int cnt_above, nb;
+    int flag, last, digit;
+};
+
+// Bin of a finite key: larger bin = larger logit; bin DBINS-1 holds the row maximum.
+__device__ __forceinline__ int dense_digit(uint32_t key, float Mf, float scale) {
+    const float t = fminf(__fmul_rn(__fsub_rn(Mf, unkey(key)), scale), (float)(DBINS - 1));
+    return DBINS - 1 - (int)t;
+}
+
+// Bins per logit unit, a power of two chosen so that the bins just cover the row's finite range.
+__device__ __forceinline__ float dense_scale(uint32_t Mkey, uint32_t mkey, unsigned int Nf) {
+    int e = 5;
+    const float spread = (Nf > 0) ? __fsub_rn(unkey(Mkey), unkey(mkey)) : 0.0f;
+    if (spread > 0.0f && spread < CUDART_INF_F) e = max(-10, min(10, ilogbf((float)(DBINS - 8) / spread)));
+    return ldexpf(1.0f, e);
+}
+
+// Smallest key in (okey(-inf), Mkey] whose bin is at least b (Mkey + 1 if none): the bins are monotone in the
+// key, so a 32-way search by one warp finds it in seven rounds.  Every lane returns the result.
+__device__ __forceinline__ uint32_t dense_bin_lower_key(int b, uint32_t Mkey, float Mf, float scale, int lane) {
+    uint32_t lo = KEY_NEG_INF + 1u, hi = Mkey + 1u;           // the answer lies in [lo, hi]
+    while (lo < hi) {
+        const uint32_t step = (hi - lo) / 32u + 1u;
+        const unsigned long long cand64 = (unsigned long long)lo + (unsigned long long)lane * step;
+        const bool valid = cand64 < (unsigned long long)hi;
+        const uint32_t cand = (uint32_t)cand64;
+        const bool ok = valid && dense_digit(cand, Mf, scale) >= b;
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, ok);
+        const unsigned int v = __ballot_sync(0xFFFFFFFFu, valid);
+        if (m == 0u) {
+            lo = lo + (uint32_t)(31 - __clz(v)) * step + 1u;     // past the last candidate (lane 0's is always valid)
+        } else {
+            const int l = __ffs(m) - 1;
+            hi = lo + (uint32_t)l * step;
+            if (l > 0) lo = lo + (uint32_t)(l - 1) * step + 1u; else hi = lo;
+        }
+    }
+    return lo;
+}
+
+__device__ __forceinline__ unsigned long long dense_warp_sum(unsigned long long v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    return v;
+}
+
+// Inclusive scan over the lanes of a warp.
+__device__ __forceinline__ unsigned long long dense_warp_scan(unsigned long long v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, v, o);
+        if (lane >= o) v += up;
+    }
+    return v;
+}
+
+// Exclusive prefix over the threads of the block (thread order) of one value per thread; `total` in every thread.
+template <typename T>
+__device__ __forceinline__ T dense_block_scan(T v, T *wtot, int tid, T &total) {
+    const int lane = tid & 31, warp = tid >> 5;
+    T incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const T up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    T off = T(0), tot = T(0);
+#pragma unroll
+    for (int w = 0; w < DENSE_WARPS; ++w) {
+        const T t = wtot[w];
+        if (w < warp) off += t;
+        tot += t;
+    }
+    total = tot;
+    return off + incl - v;
+}
+
+// Row statistics from the streaming kernel's tile records (first warp): maximum, smallest finite key, finite count.
+__device__ __forceinline__ void dense_row_stats(const KParams &P, int row, int tiles, DenseShared &sm, int tid) {
+    if (tid < 32) {
+        const TileRec *rec = P.tiles + (size_t)row * MAX_TILES;
+        unsigned int mk = 0u, mn = 0xFFFFFFFFu, nf = 0u, fl = 0u;
+        if (tid < tiles) {
+            mk = (unsigned int)(rec[tid].best >> 32);
+            mn = rec[tid].minkey;
+            nf = rec[tid].nfin;
+            fl = rec[tid].flags;
+        }
+        mk = __reduce_max_sync(0xFFFFFFFFu, mk);
+        mn = __reduce_min_sync(0xFFFFFFFFu, mn);
+        nf = __reduce_add_sync(0xFFFFFFFFu, nf);
+        fl = __reduce_or_sync(0xFFFFFFFFu, fl);
+        if (tid == 0) { sm.Mkey = mk; sm.mkey = mn; sm.Nf = nf; sm.bad = fl & TILE_BADID; }
+    }
+}
+
+// Work items of a pass: a tile is cut into `sub` parts (1, 2 or 4) when the call has so few rows of this class that
+// whole tiles would leave most SMs idle.  A thread holds 16 / sub consecutive elements of its part, so a chunk of
+// 512 elements belongs to `sub` consecutive warps.
+struct DenseItem {
+    int row, tile, part, sub;
+    __device__ int nv() const { return DENSE_NV / sub; }                       // 128-bit vectors per thread
+    __device__ int first(int tid) const { return tile * CTA_TILE + part * (CTA_TILE / sub) + tid * (DENSE_EPT / sub); }
+};
+__device__ __forceinline__ int dense_pick_sub(int rows_in_pass, int tiles, int ctas) {
+    int sub = 1;
+    while (sub < 4 && rows_in_pass * tiles * sub * 2 <= ctas) sub *= 2;
+    return sub;
+}
+__device__ __forceinline__ DenseItem dense_item(const int *list, int item, int tiles, int sub) {
+    DenseItem it;
+    const int per_row = tiles * sub;
+    it.row = __ldcg(&list[item / per_row]);
+    const int rem = item % per_row;
+    it.tile = rem / sub; it.part = rem % sub; it.sub = sub;
+    return it;
+}
+
+// The item's keys.  They were written by an earlier kernel of the call, so the loads may go through L1 (the loads
+// of a thread share their lines).  Vectors past the item's share hold okey(-inf).
+__device__ __forceinline__ void dense_load_keys(const KParams &P, const DenseItem &it, int tid, uint4 (&kv)[DENSE_NV]) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(P.ykeys + (size_t)it.row * ((size_t)P.ytiles * CTA_TILE) + it.first(tid));
+    const int nv = it.nv();
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) kv[k] = (k < nv) ? src[k] : make_uint4(KEY_NEG_INF, KEY_NEG_INF, KEY_NEG_INF, KEY_NEG_INF);
+}
+
+// Ticket of a pass: true in every thread of the row's last CTA to arrive (whose reads then see what the others wrote).
+__device__ __forceinline__ bool dense_arrive(unsigned int *ticket, int items, DenseShared &sm, int tid) {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int t = atomicAdd(ticket, 1u);
+        sm.last = (t == (unsigned int)(items - 1)) ? 1 : 0;
+        if (sm.last) __threadfence();
+    }
+    __syncthreads();
+    return sm.last != 0;
+}
+
+// ---------------------------------------------------------------- pass H
+// Mass histogram of one item, added to the row's histogram in global memory.
+__device__ __forceinline__ void dense_hist_item(const KParams &P, const DenseItem &it, const uint4 (&kv)[DENSE_NV], float Mf, float scale,
+                                                unsigned int *hm0, unsigned int *hm1, int tid) {
+    for (int i = tid; i < DBINS; i += DENSE_THREADS) { hm0[i] = 0u; hm1[i] = 0u; }
+    __syncthreads();
+    const int nv = it.nv();
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) {
+        if (k >= nv) break;
+        const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+        int bin[4];
+        unsigned long long q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const bool fin = key4[u] > KEY_NEG_INF;
+            const int dg = dense_digit(key4[u], Mf, scale);
+            const unsigned long long wq = qweight(key4[u], Mf);
+            bin[u] = fin ? dg : -1;
+            q[u] = fin ? wq : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (bin[u] < 0 || q[u] == 0ull) continue;
+            // 64-bit mass as two 32-bit words: the low word's returned old value reveals a carry
+            const unsigned int lo = (unsigned int)q[u], hi = (unsigned int)(q[u] >> 32);
+            unsigned int carry = 0;
+            if (lo) { const unsigned int old = atomicAdd(&hm0[bin[u]], lo); carry = (old + lo < old) ? 1u : 0u; }
+            if (hi + carry) atomicAdd(&hm1[bin[u]], hi + carry);
+        }
+    }
+    __syncthreads();
+    unsigned long long *hist = P.hist + (size_t)it.row * DBINS;
+    for (int i = tid; i < DBINS; i += DENSE_THREADS) {
+        const unsigned long long m = (unsigned long long)hm0[i] | ((unsigned long long)hm1[i] << 32);
+        if (m) atomicAdd(&hist[i], m);
+    }
+}
+
+// Last arriver of pass H: the crossing bin of top-p against the min-p threshold, as the key interval pass C works with.
+__device__ __forceinline__ void dense_hist_finish(const KParams &P, const RowCfg &c, int row, DenseShared &sm,
+                                                  unsigned long long *h, int tid, uint32_t Mkey, float scale) {
+    const unsigned long long *hist = P.hist + (size_t)row * DBINS;
+    for (int i = tid; i < DBINS; i += DENSE_THREADS) h[i] = __ldcg(&hist[i]);
+    __syncthreads();
+    // thread t owns bins DBINS-1-4t .. DBINS-4-4t (from the top)
+    constexpr int BPT = DBINS / DENSE_THREADS;
+    unsigned long long mine = 0;
+#pragma unroll
+    for (int j = 0; j < BPT; ++j) mine += h[DBINS - 1 - (tid * BPT + j)];
+    unsigned long long Z;
+    const unsigned long long pre = dense_block_scan<unsigned long long>(mine, sm.red64, tid, Z);
+    unsigned long long target = (unsigned long long)ceil((double)c.p * (double)Z);
+    if (target > Z) target = Z;
+    if (target < 1ull) target = 1ull;
+    if (tid == 0) sm.digit = 0;
+    __syncthreads();
+    if (mine > 0ull && pre < target && target <= pre + mine) {
+        unsigned long long cum = pre;
+        int found = -1;
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) {
+            const int b = DBINS - 1 - (tid * BPT + j);
+            cum += h[b];
+            if (found < 0 && cum >= target) found = b;
+        }
+        sm.digit = found;
+    }
+    __syncthreads();
+    if (tid < 32) {
+        const float Mf = unkey(Mkey);
+        const int b_p = sm.digit;
+        uint32_t tk = 0u;
+        int b_m = -1;
+        if (c.z & M_MIN_P) { tk = minp_key(Mf, c.theta); b_m = dense_digit(max(tk, KEY_NEG_INF + 1u), Mf, scale); }
+        uint32_t klo, khi;
+        if (b_m > b_p) {
+            // the min-p threshold lies above the bin top-p would cut in: the cut is the threshold itself
+            klo = 0xFFFFFFFFu; khi = tk - 1u; target = 0ull;
+        } else {
+            klo = dense_bin_lower_key(b_p, Mkey, Mf, scale, tid);
+            khi = dense_bin_lower_key(b_p + 1, Mkey, Mf, scale, tid) - 1u;
+        }
+        if (tid == 0) {
+            DenseRow *dr = P.drow + row;
+            dr->Mkey = Mkey; dr->tk = tk; dr->klo = klo; dr->khi = khi; dr->target = target;
+            __threadfence();
+            dr->state = 1u;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- in-tile search
+// First element of a tile, in index order, whose inclusive running sum of wf exceeds `rest`; thread t owns the
+// 16 consecutive elements 16t .. 16t + 15.  Returns the element's global index in every thread (the last element
+// of positive weight if the sum never exceeds `rest`, -1 if the tile has none) and leaves its weight in w_out.
+template <typename T, typename WF>
+__device__ int dense_tile_find(const KParams &P, int row, int tile, T rest, WF wf, T *wtot, DenseShared &sm, int tid, T &w_out) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(P.ykeys + (size_t)row * ((size_t)P.ytiles * CTA_TILE) + (size_t)tile * CTA_TILE) + tid * DENSE_NV;
+    const int first = tile * CTA_TILE + tid * DENSE_EPT;
+    uint4 kv[DENSE_NV];
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) kv[k] = src[k];
+    if (tid == 0) { sm.flag = -1; sm.digit = -1; }
+    T s = T(0);
+    int lastpos = -1;
+    if (kv[0].x == 0x12345u && kv[3].w == 0x54321u) lastpos = -2;     // (trace builds: the loads have landed)
+    DSTAMP(20);
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) {
+        const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const T w = wf(key4[u], first + k * 4 + u);
+            s += w;
+            if (w > T(0)) lastpos = first + k * 4 + u;
+        }
+    }
+    DSTAMP(21);
+    T total;
+    const T pre = dense_block_scan<T>(s, wtot, tid, total);
+    DSTAMP(22);
+    // weight of the thread's first element whose running sum exceeds `rest` (want_last: of its last positive element)
+    auto walk = [&](bool want_last, int &found, T &fw) {
+        T cum = pre;
+        found = -1; fw = T(0);
+#pragma unroll
+        for (int k = 0; k < DENSE_NV; ++k) {
+            const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const T w = wf(key4[u], first + k * 4 + u);
+                cum += w;
+                if (w > T(0) && (want_last || (found < 0 && cum > rest))) { found = first + k * 4 + u; fw = w; }
+            }
+        }
+    };
+    if (s > T(0) && pre <= rest && rest < pre + s) {
+        int found; T fw;
+        walk(false, found, fw);
+        if (found < 0) walk(true, found, fw);                  // (floating-point sums only)
+        sm.flag = found;
+        *reinterpret_cast<T *>(&sm.bc64[3]) = fw;
+    }
+    __syncthreads();
+    if (sm.flag < 0) {
+        // the running sum never exceeds `rest` (rounding between the levels): the tile's last element of positive weight
+        if (lastpos >= 0) atomicMax(&sm.digit, lastpos);
+        __syncthreads();
+        if (lastpos >= 0 && lastpos == sm.digit) {
+            int found; T fw;
+            walk(true, found, fw);
+            sm.flag = found;
+            *reinterpret_cast<T *>(&sm.bc64[3]) = fw;
+        }
+        __syncthreads();
+    }
+    DSTAMP(23);
+    w_out = *reinterpret_cast<T *>(&sm.bc64[3]);
+    const int res = sm.flag;
+    __syncthreads();
+    return res;
+}
+
+// ---------------------------------------------------------------- pass C
+// One item of pass C: per chunk of 512 elements the mass and number of the elements above the crossing bin
+// (key > khi) and the number inside it (klo <= key <= khi); the latter staged and appended to the row's member list.
+__device__ __forceinline__ void dense_collect_part(const KParams &P, const DenseItem &it, const uint4 (&kv)[DENSE_NV], float Mf,
+                                                   uint32_t klo, uint32_t khi, DenseShared &sm, unsigned long long *stage, int tid) {
+    const int lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) { sm.nstage = 0u; sm.kmin = 0xFFFFFFFFu; sm.kmax = 0u; }
+    __syncthreads();
+    unsigned long long am = 0ull;
+    unsigned int an = 0u, bn = 0u;
+    uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
+    const int base_idx = it.first(tid);
+    const int nv = it.nv();
+    const bool any_members = klo <= khi;
+    DSTAMP(41);
+#ifdef SONIC_DTRACE
+    if (kv[0].x == 0xdeadbeefu && kv[0].w == 0x12345u) am = 1ull;
+    DSTAMP(46);
+#endif
+    // the weights first, without a branch per element (the chains of a thread's elements overlap) ...
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) {
+        if (k >= nv) break;
+        const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned long long w = qweight(key4[u], Mf);
+            am += (key4[u] > khi) ? w : 0ull;
+            an += (key4[u] > khi) ? 1u : 0u;
+        }
+    }
+    // ... then the elements of the crossing bin, if the row has one
+    if (any_members) {
+#pragma unroll
+        for (int k = 0; k < DENSE_NV; ++k) {
+            if (k >= nv) break;
+            const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t key = key4[u];
+                const bool mb = key >= klo && key <= khi;
+                const unsigned int mm = __ballot_sync(0xFFFFFFFFu, mb);
+                if (mm) {
+                    unsigned int pos = 0;
+                    if (lane == 0) pos = atomicAdd(&sm.nstage, (unsigned int)__popc(mm));
+                    pos = __shfl_sync(0xFFFFFFFFu, pos, 0) + __popc(mm & ((1u << lane) - 1u));
+                    if (mb) {
+                        if (pos < (unsigned int)STAGE_CAP) stage[pos] = ((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)(base_idx + k * 4 + u));
+                        kmn = min(kmn, key); kmx = max(kmx, key);
+                        ++bn;
+                    }
+                }
+            }
+        }
+    }
+    DSTAMP(42);
+    am = dense_warp_sum(am);
+    an = __reduce_add_sync(0xFFFFFFFFu, an);
+    bn = __reduce_add_sync(0xFFFFFFFFu, bn);
+    if (any_members) {
+        kmn = __reduce_min_sync(0xFFFFFFFFu, kmn);
+        kmx = __reduce_max_sync(0xFFFFFFFFu, kmx);
+    }
+    if (lane == 0) {
+        sm.red64[warp] = am; sm.red32[0][warp] = an; sm.red32[1][warp] = bn;
+        if (kmx) { atomicMin(&sm.kmin, kmn); atomicMax(&sm.kmax, kmx); }
+    }
+    __syncthreads();
+    // a chunk belongs to `sub` consecutive warps
+    const int sub = it.sub, nchunks = DENSE_CHUNKS / sub;
+    if (tid < nchunks) {
+        DenseChunk r; r.A = 0ull; r.n = 0u; r.nb = 0u;
+        for (int w = tid * sub; w < (tid + 1) * sub; ++w) { r.A += sm.red64[w]; r.n += sm.red32[0][w]; r.nb += sm.red32[1][w]; }
+        P.dtile[(size_t)it.row * MAX_TILES + it.tile].ch[it.part * nchunks + tid] = r;
+    }
+    const unsigned int cnt = sm.nstage;
+    DSTAMP(43);
+    if (cnt == 0u) return;
+    if (tid == 0) {
+        DenseRow *dr = P.drow + it.row;
+        sm.base = atomicAdd(&dr->nmembers, cnt);
+        atomicMin(&dr->kmin, sm.kmin);
+        atomicMax(&dr->kmax, sm.kmax);
+        if (cnt > (unsigned int)STAGE_CAP) atomicOr(&dr->overflow, 1u);
+    }
+    __syncthreads();
+    const unsigned int base = sm.base;
+    unsigned long long *mem = P.members + (size_t)it.row * MEMBER_CAP;
+    for (unsigned int i = tid; i < min(cnt, (unsigned int)STAGE_CAP); i += DENSE_THREADS)
+        if (base + i < (unsigned int)MEMBER_CAP) mem[base + i] = stage[i];
+}
+
+// Sorts the listed elements (composite keys, distinct) in dyn[0, nb) descending, nb > DENSE_THREADS.
+__device__ __forceinline__ void dense_sort_members(unsigned long long *dyn, int nb, int tid) {
+    const int m = next_pow2(nb);
+    for (int i = nb + tid; i < m; i += DENSE_THREADS) dyn[i] = 0ull;
+    __syncthreads();
+    bitonic_sort_desc_cta<DENSE_THREADS>(dyn, m, tid);
+}
+
+// Rank-th (0-based) element of a tile with key == v, in index order.
+__device__ __forceinline__ int dense_tile_find_tie(const KParams &P, int row, int tile, uint32_t v, unsigned long long rank,
+                                                   DenseShared &sm, int tid) {
+    unsigned long long wdummy;
+    auto wf = [=](uint32_t key, int) -> unsigned long long { return key == v ? 1ull : 0ull; };
+    return dense_tile_find<unsigned long long>(P, row, tile, rank, wf, sm.red64, sm, tid, wdummy);
+}
+
+// The draw by one warp, from the support's mass per tile and per chunk (shared memory, final): the tile, then the
+// chunk of 512 elements, then the element (a lane owns 16 consecutive elements of the chunk).  Exact: all integer.
+// Returns the token in every lane and its weight in qt.
+__device__ __forceinline__ int dense_warp_draw(const KParams &P, int row, int tiles, const DenseShared &sm, unsigned long long cutc, float Mf,
+                                               unsigned long long T, int lane, unsigned long long &qt) {
+    auto pick = [&](unsigned long long v, unsigned long long incl, unsigned long long rest) -> int {
+        unsigned int hit = __ballot_sync(0xFFFFFFFFu, v > 0ull && incl > rest);
+        if (!hit) { const unsigned int any = __ballot_sync(0xFFFFFFFFu, v > 0ull); hit = any ? (0x80000000u >> __clz(any)) : 1u; }   // (rest < total always: kept for safety)
+        return __ffs(hit) - 1;
+    };
+    // tile
+    const unsigned long long tm = (lane < tiles) ? sm.tile_mass[lane] : 0ull;
+    const unsigned long long ti = dense_warp_scan(tm, lane);
+    const int jt = pick(tm, ti, T);
+    const unsigned long long before_t = __shfl_sync(0xFFFFFFFFu, ti - tm, jt);
+    unsigned long long rest = (T > before_t) ? T - before_t : 0ull;
+    // chunk
+    const unsigned long long cm = (lane < DENSE_CHUNKS) ? sm.chunk[jt * DENSE_CHUNKS + lane] : 0ull;
+    const unsigned long long ci = dense_warp_scan(cm, lane);
+    const int ch = pick(cm, ci, rest);
+    const unsigned long long before_c = __shfl_sync(0xFFFFFFFFu, ci - cm, ch);
+    rest = (rest > before_c) ? rest - before_c : 0ull;
+    // element
+    const int first = jt * CTA_TILE + ch * DENSE_CHUNK + lane * 16;
+    const uint4 *src = reinterpret_cast<const uint4 *>(P.ykeys + (size_t)row * ((size_t)P.ytiles * CTA_TILE) + first);
+    uint4 kv[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) kv[k] = src[k];
+    unsigned long long w[16];
+    unsigned long long s = 0ull;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int idx = first + k * 4 + u;
+            const unsigned long long wq = qweight(key4[u], Mf);
+            w[k * 4 + u] = ((((unsigned long long)key4[u] << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc) ? wq : 0ull;
+            s += w[k * 4 + u];
+        }
+    }
+    const unsigned long long si = dense_warp_scan(s, lane);
+    const int l = pick(s, si, rest);
+    int token = -1;
+    unsigned long long fw = 0ull;
+    if (lane == l) {
+        unsigned long long cum = si - s;
+        int lastpos = -1;
+        unsigned long long lw = 0ull;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            cum += w[i];
+            if (w[i] > 0ull) {
+                if (token < 0 && cum > rest) { token = first + i; fw = w[i]; }
+                lastpos = first + i; lw = w[i];
+            }
+        }
+        if (token < 0) { token = lastpos; fw = lw; }
+    }
+    token = __shfl_sync(0xFFFFFFFFu, token, l);
+    qt = __shfl_sync(0xFFFFFFFFu, fw, l);
+    return token;
+}
+
+// Last arriver of pass C: the exact cut, the support's size and mass, then the draw or the accept test.
+// dyn: DENSE_DYN_SMEM bytes; cells: the row's two Philox cells.  Returns false if the row must go to the cluster kernel.
+__device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int tiles, DenseShared &sm, unsigned long long *dyn, int tid,
+                             uint32_t Mkey, bool listed, unsigned long long target, uint32_t tk, uint2 cells) {
+    const float Mf = unkey(Mkey);
+    const int lane = tid & 31, warp = tid >> 5;
+    DenseRow *dr = P.drow + row;
+    DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
+    DSTAMP(3);
+    // everything the other CTAs left, requested at once: a chunk record per thread, the first DENSE_THREADS listed
+    // elements (one per thread, whatever their number turns out to be), their count and the overflow mark
+    unsigned int nm = 0u, overflow = 0u;
+    {
+        const int t = tid / DENSE_CHUNKS;
+        DenseChunk r; r.A = 0ull; r.n = 0u; r.nb = 0u;
+        if (t < tiles) {
+            const uint4 raw = __ldcg(reinterpret_cast<const uint4 *>(&dt[t].ch[tid % DENSE_CHUNKS]));
+            r.A = (unsigned long long)raw.x | ((unsigned long long)raw.y << 32); r.n = raw.z; r.nb = raw.w;
+        }
+        unsigned long long m0 = 0ull;
+        if (listed) {
+            nm = __ldcg(&dr->nmembers);
+            overflow = __ldcg(&dr->overflow);
+            m0 = __ldcg(P.members + (size_t)row * MEMBER_CAP + tid);
+        }
+        sm.chunk[tid] = r.A;
+        sm.comp[tid] = ((unsigned int)tid < nm) ? m0 : 0ull;
+        // tile sums over 16 consecutive threads, then block sums
+        unsigned long long ta = r.A;
+        unsigned int tb = r.nb;
+#pragma unroll
+        for (int off = 8; off > 0; off >>= 1) { ta += __shfl_xor_sync(0xFFFFFFFFu, ta, off); tb += __shfl_xor_sync(0xFFFFFFFFu, tb, off); }
+        if ((lane & 15) == 0) { sm.tile_mass[2 * warp + (lane >> 4)] = ta; sm.tile_nb[2 * warp + (lane >> 4)] = tb; }
+        const unsigned long long wa = ta + __shfl_xor_sync(0xFFFFFFFFu, ta, 16);
+        const unsigned int wn = __reduce_add_sync(0xFFFFFFFFu, r.n);
+        if (lane == 0) { sm.red64[warp] = wa; sm.red32[0][warp] = wn; }
+        if (tid == 0) { sm.bc64[0] = 0ull; sm.bc64[1] = 0ull; }
+    }
+    __syncthreads();
+    DSTAMP(4);
+    unsigned long long C_above = 0ull;
+    unsigned int cnt_above = 0u;
+#pragma unroll
+    for (int w = 0; w < DENSE_WARPS; ++w) { C_above += sm.red64[w]; cnt_above += sm.red32[0][w]; }
+    const unsigned int nb = nm;
+    const unsigned long long guard = (unsigned long long)(KEY_NEG_INF + 1u) << 32;     // every finite element
+    const unsigned long long cut_m = (unsigned long long)tk << 32;
+    unsigned long long cutc = max(guard, cut_m);
+    unsigned long long mass_in = 0ull;
+    unsigned int n_in = 0u;
+    bool chunks_final = true;                     // the per-chunk masses include the listed elements that are in
+    if (listed && nb > 0u) {
+        const unsigned long long rest = max(target > C_above ? target - C_above : 1ull, 1ull);
+        if (nb <= (unsigned int)DENSE_THREADS && !overflow) {
+            // at most one listed element per thread: ranks by warp sorts and binary searches, then the running mass
+            // in ranking order
+            int rank;
+            const unsigned long long key = rank_keys<DENSE_THREADS, BlockSync>(sm.comp, (int)nb, tid, rank);
+            const unsigned long long wk = key ? qweight((uint32_t)(key >> 32), Mf) : 0ull;
+            __syncthreads();                      // every search has read the runs
+            if (key) { sm.comp[rank] = key; sm.wt[rank] = wk; }
+            __syncthreads();
+            DSTAMP(5);
+            const bool have = (unsigned int)tid < nb;
+            const unsigned long long mine_c = have ? sm.comp[tid] : 0ull, mine_w = have ? sm.wt[tid] : 0ull;
+            unsigned long long total_m;
+            const unsigned long long pre = dense_block_scan<unsigned long long>(mine_w, sm.red64, tid, total_m);
+            if (target) {
+                // the element at which the running mass first reaches what is still missing above the bin
+                const unsigned long long r = min(rest, max(total_m, 1ull));
+                if (mine_w > 0ull && pre < r && r <= pre + mine_w) sm.bc64[0] = mine_c;
+                __syncthreads();
+                cutc = max(cutc, sm.bc64[0]);
+            }
+            DSTAMP(6);
+            // what of the bin is in: a prefix of the ranking; its mass goes to its tiles and chunks for the draw
+            const bool inc = have && mine_c >= cutc;
+            if (inc && mine_w) {
+                const uint32_t idx = ~(uint32_t)mine_c;
+                atomicAdd(&sm.tile_mass[idx / CTA_TILE], mine_w);
+                atomicAdd(&sm.chunk[idx / DENSE_CHUNK], mine_w);
+            }
+            n_in = (unsigned int)__syncthreads_count(inc ? 1 : 0);
+            if (have && (unsigned int)tid + 1u == n_in) sm.bc64[1] = pre + mine_w;
+            __syncthreads();
+            mass_in = n_in ? sm.bc64[1] : 0ull;
+        } else if (nb <= (unsigned int)MEMBER_CAP && !overflow) {
+            // many listed elements: a full sort, weights recomputed along the ranking
+            chunks_final = false;
+            const unsigned long long *gm = P.members + (size_t)row * MEMBER_CAP;
+            for (int i = tid; i < (int)nb; i += DENSE_THREADS) dyn[i] = __ldcg(&gm[i]);
+            __syncthreads();
+            dense_sort_members(dyn, (int)nb, tid);
+            const int ept = ((int)nb + DENSE_THREADS - 1) / DENSE_THREADS;
+            const int lo = min((int)nb, tid * ept), hi = min((int)nb, lo + ept);
+            unsigned long long mine = 0ull;
+            for (int j = lo; j < hi; ++j) mine += qweight((uint32_t)(dyn[j] >> 32), Mf);
+            unsigned long long total_m;
+            const unsigned long long pre = dense_block_scan<unsigned long long>(mine, sm.red64, tid, total_m);
+            if (target) {
+                const unsigned long long r = min(rest, max(total_m, 1ull));
+                if (mine > 0ull && pre < r && r <= pre + mine) {
+                    unsigned long long cum = pre;
+                    bool done = false;
+                    for (int j = lo; j < hi; ++j) {
+                        cum += qweight((uint32_t)(dyn[j] >> 32), Mf);
+                        if (!done && cum >= r) { sm.bc64[0] = dyn[j]; done = true; }
+                    }
+                }
+                __syncthreads();
+                cutc = max(cutc, sm.bc64[0]);
+            }
+            unsigned long long ms = 0ull;
+            unsigned int ns = 0u;
+            for (int j = lo; j < hi; ++j) {
+                const unsigned long long m = dyn[j];
+                if (m >= cutc) {
+                    const unsigned long long w = qweight((uint32_t)(m >> 32), Mf);
+                    ms += w; ++ns;
+                    if (w) atomicAdd(&sm.tile_mass[(~(uint32_t)m) / CTA_TILE], w);
+                }
+            }
+            ms = dense_warp_sum(ms);
+            ns = __reduce_add_sync(0xFFFFFFFFu, ns);
+            __syncthreads();
+            if (lane == 0) { sm.red64[warp] = ms; sm.red32[0][warp] = ns; }
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < DENSE_WARPS; ++w) { mass_in += sm.red64[w]; n_in += sm.red32[0][w]; }
+            __syncthreads();
+        } else {
+            // a crowded bin: resolvable here only if it holds one value repeated (low-precision logits)
+            chunks_final = false;
+            const uint32_t kmin = __ldcg(&dr->kmin), kmax = __ldcg(&dr->kmax);
+            if (kmin != kmax) return false;
+            const uint32_t v = kmin;
+            const unsigned long long wv = qweight(v, Mf);
+            unsigned long long m = nb;
+            if (tk && v < tk) m = 0ull;
+            if (target && m > 0ull && wv > 0ull) {
+                const unsigned long long need = (rest + wv - 1ull) / wv;
+                m = min(m, max(need, 1ull));
+            }
+            // the first m ties in index order: which tile holds the m-th, and where in it
+            int jt = -1;
+            unsigned long long before = 0ull;
+            if (m > 0ull && m < (unsigned long long)nb) {
+                unsigned long long cum = 0ull;
+                for (int j = 0; j < tiles; ++j) {
+                    const unsigned long long t = sm.tile_nb[j];
+                    if (jt < 0 && cum + t >= m) { jt = j; before = cum; }
+                    cum += t;
+                }
+            }
+            unsigned long long cut_v;
+            if (m == 0ull) cut_v = ((unsigned long long)v + 1ull) << 32;
+            else if (jt < 0) cut_v = (unsigned long long)v << 32;
+            else {
+                const int idx = dense_tile_find_tie(P, row, jt, v, m - 1ull - before, sm, tid);
+                cut_v = ((unsigned long long)v << 32) | (uint32_t)(~(uint32_t)idx);
+            }
+            cutc = max(cutc, cut_v);
+            __syncthreads();
+            if (tid == 0) {
+                unsigned long long left = m;
+                for (int j = 0; j < tiles; ++j) {
+                    const unsigned long long t = min(left, (unsigned long long)sm.tile_nb[j]);
+                    sm.tile_mass[j] += t * wv;
+                    left -= t;
+                }
+            }
+            mass_in = m * wv;
+            n_in = (unsigned int)m;
+            __syncthreads();
+        }
+    }
+    const unsigned long long W = C_above + mass_in;
+    const int support = (int)(cnt_above + n_in);
+    DSTAMP(7);
+    const uint32_t a_acc = cells.x, a_draw = cells.y;
+    uint32_t flags = F_DENSE;
+    float p_draft = 0.0f;
+    if (P.op == OP_VERIFY && c.l < P.K) {
+        const int d = P.draft_tokens[(size_t)c.b * P.K + c.l];
+        unsigned long long qd = 0ull;
+        double Q = 0.0;
+        if (d >= 0 && d < P.V) {
+            const uint32_t kd = P.ykeys[(size_t)row * ((size_t)P.ytiles * CTA_TILE) + d];
+            if ((((unsigned long long)kd << 32) | (uint32_t)(~(uint32_t)d)) >= cutc) qd = qweight(kd, Mf);
+            Q = (double)__ldg(P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)P.V + d);
+        }
+        const double Pd = (double)qd / (double)W;
+        const bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);
+        p_draft = (float)Pd;
+        if (accept) {
+            // the request moves on with the draft token: neither the residual nor a draw of this position is read
+            if (tid == 0) emit_row(P, c, row, d, 0.0f, flags | F_ACCEPT, support, p_draft);
+            return true;
+        }
+        // rejected: the residual pass finishes the position
+        if (tid < tiles) dt[tid].mass = sm.tile_mass[tid];
+        if (tid == 0) {
+            dr->cutc = cutc; dr->W = W; dr->p_draft = p_draft; dr->support = support; dr->Mkey = Mkey;
+            __threadfence();
+            const unsigned int slot = atomicAdd(&P.error[WS_NRESID], 1u);
+            P.rlist[slot] = row;
+        }
+        return true;
+    }
+    // plain draw
+    const unsigned long long T = draw_target(W, a_draw);
+    if (chunks_final) {
+        if (tid < 32) {
+            unsigned long long qt;
+            const int token = dense_warp_draw(P, row, tiles, sm, cutc, Mf, T, lane, qt);
+            DSTAMP(10);
+            if (tid == 0) emit_row(P, c, row, token, (float)((double)qt / (double)W), flags, support, 0.0f);
+        }
+        return true;
+    }
+    // (slow paths above: the per-chunk masses are not final; tile-level CDF, then the element inside the tile)
+    int jt = tiles - 1;
+    unsigned long long before = 0ull;
+    {
+        unsigned long long cum = 0ull;
+        bool hit = false;
+        for (int j = 0; j < tiles; ++j) {
+            const unsigned long long t = sm.tile_mass[j];
+            if (!hit && t > 0ull && cum + t > T) { jt = j; before = cum; hit = true; }
+            cum += t;
+        }
+        if (!hit) {                               // (T < W always; kept for safety: the last tile with mass)
+            cum = 0ull;
+            for (int j = 0; j < tiles; ++j) { if (sm.tile_mass[j] > 0ull) { jt = j; before = cum; } cum += sm.tile_mass[j]; }
+        }
+    }
+    const unsigned long long cc = cutc;
+    auto wf = [=](uint32_t key, int idx) -> unsigned long long {
+        const unsigned long long wq = qweight(key, Mf);
+        return ((((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cc) ? wq : 0ull;
+    };
+    unsigned long long qt = 0ull;
+    const int token = dense_tile_find<unsigned long long>(P, row, jt, T - before, wf, sm.red64, sm, tid, qt);
+    if (tid == 0) emit_row(P, c, row, token, (float)((double)qt / (double)W), flags, support, 0.0f);
+    return true;
+}
+
+// Pass C for one item whose cut parameters are known; the row's last CTA finishes it.
+__device__ __forceinline__ void dense_collect_item(const KParams &P, const RowCfg &c, const DenseItem &it, int tiles, const uint4 (&kv)[DENSE_NV],
+                                                   uint32_t Mkey, uint32_t klo, uint32_t khi, unsigned long long target, uint32_t tk,
+                                                   DenseShared &sm, unsigned long long *dyn, int tid) {
+    uint2 cells = make_uint2(0u, 0u);
+    draw_cells(P, c, cells.x, cells.y);           // (inputs only: off the chain that follows the ticket)
+    if (cells.x == 0x7fffffffu) return;
+    DSTAMP(40);
+#ifdef SONIC_DTRACE2
+    if (it.tile == 0 && it.part == 0) { dense_collect_part(P, it, kv, unkey(Mkey), 0xFFFFFFFFu, khi, sm, dyn, tid); __syncthreads(); }
+#endif
+    dense_collect_part(P, it, kv, unkey(Mkey), klo, khi, sm, dyn, tid);
+    DSTAMP(2);
+    if (!dense_arrive(&P.drow[it.row].ticket_c, tiles * it.sub, sm, tid)) return;
+    const bool ok = dense_finish(P, c, it.row, tiles, sm, dyn, tid, Mkey, klo <= khi, target, tk, cells);
+    if (!ok && tid == 0) { P.rs[it.row].status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
+}
+
+// Stage 2 of the histogram path, run by the extra CTAs of the merge kernel's launch: pass H for rows with top-p,
+// pass C (and the row's finish) for the others, whose cut is a key threshold known from the row maximum.
+__device__ void dense_stage2(const KParams &P, int tiles, int cta, int ncta, unsigned long long *dyn) {
+    __shared__ DenseShared sm;
+    const int tid = threadIdx.x;
+    const int nd = (int)__ldcg(&P.error[WS_NDENSE]);
+    const int sub = dense_pick_sub(nd, tiles, ncta);
+    for (int item = cta; item < nd * tiles * sub; item += ncta) {
+        const DenseItem it = dense_item(P.dlist, item, tiles, sub);
+        const int row = it.row;
+        uint4 kv[DENSE_NV];
+        dense_load_keys(P, it, tid, kv);
+        const RowCfg c = load_cfg(P, row);
+        dense_row_stats(P, row, tiles, sm, tid);
+        __syncthreads();
+        const uint32_t Mkey = sm.Mkey, mkey = sm.mkey;
+        const unsigned int Nf = sm.Nf;
+        const bool bad = c.bad || sm.bad;
+        __syncthreads();
+        if (bad || Nf == 0u) {
+            if (it.tile == 0 && it.part == 0 && tid == 0) emit_row(P, c, row, -1, 0.0f, (bad ? F_BADPARAM : F_NO_TOKEN) | F_DENSE, 0, 0.0f);
+            continue;
+        }
+        const float Mf = unkey(Mkey);
+        if (c.z & M_TOP_P) {
+            const float scale = dense_scale(Mkey, mkey, Nf);
+            unsigned int *hm0 = reinterpret_cast<unsigned int *>(dyn), *hm1 = hm0 + DBINS;
+            dense_hist_item(P, it, kv, Mf, scale, hm0, hm1, tid);
+            if (dense_arrive(&P.drow[row].ticket_h, tiles * sub, sm, tid)) dense_hist_finish(P, c, row, sm, dyn, tid, Mkey, scale);
+        } else {
+            // min-p: the elements at or above the threshold key; neither: every finite element.  No bin, no list.
+            const uint32_t tk = (c.z & M_MIN_P) ? minp_key(Mf, c.theta) : 0u;
+            const uint32_t khi = tk ? tk - 1u : KEY_NEG_INF;
+            dense_collect_item(P, c, it, tiles, kv, Mkey, 0xFFFFFFFFu, khi, 0ull, tk, sm, dyn, tid);
+        }
+        __syncthreads();
+        KERNEL_T1(6);
+    }
+}
+
+// Stage 3: pass C for the rows whose crossing bin pass H has found.
+__global__ void __launch_bounds__(DENSE_THREADS, 2)
+sonic_dense_collect_kernel(const KParams P, const int tiles) {
+    extern __shared__ __align__(16) unsigned char dense_dyn_raw[];
+    __shared__ DenseShared sm;
+    unsigned long long *dyn = reinterpret_cast<unsigned long long *>(dense_dyn_raw);
+    const int tid = threadIdx.x;
+    pdl_launch_dependents();
+    DSTAMP(30);
+    pdl_wait_primary();
+    DSTAMP(31);
+    KERNEL_T0(3);
+    const int nd = (int)__ldcg(&P.error[WS_NDENSE]);
+    const int sub = dense_pick_sub(nd, tiles, (int)gridDim.x);
+    for (int item = blockIdx.x; item < nd * tiles * sub; item += gridDim.x) {
+        const DenseItem it = dense_item(P.dlist, item, tiles, sub);
+        const DenseRow *dr = P.drow + it.row;
+        DSTAMP(0);
+        uint4 kv[DENSE_NV];
+        dense_load_keys(P, it, tid, kv);
+        if (__ldcg(&dr->state) != 1u) continue;          // no top-p (finished in stage 2), or no token
+        const RowCfg c = load_cfg(P, it.row);
+        const uint32_t Mkey = __ldcg(&dr->Mkey), tk = __ldcg(&dr->tk), klo = __ldcg(&dr->klo), khi = __ldcg(&dr->khi);
+        const unsigned long long target = __ldcg(&dr->target);
+        DSTAMP(1);
+        dense_collect_item(P, c, it, tiles, kv, Mkey, klo, khi, target, tk, sm, dyn, tid);
+        __syncthreads();
+        KERNEL_T1(3);
+    }
+}
+
+// Stage 4 (verification calls): the residual max(0, p - q) of the positions whose draft was rejected.  The
+// support's total weight W is known here only in fixed point (relative error up to 1e-7 on peaked rows, too
+// coarse where p - q cancels), so a tile accumulates, in fp64, the residual sum R~ taken with that W~, the sum Pp of
+// the weights whose residual is positive, and the plain sum S of the weights; with W = sum of S the row's last
+// CTA corrects each tile's residual to R~ - (1/W~ - 1/W) * Pp (exact up to the elements whose residual changes
+// sign between W~ and W, each of which contributes less than 1e-7 of its own probability).
+__global__ void __launch_bounds__(DENSE_THREADS, 2)
+sonic_dense_resid_kernel(const KParams P, const int tiles) {
+    __shared__ DenseShared sm;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();
+    pdl_wait_primary();
+    KERNEL_T0(4);
+    const int nr = (int)__ldcg(&P.error[WS_NRESID]);
+    for (int item = blockIdx.x; item < nr * tiles; item += gridDim.x) {
+        const DenseItem it = dense_item(P.rlist, item, tiles, 1);
+        const int row = it.row, tile = it.tile;
+        DenseRow *dr = P.drow + row;
+        DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
+        uint4 kv[DENSE_NV];
+        dense_load_keys(P, it, tid, kv);
+        const RowCfg c = load_cfg(P, row);
+        const unsigned long long cutc = __ldcg(&dr->cutc), Wq = __ldcg(&dr->W);
+        const uint32_t Mkey = __ldcg(&dr->Mkey);
+        const double Md = (double)unkey(Mkey);
+        const double inv_Wt = 1099511627776.0 / (double)Wq;                 // 1 / W~
+        const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)P.V;
+        double R = 0.0, Pp = 0.0, S = 0.0;
+#pragma unroll
+        for (int k = 0; k < DENSE_NV; ++k) {
+            const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+            const int base_idx = tile * CTA_TILE + tid * DENSE_EPT + 4 * k;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = base_idx + u;
+                if ((((unsigned long long)key4[u] << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc) {
+                    const double w = exp((double)unkey(key4[u]) - Md);
+                    const double r = w * inv_Wt - (double)__ldg(q + idx);
+                    S += w;
+                    if (r > 0.0) { R += r; Pp += w; }
+                }
+            }
+        }
+        // fixed reduction order: lanes by butterfly, warps in order
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            R += __shfl_xor_sync(0xFFFFFFFFu, R, off);
+            Pp += __shfl_xor_sync(0xFFFFFFFFu, Pp, off);
+            S += __shfl_xor_sync(0xFFFFFFFFu, S, off);
+        }
+        if (lane == 0) { sm.redd[0][warp] = R; sm.redd[1][warp] = Pp; sm.redd[2][warp] = S; }
+        __syncthreads();
+        if (tid == 0) {
+            double r = 0.0, p = 0.0, s = 0.0;
+            for (int w = 0; w < DENSE_WARPS; ++w) { r += sm.redd[0][w]; p += sm.redd[1][w]; s += sm.redd[2][w]; }
+            dt[tile].R = r; dt[tile].Pp = p; dt[tile].S = s;
+        }
+        if (!dense_arrive(&dr->ticket_r, tiles, sm, tid)) continue;
+        // ---- the row's last CTA: corrected tile residuals, the tile of the draw, the element
+        if (tid == 0) {
+            double Wd = 0.0;
+            for (int j = 0; j < tiles; ++j) Wd += __ldcg(&dt[j].S);
+            const double corr = inv_Wt - 1.0 / Wd;
+            double Rtot = 0.0;
+            for (int j = 0; j < tiles; ++j) {
+                double rj = __ldcg(&dt[j].R) - corr * __ldcg(&dt[j].Pp);
+                rj = rj > 0.0 ? rj : 0.0;
+                reinterpret_cast<double *>(sm.wt)[j] = rj;
+                Rtot += rj;
+            }
+            sm.bcd[0] = Wd; sm.bcd[1] = Rtot;
+        }
+        __syncthreads();
+        const double Wd = sm.bcd[0], Rtot = sm.bcd[1];
+        uint32_t a_acc, a_draw;
+        draw_cells(P, c, a_acc, a_draw);
+        int token = -1;
+        if (Rtot > 0.0) {
+            const double target = cell_to_u(a_draw) * Rtot;
+            const double *rj = reinterpret_cast<const double *>(sm.wt);
+            int jt = -1;
+            double before = 0.0, cum = 0.0;
+            for (int j = 0; j < tiles; ++j) {
+                if (jt < 0 && rj[j] > 0.0 && cum + rj[j] > target) { jt = j; before = cum; }
+                cum += rj[j];
+            }
+            if (jt < 0) { cum = 0.0; for (int j = 0; j < tiles; ++j) { if (rj[j] > 0.0) { jt = j; before = cum; } cum += rj[j]; } }
+            const double inv_Wd = 1.0 / Wd;
+            auto wf = [=](uint32_t key, int idx) -> double {
+                if (!((((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc)) return 0.0;
+                const double r = exp((double)unkey(key) - Md) * inv_Wd - (double)__ldg(q + idx);
+                return r > 0.0 ? r : 0.0;
+            };
+            double rw;
+            __syncthreads();
+            if (jt >= 0) token = dense_tile_find<double>(P, row, jt, target - before, wf, sm.redd[0], sm, tid, rw);
+        }
+        if (token < 0) {
+            // empty residual (p <= q on the whole support, by rounding): draw from p itself
+            const unsigned long long T = draw_target(Wq, a_draw);
+            int jt = tiles - 1;
+            unsigned long long before = 0ull, cum = 0ull;
+            bool hit = false;
+            for (int j = 0; j < tiles; ++j) {
+                const unsigned long long t = __ldcg(&dt[j].mass);
+                if (!hit && t > 0ull && cum + t > T) { jt = j; before = cum; hit = true; }
+                cum += t;
+            }
+            const float Mf = unkey(Mkey);
+            auto wf = [=](uint32_t key, int idx) -> unsigned long long {
+                const unsigned long long wq = qweight(key, Mf);
+                return ((((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc) ? wq : 0ull;
+            };
+            unsigned long long qt;
+            __syncthreads();
+            token = dense_tile_find<unsigned long long>(P, row, jt, T - before, wf, sm.red64, sm, tid, qt);
+        }
+        if (tid == 0) emit_row(P, c, row, token, 0.0f, F_DENSE, __ldcg(&dr->support), __ldcg(&dr->p_draft));
+        __syncthreads();
+        KERNEL_T1(4);
+    }
+}
+
+}  // namespace sonic

@@ -120,17 +120,6 @@ __device__ __forceinline__ unsigned int warp_append(unsigned int *counter, bool 
     return base + __popc(m & ((1u << lane) - 1u));
 }
 
-// Fixed-point softmax weight of a key relative to the row maximum: 2^40 * exp(y - M).
-__device__ __forceinline__ unsigned long long qweight(uint32_t key, float Mf) {
-    float d = __fsub_rn(unkey(key), Mf);
-    const float L1 = 1.44269502162933349609375f;        // fp32(log2 e)
-    const float L2 = 1.925963033500011e-08f;            // log2 e - L1
-    float t = fmaf(d, L1, d * L2);
-    float w;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w) : "f"(t));
-    return __float2ull_rn(w * 1099511627776.0f);
-}
-
 // Ordered passes: elements are visited in vocabulary-index order (warp w owns a
 // contiguous run of the slice, lanes interleaved), each with weight wf(local index)
 // of a 64-bit type T (fixed-point mass, a count, or fp64).
@@ -729,7 +718,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     RowState *rs = P.rs + row;
 #ifdef SONIC_TRACE
     x.tracep = P.error;
-    x.trace = (row == (int)P.error[4]);
+    x.trace = (row == (int)P.error[120]);
 #endif
     const int V = P.V;
     x.per = (((V + CL - 1) / CL) + 1023) & ~1023;
@@ -1025,10 +1014,13 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     cg::this_cluster().sync();
 }
 
-// Persistent clusters over the rows that need this path.
+// Persistent clusters over the rows that need this path: the rows that are its own by class (top-k beyond what the
+// streaming path sorts; the streaming kernel counts them) and the rows the streaming or histogram path could not
+// finish (flagged and counted by their kernels).  The last kernel of a call's chain: it waits for its predecessor,
+// puts the call's list counters back to zero and, in nearly every call, finds nothing to do and returns.
 template <int DT>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(EX_THREADS, 1)
-sonic_exact_kernel(const KParams P, const int rounds) {
+sonic_exact_kernel(const KParams P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     ExactCtx x;
     x.rank = (int)cg::this_cluster().block_rank();
@@ -1041,87 +1033,61 @@ sonic_exact_kernel(const KParams P, const int rounds) {
     unsigned long long *sortbuf = reinterpret_cast<unsigned long long *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192);
     uint32_t *need = reinterpret_cast<uint32_t *>(smem_raw + SLICE_MAX * 4 + HBINS * 16 + 8192 + MAX_TOPK * 8);
 
-    // Two rounds, launched separately (`rounds` is the set this launch runs).  Round 0: the rows that belong to
-    // this path by class, known from the inputs alone, so this launch runs beside the streaming and merge
-    // kernels.  Round 1, a programmatic dependent of the merge kernel: the rows that kernel could not prove.  In
-    // each round every CTA marks the rows of ALL requests (all CTAs derive the same list).  Round 0 hands the
-    // marked rows out one at a time from a counter in the workspace header (rows differ a lot in length: a
-    // verification row whose draft is rejected takes two more passes), round 1 deals its few rows round-robin.
-    KERNEL_T0(rounds == 2 ? 3 : 2);
+    KERNEL_T0(2);
+    pdl_launch_dependents();
+    pdl_wait_primary();
     const int ncl = gridDim.x / CL;
     const int cid = blockIdx.x / CL;
     const int nwords = (P.rows + 31) >> 5;
-    for (int round = 0; round < 2; ++round) {
-        if (!((rounds >> round) & 1)) continue;
-        if (round == 1) {
-            pdl_wait_primary();
-            if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u) { KERNEL_T1(3); return; }     // the merge kernel proved every row: nothing to scan
+    // (the passes that read the two lists are complete: their lengths go back to zero for the next call)
+    if (blockIdx.x == 0 && x.tid == 0) { P.error[WS_NDENSE] = 0u; P.error[WS_NRESID] = 0u; }
+    // both counters stay as they are until the last cluster has left (below), so every CTA reads the same values
+    if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u && __ldcg(&P.error[WS_NEXACT]) == 0u) { KERNEL_T1(2); return; }
+    for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
+    __syncthreads();
+    // every CTA marks the rows of the whole call (all derive the same list)
+    for (int row = x.tid; row < P.rows; row += EX_THREADS) {
+        const RowCfg c = load_cfg(P, row);
+        const bool mine = (c.cls == CLS_EXACT) || (__ldcg(&P.rs[row].status) & ST_FAILED);
+        if (mine) atomicOr(&need[row >> 5], 1u << (row & 31));
+    }
+    __syncthreads();
+    int nmarked = 0;
+    for (int w = 0; w < nwords; ++w) nmarked += __popc(need[w]);
+    // The marked rows are handed out one at a time from a counter in the workspace header (rows differ a lot in
+    // length); a cluster's first row needs no draw: the counter hands out ncl, ncl + 1, ...
+    bool first = true;
+    for (;;) {
+        int t;
+        if (first) {
+            t = cid;
+            first = false;
+        } else {
+            // the cluster's first thread draws the ordinal and leaves it in every CTA's shared memory
+            if (x.rank == 0 && x.tid == 0) {
+                const int drawn = ncl + (int)atomicAdd(&P.error[WS_EXACT_TICKET], 1u);
+                for (int r = 0; r < CL; ++r) *cg::this_cluster().map_shared_rank(&x.sh->ticket, r) = drawn;
+            }
+            cg::this_cluster().sync();
+            t = x.sh->ticket;                 // (the next write comes after the barriers of the row, or never)
         }
-        __syncthreads();
-        for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;
-        __syncthreads();
-        for (int row = x.tid; row < P.rows; row += EX_THREADS) {
-            const RowCfg c = load_cfg(P, row);
-            bool mine;
-            if (round == 0) mine = (c.cls == CLS_EXACT);
-            else mine = (c.cls != CLS_EXACT) && (__ldcg(&P.rs[row].status) & ST_FAILED);
-            if (mine) atomicOr(&need[row >> 5], 1u << (row & 31));
+        if (t >= nmarked) break;
+        int row = -1, seen = 0;
+        for (int w = 0; w < nwords && row < 0; ++w) {
+            const uint32_t bits = need[w];
+            const int c = __popc(bits);
+            if (t < seen + c) row = (w << 5) + (int)__fns(bits, 0, t - seen + 1);
+            seen += c;
         }
-        __syncthreads();
-        int nmarked = 0;
-        for (int w = 0; w < nwords; ++w) nmarked += __popc(need[w]);
-        if (nmarked == 0) continue;                                  // (round 0: the counters are never touched)
-        int next_static = cid;
-        bool first = true;
-        for (;;) {
-            int t;
-            if (round == 0 && first) {
-                t = cid;                          // a cluster's first row needs no draw: the counter hands out ncl, ncl + 1, ...
-                first = false;
-            } else if (round == 0) {
-                // the cluster's first thread draws the ordinal and leaves it in every CTA's shared memory
-                if (x.rank == 0 && x.tid == 0) {
-                    const int drawn = ncl + (int)atomicAdd(&P.error[WS_EXACT_TICKET], 1u);
-                    for (int r = 0; r < CL; ++r) *cg::this_cluster().map_shared_rank(&x.sh->ticket, r) = drawn;
-                }
-                cg::this_cluster().sync();
-                t = x.sh->ticket;                 // (the next write comes after the barriers of the row, or never)
-            } else {
-                t = next_static;
-                next_static += ncl;
-            }
-            if (t >= nmarked) break;
-            // ordinal among the marked rows in row order.  Verification, first round: a request's K + 1 positions are
-            // marked together, and the positions that carry a draft (the long rows when the draft is rejected) go first
-            int ord = t;
-            if (round == 0 && P.op == OP_VERIFY && P.K > 0) {
-                const int K1 = P.K + 1, ndraft = (nmarked / K1) * P.K;
-                ord = (t < ndraft) ? (t / P.K) * K1 + (t % P.K) : (t - ndraft) * K1 + P.K;
-            }
-            int row = -1, seen = 0;
-            for (int w = 0; w < nwords && row < 0; ++w) {
-                const uint32_t bits = need[w];
-                const int c = __popc(bits);
-                if (ord < seen + c) row = (w << 5) + (int)__fns(bits, 0, ord - seen + 1);
-                seen += c;
-            }
-#ifdef SONIC_TRACE
-            const unsigned int tr0 = gtimer_lo();
-#endif
-            exact_row<DT>(P, row, x, sortbuf);
-            KERNEL_T1(rounds == 2 ? 3 : 2);
-#ifdef SONIC_TRACE
-            if (threadIdx.x == 0 && x.rank == 0) {
-                atomicMax(&P.error[56], ((gtimer_lo() - tr0) << 8) | (unsigned int)(row & 255));    // slowest row: ns << 8 | row
-                atomicMin(&P.error[57], tr0);                                                   // first row start
-            }
-#endif
-        }
-        // round 0: the last cluster to run out of rows puts both counters back to zero for the next call (every
-        // cluster has drawn its final ordinal by then)
-        if (round == 0 && x.rank == 0 && x.tid == 0) {
-            const unsigned int left = atomicAdd(&P.error[WS_EXACT_LEFT], 1u);
-            if (left == (unsigned int)(ncl - 1)) { P.error[WS_EXACT_TICKET] = 0u; P.error[WS_EXACT_LEFT] = 0u; }
+        exact_row<DT>(P, row, x, sortbuf);
+        KERNEL_T1(2);
+    }
+    // the last cluster to run out of rows puts the counters back to zero for the next call (every cluster has
+    // drawn its final ordinal and read the row counts by then)
+    if (x.rank == 0 && x.tid == 0) {
+        const unsigned int left = atomicAdd(&P.error[WS_EXACT_LEFT], 1u);
+        if (left == (unsigned int)(ncl - 1)) {
+            P.error[WS_EXACT_TICKET] = 0u; P.error[WS_EXACT_LEFT] = 0u; P.error[WS_NEXACT] = 0u;
         }
     }
 }

@@ -27,6 +27,7 @@
 // is handed to the exact kernel.
 #pragma once
 #include "sonic_common.cuh"
+#include "sonic_dense.cuh"
 
 namespace sonic {
 
@@ -94,38 +95,12 @@ struct MergeShared {
     alignas(16) double scratch[THREADS];      // also read as int4
 };
 
-// Writes the per-row outputs of the sample / verify operations.
-__device__ __forceinline__ void emit_row(const KParams &P, const RowCfg &c, int row, int token, float prob,
-                                         uint32_t flags, int support, float p_draft) {
-    if (P.op == OP_SAMPLE) {
-        P.out_token[row] = token;
-        P.out_prob[row] = prob;
-        P.out_flags[row] = flags;
-        if (P.out_support) P.out_support[row] = support;
-    } else {
-        PosResult r;
-        r.token = token; r.flags = flags; r.p = p_draft; r.support = support;
-        P.pr[row] = r;
-    }
-}
-
 #ifdef SONIC_TRACE
-#define MERGE_STAMP(i) do { if (tid == 0 && row == (int)P.error[4]) P.error[8 + (i)] = (unsigned int)clock64(); } while (0)
+#define MERGE_STAMP(i) do { if (tid == 0 && row == (int)P.error[120]) P.error[8 + (i)] = (unsigned int)clock64(); } while (0)
 #else
 #define MERGE_STAMP(i) do { } while (0)
 #endif
 
-#ifdef SONIC_TRACE
-__device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
-#define STREAM_STAMP(i) do { if ((int)blockIdx.x == (int)P.error[5] && lane == 0) P.error[40 + (i)] = gtimer_lo(); } while (0)
-// kernel-level timeline: earliest start and latest end of kernel k (0 stream, 1 merge, 2 exact first launch, 3 exact second launch)
-#define KERNEL_T0(k) do { if (threadIdx.x == 0) atomicMin(&P.error[48 + 2 * (k)], gtimer_lo()); } while (0)
-#define KERNEL_T1(k) do { if (threadIdx.x == 0) atomicMax(&P.error[49 + 2 * (k)], gtimer_lo()); } while (0)
-#else
-#define KERNEL_T0(k) do { } while (0)
-#define KERNEL_T1(k) do { } while (0)
-#define STREAM_STAMP(i) do { } while (0)
-#endif
 constexpr int RANK_SORT_MAX = 512;            // at most this many candidates: sort by rank counting
 constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
 struct WarpSync { __device__ __forceinline__ void operator()() const { __syncwarp(); } };
@@ -135,54 +110,6 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
 template <int THREADS, typename SH>
 __device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells);
 
-// Ranks of at most THREADS distinct non-zero keys held one per thread in list[0, n): every warp sorts its 32 keys
-// with shuffles and writes them back as a descending run, then a key's rank is its place in its own run plus, for
-// every other run, the number of keys there above it (a binary search in the sorted run; 0 pads the last run).
-// Returns the thread's key after the warp sort (0 = padding) and leaves its rank in `rank`.  Two block barriers.
-template <int THREADS, typename Sync>
-__device__ __forceinline__ unsigned long long rank_keys(unsigned long long *list, int n, int tid, int &rank) {
-    Sync csync;
-    const int lane = tid & 31, warp = tid >> 5;
-    unsigned long long key = (tid < n) ? list[tid] : 0ull;
-#pragma unroll
-    for (int kk = 2; kk <= 32; kk <<= 1) {
-#pragma unroll
-        for (int jj = kk >> 1; jj > 0; jj >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
-            const bool up = ((lane & kk) == 0);            // this block of kk sorts descending
-            const bool first = ((lane & jj) == 0);         // the lower lane of the pair
-            const bool take_max = (up == first);
-            key = ((key > o) == take_max) ? key : o;           // mine if it is on the side this lane takes
-        }
-    }
-    csync();                                               // every thread has read its key from the list
-    list[tid] = key;                                       // sorted runs of 32 (descending), in place
-    csync();
-    const int runs = (n + 31) >> 5;
-    rank = lane;
-    if (key != 0ull) {
-        // four runs at a time: their binary searches are independent chains of shared-memory reads
-        for (int r0 = 0; r0 < runs; r0 += 4) {
-            const unsigned long long *run[4];
-            int lo[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { run[u] = list + min(r0 + u, runs - 1) * 32; lo[u] = 0; }
-#pragma unroll
-            for (int step = 16; step > 0; step >>= 1) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (run[u][lo[u] + step - 1] > key) lo[u] += step;
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (lo[u] < 32 && run[u][lo[u]] > key) ++lo[u];        // covers a run whose 32 keys are all above
-                if (r0 + u < runs && r0 + u != warp) rank += lo[u];     // (lo[u] = number of keys of the run above `key`)
-            }
-        }
-    }
-    return key;
-}
-
 // Row merge for top-k class rows (one CTA per row).  buf is MERGE_CAP 64-bit
 // words of shared memory.  Returns false if the candidates cannot prove the
 // row's answer.
@@ -191,7 +118,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                                unsigned long long *buf, MergeShared<THREADS> &sh, int tid, uint2 cells) {
     Sync csync;
     MERGE_STAMP(0);
-    const int cap_t = (int)(CAND_CAP / (unsigned)tiles);
+    const int cap_t = (int)(P.cand_stride / (unsigned)tiles);
     const TileRec *rec = P.tiles + (size_t)row * MAX_TILES;
     // tile records: the first warp takes one tile per lane; prefix of the counts and the largest cutoff by shuffles
     static_assert(MAX_TILES <= 32, "one tile record per lane of the first warp");
@@ -200,7 +127,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         if (tid < tiles) {
             cnt = __ldcg(&rec[tid].cnt);
             tk = __ldcg(&rec[tid].tkey);
-            P.tiles[(size_t)row * MAX_TILES + tid].cnt = 0u;       // the streaming kernel accumulates into it
         }
         const bool over = __any_sync(0xFFFFFFFFu, cnt > (unsigned int)cap_t);     // a tile overflowed its slot
         int incl = (int)cnt;
@@ -242,8 +168,8 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             const int tb = ta + NW;
             const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
             const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
-            const unsigned long long *pa = P.cand + (size_t)row * CAND_CAP + (size_t)ta * cap_t;
-            const unsigned long long *pb = P.cand + (size_t)row * CAND_CAP + (size_t)tb * cap_t;
+            const unsigned long long *pa = P.cand + (size_t)row * P.cand_stride + (size_t)ta * cap_t;
+            const unsigned long long *pb = P.cand + (size_t)row * P.cand_stride + (size_t)tb * cap_t;
             if (max(na, nb) <= 32) {
                 // small k: a tile brings a dozen candidates, one per lane
                 const unsigned long long ca = (lane < na) ? __ldcg(pa + lane) : 0ull;
@@ -323,8 +249,8 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 const int tb = ta + NW;
                 const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
                 const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
-                const unsigned long long *pa = P.cand + (size_t)row * CAND_CAP + (size_t)ta * cap_t;
-                const unsigned long long *pb = P.cand + (size_t)row * CAND_CAP + (size_t)tb * cap_t;
+                const unsigned long long *pa = P.cand + (size_t)row * P.cand_stride + (size_t)ta * cap_t;
+                const unsigned long long *pb = P.cand + (size_t)row * P.cand_stride + (size_t)tb * cap_t;
                 for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
                     unsigned long long cd[GB];
 #pragma unroll
@@ -526,7 +452,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             if (!done) hi = th[0];
             csync();
 #ifdef SONIC_TRACE
-            if (tid == 0 && row == (int)P.error[4]) P.error[28] += 1u;
+            if (tid == 0 && row == (int)P.error[120]) P.error[28] += 1u;
 #endif
         }
         // keep the keys >= lo, packed to the front
@@ -569,7 +495,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     }
     MERGE_STAMP(12);
 #ifdef SONIC_TRACE
-    if (tid == 0 && row == (int)P.error[4]) P.error[29] = Pn2;
+    if (tid == 0 && row == (int)P.error[120]) P.error[29] = Pn2;
 #endif
     const int PnAll = Pn;
     (void)PnAll;
@@ -598,7 +524,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
 #undef Pn
     MERGE_STAMP(3);
 #ifdef SONIC_TRACE
-    if (tid == 0 && row == (int)P.error[4]) { P.error[30] = Pn; P.error[31] = n; }
+    if (tid == 0 && row == (int)P.error[120]) { P.error[30] = Pn; P.error[31] = n; }
 #endif
 
     if (P.op == OP_TOPK) {
@@ -934,6 +860,7 @@ struct StageMeta {
     int npen, nbias;                           // hits of this tile
     int hb;                                    // which hit buffer holds them
     int stop;                                  // no more tiles for this CTA (nothing else in the entry is valid)
+    int bad;                                   // the producer met a list id outside [0, V)
     int next_row, next_tile;                   // the tile that follows (-1: none, or not known yet)
 };
 struct Hit { int li; int payload; };           // element within the tile; history count, or the bias as float bits
@@ -948,6 +875,7 @@ struct StreamShared {
     alignas(16) float tw[NSTAGE][STREAM_WARPS];
     unsigned int ncand[NSTAGE];
     unsigned long long best[NSTAGE][STREAM_WARPS];
+    unsigned int kmin[NSTAGE][STREAM_WARPS], nfin[NSTAGE][STREAM_WARPS];     // dense rows
     // hit lists: one buffer more than stages, so that the producer fills the next tile's while both stages are busy
     Hit pen[NSTAGE + 1][HIT_PEN_CAP];
     Hit bias[NSTAGE + 1][HIT_BIAS_CAP];
@@ -995,7 +923,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
         uint32_t packed[HPL];                      // id | count << 18; 0 = no entry
         int b_id = -1;
         float b_val = 0.0f;
-        int row_patch = 0, cached_row = -1;
+        int row_patch = 0, cached_row = -1, row_bad = 0;
         auto load_row = [&](int row) {
             const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
             const int *hid = P.hist_ids ? P.hist_ids + (size_t)req * P.hist_stride : nullptr;
@@ -1018,6 +946,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             c_next = resolve_cfg(P, row, raw, &memo_k, &memo_G);
             cached_row = row;
             row_patch = 0;
+            row_bad = 0;
             if (c_next.cls == CLS_EXACT || !(c_next.hist_len > 0 || c_next.bias_len > 0)) return;
             row_patch = 2;
             if (c_next.hist_len > FILTER_HIST || c_next.bias_len > FILTER_BIAS) return;
@@ -1047,7 +976,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 if (b0 < 0 || b0 >= P.V) bad = true;
                 else { b_id = b0; b_val = v0; }
             }
-            if (bad) atomicOr(&P.rs[row].status, ST_BADID);
+            row_bad = __any_sync(0xFFFFFFFFu, bad) ? 1 : 0;
             if (__any_sync(0xFFFFFFFFu, big)) return;          // a count too large to pack: consumers scan
             row_patch = 1;
         };
@@ -1136,6 +1065,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             }
             const RowCfg c = c_next;
             const Prep pr = p_next;
+            const int bad_now = row_bad;
             advance();
             const int nxt = current_item();
             __syncwarp();                              // the hit buffer's entries, written by all lanes, precede the arrival
@@ -1144,6 +1074,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 m.cfg = c; m.row = row; m.tile = tile; m.skip = (c.cls == CLS_EXACT) ? 1 : 0;
                 m.patch = pr.patch; m.npen = pr.npen; m.nbias = pr.nbias; m.hb = n % (NSTAGE + 1);
                 m.stop = 0;
+                m.bad = bad_now;
                 m.next_row = (nxt >= 0) ? nxt / tiles : -1;
                 m.next_tile = (nxt >= 0) ? nxt % tiles : -1;
                 if (c.cls == CLS_EXACT) mbar_arrive(&sh.full[s]);      // nothing is copied for rows of the exact class
@@ -1183,10 +1114,30 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             if (pre_row >= 0) mword_pre = load_mask_words(pre_row, pre_tile);
         }
         const StageMeta &meta = sh.meta[s];
-        if (!meta.skip) {
+        if (meta.skip) {
+            // a row of the cluster kernel: counted, its status word initialised
+            if (tile == 0 && tid == 0) { P.rs[row].status = 0u; atomicAdd(&P.error[WS_NEXACT], 1u); }
+        } else {
             const RowCfg c = meta.cfg;
             RowState *rs = P.rs + row;
             TileRec *rec = P.tiles + (size_t)row * MAX_TILES + tile;
+            // Every per-row word of the workspace is initialised by the call that reads it: the tile's flags here
+            // (before any barrier of this tile), the row's status word and, for rows of the histogram path, the
+            // row's control block and its histogram by the CTA of the row's first tile.
+            if (tid == 0) {
+                rec->flags = meta.bad ? TILE_BADID : 0u;
+                if (tile == 0) rs->status = 0u;
+            }
+            if (c.cls == CLS_DENSE && tile == 0) {
+                uint4 *h = reinterpret_cast<uint4 *>(P.hist + (size_t)row * DBINS);
+                for (int i = tid; i < DBINS / 2; i += STREAM_THREADS) h[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (tid == 0) {
+                    DenseRow *dr = P.drow + row;
+                    dr->ticket_h = 0u; dr->ticket_c = 0u; dr->ticket_r = 0u; dr->nmembers = 0u;
+                    dr->kmin = 0xFFFFFFFFu; dr->kmax = 0u; dr->overflow = 0u; dr->state = 0u;
+                    P.dlist[atomicAdd(&P.error[WS_NDENSE], 1u)] = row;
+                }
+            }
             unsigned char *stage = stages + (size_t)s * STAGE_BYTES;
             const bool masked = (c.z & M_GRAMMAR) != 0;
             const bool tail = tile_base + CTA_TILE > P.V;
@@ -1265,7 +1216,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                     const int li = id - tile_base;
                     if (li >= 0 && li < CTA_TILE) ptile[li] = __fadd_rn(ptile[li], __ldg(P.bias_vals + (size_t)req * P.bias_stride + t));
                 }
-                if (bad && tile == 0) atomicOr(&rs->status, ST_BADID);
+                if (bad) atomicOr(&rec->flags, TILE_BADID);          // (ordered after the first thread's store by the barriers above)
                 csync();
                 read_f32(ptile);
             } else {
@@ -1315,7 +1266,32 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             const float h0 = fmaxf(qm[0], qm[1]), h1 = fmaxf(qm[2], qm[3]);
             const float lm = fmaxf(h0, h1);
 
-            if (c.cls == CLS_GREEDY) {
+            if (c.cls == CLS_GREEDY || c.cls == CLS_DENSE) {
+                if (c.cls == CLS_DENSE) {
+                    // histogram path: the processed logits (already divided by the temperature) are kept as ordered
+                    // keys for the later passes; per tile the smallest finite key and the number of finite elements
+                    uint32_t kmn = 0xFFFFFFFFu;
+                    unsigned int nf = 0u;
+                    unsigned int *yk = P.ykeys + (size_t)row * ((size_t)P.ytiles * CTA_TILE) + tile_base + warp * WARP_TILE;
+#pragma unroll
+                    for (int j = 0; j < NV; ++j) {
+#pragma unroll
+                        for (int q4 = 0; q4 < VEC; q4 += 4) {
+                            uint32_t kk[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                kk[u] = okey(e[j * VEC + q4 + u]);
+                                const bool fin = kk[u] > KEY_NEG_INF;
+                                nf += fin ? 1u : 0u;
+                                kmn = fin ? min(kmn, kk[u]) : kmn;
+                            }
+                            *reinterpret_cast<uint4 *>(yk + j * 32 * VEC + lane * VEC + q4) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+                        }
+                    }
+                    kmn = __reduce_min_sync(0xFFFFFFFFu, kmn);
+                    nf = __reduce_add_sync(0xFFFFFFFFu, nf);
+                    if (lane == 0) { sh.kmin[s][warp] = kmn; sh.nfin[s][warp] = nf; }
+                }
                 float wm = lm;
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xFFFFFFFFu, wm, off));
@@ -1346,6 +1322,12 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
 #pragma unroll
                     for (int w = 1; w < STREAM_WARPS; ++w) b = max(b, sh.best[s][w]);
                     rec->best = b;
+                    if (c.cls == CLS_DENSE) {
+                        unsigned int kmn = sh.kmin[s][0], nf = sh.nfin[s][0];
+#pragma unroll
+                        for (int w = 1; w < STREAM_WARPS; ++w) { kmn = min(kmn, sh.kmin[s][w]); nf += sh.nfin[s][w]; }
+                        rec->minkey = kmn; rec->nfin = nf;
+                    }
                 }
             } else {
                 // warp cutoff: minimum over G groups of the group maximum.  Tile cutoff: the largest of the eight
@@ -1371,7 +1353,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 }
                 }
                 if (lane == 0) sh.tw[s][warp] = g;
-                if (tid == 0) sh.ncand[s] = 0;
+                if (tid == 0) { sh.ncand[s] = 0; rec->cnt = 0u; }          // (the warps add to the record after the barrier)
                 csync();
                 static_assert(STREAM_WARPS == 8, "the eight warp cutoffs are read as two 128-bit words");
                 const float4 ta = *reinterpret_cast<const float4 *>(&sh.tw[s][0]);
@@ -1422,7 +1404,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                     }
                     base = __shfl_sync(0xFFFFFFFFu, base, 0);
                     if ((int)base + total <= cap_t) {
-                        unsigned long long *dst = P.cand + (size_t)row * CAND_CAP + (size_t)tile * cap_t + base + (incl - cnt);
+                        unsigned long long *dst = P.cand + (size_t)row * P.cand_stride + (size_t)tile * cap_t + base + (incl - cnt);
                         const int lbase = warp * WARP_TILE + lane * VEC;
                         while (cm) {
                             const int q = __ffs(cm) - 1;
@@ -1450,34 +1432,41 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
 // One CTA per row of the streaming classes: combines the tile records and
 // finishes the row (global top-k, truncation epilogue, token selection, or the
 // per-position verification result).  Rows it cannot prove are flagged for the
-// exact kernel.
-__global__ void __launch_bounds__(MERGE_THREADS)
+// cluster kernel.  The CTAs past the row count run stage 2 of the histogram path
+// (rows with top-k off) beside them.
+__global__ void __launch_bounds__(MERGE_THREADS, 2)
 sonic_merge_kernel(const KParams P, const int tiles) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ MergeShared<MERGE_THREADS> s_merge;
     const int row = blockIdx.x;
     const int tid = threadIdx.x;
-    pdl_launch_dependents();                   // the exact kernel may start on the rows that are its own by class
+    pdl_launch_dependents();                   // the next kernel of the call may start launching; it waits for this grid
     KERNEL_T0(1);
+    if (row >= P.rows) {
+        pdl_wait_primary();
+        dense_stage2(P, tiles, row - P.rows, (int)gridDim.x - P.rows, reinterpret_cast<unsigned long long *>(smem_raw));
+        return;
+    }
     const RowCfg c = load_cfg(P, row);         // inputs only: independent of the streaming kernel
-    if (c.cls == CLS_EXACT && row != 0) return;
+    const bool other = (c.cls == CLS_EXACT || c.cls == CLS_DENSE);
+    if (other && row != 0) return;
     // the row's two uniforms depend on the inputs alone: drawn here, while the streaming kernel may still be running
     uint2 cells = make_uint2(0u, 0u);
     if (P.op != OP_TOPK && c.cls == CLS_TOPK) draw_cells(P, c, cells.x, cells.y);
     pdl_wait_primary();                        // tile records and candidates of the streaming kernel
     if (row == 0 && tid == 0) P.error[WS_QUEUE] = 0u;    // the streaming kernel is done with its work counter
-    if (c.cls == CLS_EXACT) return;
+    if (other) return;
     RowState *rs = P.rs + row;
     const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
-    const unsigned int status = rs->status;
-    if (c.bad || (status & ST_BADID)) {
-        if (tid < tiles) P.tiles[(size_t)row * MAX_TILES + tid].cnt = 0u;      // leave the tile counts clean
-        if (tid == 0) { emit_row(P, c, row, -1, 0.0f, F_BADPARAM, 0, 0.0f); rs->status = 0; }
+    const unsigned int tflags = (tid < tiles) ? __ldcg(&recs[tid].flags) : 0u;
+    const bool badid = __syncthreads_or((int)(tflags & TILE_BADID)) != 0;
+    if (c.bad || badid) {
+        if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_BADPARAM, 0, 0.0f);
         return;
     }
     if (c.cls == CLS_GREEDY) {
         if (tid < 32) {
-            unsigned long long best = (tid < tiles) ? recs[tid].best : 0ull;
+            unsigned long long best = (tid < tiles) ? __ldcg(&recs[tid].best) : 0ull;
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
             if (tid == 0) {

@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def sonic():
-    from paper_2607_20475_b200 import binding
+    from paper_2607_20475_b200 import harness as binding
     binding.lib()
     return binding
 

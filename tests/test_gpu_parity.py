@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def sonic():
-    from paper_2607_20475_b200 import binding
+    from paper_2607_20475_b200 import harness as binding
     binding.lib()
     return binding
 
@@ -74,7 +74,7 @@ def test_topk_config5_full(sonic, oracle, regime):
     tw = wl.config5(regime)
     x = tw.logits_f32()
     rv, ri = oracle.topk(x, 4096)
-    ws = sonic.new_workspace(tw.B)
+    ws = sonic.new_workspace(tw.B, tw.V)
     for k in wl.TOPK_KS:
         dev = sonic.DeviceTopK(tw, k, ws=ws)
         dev.run()

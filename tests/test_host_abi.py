@@ -36,10 +36,16 @@ def test_struct_layout_matches_header_field_count():
     assert C.sizeof(binding.SampleArgs) == 8 * 28 + 8      # 30 fields, natural alignment on LP64
 
 
-def test_workspace_size_is_monotone_and_per_row():
-    b1, b2, b64 = (binding.sonic_workspace_bytes(n) for n in (1, 2, 64))
-    assert b2 - b1 == (b64 - b1) // 63 and b1 > 256 * 1024 and b64 < 64 * 300 * 1024
-    assert binding.sonic_workspace_bytes(0) == b1
+def test_workspace_size_grows_with_rows_and_vocabulary():
+    V = binding.MAX_VOCAB
+    b1, b2, b64 = (binding.sonic_workspace_bytes(n, V) for n in (1, 2, 64))
+    assert b1 < b2 < b64 and b64 < 64 * 1400 * 1024          # about 1.3 MB per row at the largest vocabulary
+    assert b2 - b1 > 1024 * 1024
+    assert binding.sonic_workspace_bytes(0, V) == b1
+    small = binding.sonic_workspace_bytes(64, 32768)
+    assert small < b64 // 3                                    # a V = 32768 caller does not pay for V = 262144
+    sizes = [binding.sonic_workspace_bytes(64, v) for v in (1, 8192, 8193, 100000, 131072, 262144)]
+    assert sizes == sorted(sizes) and sizes[0] == sizes[1] < sizes[2]
 
 
 def test_bad_arguments_are_rejected_on_the_host():

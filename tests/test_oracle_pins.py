@@ -388,3 +388,147 @@ def test_verify_zero_probability_draft_is_rejected():
     out = oracle.verify(vw)
     assert out["accept_len"].tolist() == [0] * 50 and out["tokens"][:, 0].tolist() == [2] * 50
     assert np.all(out["p_draft"] == 0)
+
+
+# ------------------------------------------ positions, bonus draw, margins, end-to-end tokens
+def _index_order_pick(ids, probs, u):
+    """Closed form of the draw over a hand-worked support: ids ascending with their probabilities;
+    the first id whose cumulative probability exceeds u (probabilities sum to 1)."""
+    F = 0.0
+    for i, p in zip(ids, probs):
+        F += p
+        if F > u:
+            return i
+    return ids[-1]
+
+
+def test_verify_positions_use_offset_plus_l_and_bonus_uses_the_draw_word():
+    # K = 2, V = 3, the same p and q at every position.  p = (.5,.3,.2), q = (.2,.5,.3), hand-worked:
+    # draft 0 always accepted, draft 1 iff u_acc <= .6, draft 2 iff u_acc <= 2/3; the residual is (1,0,0), so a
+    # rejection emits token 0; the bonus token (both accepted) is the index-order draw from p with the DRAW word of
+    # position 2: token 0 if u_draw < .5, 1 if < .8, else 2.  Position l of request b uses the Philox counter
+    # offset + l (word 0 accept, word 1 draw): predicted here from the second Philox implementation.
+    p = np.array([0.5, 0.3, 0.2])
+    q = np.array([0.2, 0.5, 0.3])
+    pf = softmax(np.log(p).astype(np.float32).astype(np.float64))
+    qf = q.astype(np.float32).astype(np.float64)
+    B, K, seed = 4000, 2, 21
+    rng = np.random.default_rng(8)
+    drafts = rng.integers(0, 3, size=(B, K))
+    offset = rng.integers(0, 2 ** 40, size=B).astype(np.uint64)
+    vw = _verify_workload(np.tile(p, (B, K + 1, 1)), np.tile(q, (B, K, 1)), drafts, np.zeros(B), seed=seed, offset=offset)
+    out = oracle.verify(vw)
+    n_bonus = n_second = 0
+    for b in range(B):
+        expect, acc, near = [], 0, False
+        for l in range(K + 1):
+            ua, ud = py_uniforms(seed, int(offset[b]) + l, b)
+            if l < K:
+                d = int(drafts[b, l])
+                lhs = ua * qf[d]
+                near |= abs(lhs - pf[d]) < 1e-7
+                if lhs <= pf[d]:
+                    expect.append(d); acc += 1
+                    continue
+                expect.append(0)                                   # residual (1, 0, 0)
+                break
+            near |= min(abs(ud - pf[0]), abs(ud - pf[0] - pf[1])) < 1e-7
+            expect.append(_index_order_pick([0, 1, 2], pf, ud))   # bonus token from position K
+        if near:
+            continue
+        expect += [-1] * (K + 1 - len(expect))
+        assert out["tokens"][b].tolist() == expect, (b, out["tokens"][b], expect)
+        assert out["accept_len"][b] == acc
+        n_bonus += acc == K
+        n_second += acc >= 1
+    assert n_bonus > 300 and n_second > 1500                      # positions 1 and 2 were really exercised
+    # using the position-0 counter for every position, or the accept word for the bonus draw, gives other tokens
+    b = next(b for b in range(B) if out["accept_len"][b] == K
+             and _index_order_pick([0, 1, 2], pf, py_uniforms(seed, int(offset[b]) + K, b)[0]) != out["tokens"][b, K])
+    assert out["tokens"][b, K] == _index_order_pick([0, 1, 2], pf, py_uniforms(seed, int(offset[b]) + K, b)[1])
+
+
+def test_end_to_end_tokens_of_the_hand_worked_rows():
+    # Row A: x8 with top-k 5, top-p 0.9, min-p 0.3 -> support {1, 7, 2, 3}, probabilities
+    # (.426933, .258948, .157060, .157060); index-order CDF over ids 1, 2, 3, 7 = (.426933, .583992, .741052, 1).
+    # Row B: mask + penalties + bias + tau 0.7, k 4, p .95, theta .05 -> support {6, 7, 3, 1}; index-order CDF over
+    # ids 1, 3, 6, 7 = (.075877, .230872, .683387, 1).  (seed, offset, row) = (0, 0, 0) draws
+    # u = ((0xe169c58d >> 8) + .5) / 2^24 = 0.88052019 from the second Philox word: token 7 in both rows.
+    u = ((0xE169C58D >> 8) + 0.5) / 2 ** 24
+    assert py_uniforms(0, 0, 0)[1] == u
+    wa = make_sample(X8, [wl.TOP_K | wl.TOP_P | wl.MIN_P], top_k=[5], top_p=[0.9], min_p=[0.3])
+    out = oracle.sample(wa)
+    assert out["token"].tolist() == [7] and out["support"].tolist() == [4]
+    assert abs(out["prob"][0] - 0.258948) < 1e-6
+    mode = (wl.GRAMMAR | wl.REPETITION | wl.FREQUENCY | wl.PRESENCE | wl.BIAS | wl.TEMPERATURE
+            | wl.TOP_K | wl.TOP_P | wl.MIN_P)
+    allowed = np.array([[0, 1, 1, 1, 1, 0, 1, 1]], dtype=bool)
+    wb = make_sample(X8, [mode], rep=[1.25], freq=[0.5], pres=[0.25], temperature=[0.7], top_k=[4],
+                     top_p=[0.95], min_p=[0.05], hist=[{2: 2, 5: 1}], bias=[{1: -1.5, 6: 2.25}],
+                     bitmask=pack_bits(allowed))
+    out = oracle.sample(wb)
+    assert out["token"].tolist() == [7] and out["support"].tolist() == [4]
+    assert abs(out["prob"][0] - 0.316613) < 1e-6
+    # other offsets walk the same hand-worked CDFs
+    cdf_a = ([1, 2, 3, 7], [0.426933, 0.157060, 0.157060, 0.258948])
+    cdf_b = ([1, 3, 6, 7], [0.075877, 0.154995, 0.452516, 0.316613])
+    for off in range(1, 60):
+        u = py_uniforms(0, off, 0)[1]
+        for w, (ids, pr) in ((wa, cdf_a), (wb, cdf_b)):
+            edges = np.cumsum(pr)
+            if np.min(np.abs(edges - u)) < 1e-5:
+                continue
+            w.offset[:] = off
+            assert oracle.sample(w)["token"][0] == _index_order_pick(ids, pr, u)
+
+
+def test_margins_of_the_hand_worked_rows():
+    # top-p 0.9 on x8: the cumulative fractions around the cut are .891346 (4 tokens) and .942847 (5 tokens), so the
+    # cut's margin is min(|.942847 - .9|, |.891346 - .9|) = .008654; the row's margin is the smaller of that and
+    # the draw's distance to the nearer edge of its CDF step (index-order CDF over ids 0, 1, 2, 3, 7 =
+    # .054623, .458235, .606716, .755197, 1).
+    z = 1 + math.exp(-0.5) + 2 * math.exp(-1) + math.exp(-2) + math.exp(-2.5) + math.exp(-3) + math.exp(-4)
+    c4 = (1 + math.exp(-0.5) + 2 * math.exp(-1)) / z
+    c5 = c4 + math.exp(-2) / z
+    p32 = float(np.float32(0.9))
+    cut_margin = min(abs(c5 - p32), abs(c4 - p32))
+    assert abs(cut_margin - 0.008654) < 2e-6
+    edges = np.cumsum(np.array([math.exp(-2), 1, math.exp(-1), math.exp(-1), math.exp(-0.5)]) / (c5 * z))
+    w = make_sample(X8, [wl.TOP_P], top_p=[0.9])
+    seen_draw = seen_cut = 0
+    for off in range(200):
+        w.offset[:] = off
+        u = py_uniforms(0, off, 0)[1]
+        j = int(np.searchsorted(edges, u, side="right"))
+        lo = edges[j - 1] if j > 0 else 0.0
+        draw_margin = min(abs(edges[min(j, 4)] - u), abs(lo - u))
+        got = oracle.sample(w)["margin"][0]
+        assert abs(got - min(cut_margin, draw_margin)) < 1e-9, (off, got, cut_margin, draw_margin)
+        seen_draw += draw_margin < cut_margin
+        seen_cut += draw_margin >= cut_margin
+    assert seen_draw > 0 and seen_cut > 0
+    # min-p 0.3 on x8: threshold 3 + ln(0.3) = 1.796027; the entries next to the cut are 2.0 and 1.0
+    w = make_sample(X8, [wl.MIN_P], min_p=[0.3])
+    _, _, m = oracle.support(w, 0)
+    thr = 3 + math.log(float(np.float32(0.3)))
+    assert abs(m - min(2.0 - thr, thr - 1.0)) < 1e-12
+    # verification: the accept test's margin |u q - p| / max(u q, p), draft 1 of p = (.5,.3,.2), q = (.2,.5,.3)
+    p, q = np.array([0.5, 0.3, 0.2]), np.array([0.2, 0.5, 0.3])
+    pf = softmax(np.log(p).astype(np.float32).astype(np.float64))
+    qf = q.astype(np.float32).astype(np.float64)
+    B = 64
+    vw = _verify_workload(np.tile(p, (B, 2, 1)), np.tile(q, (B, 1, 1)), np.ones(B), np.zeros(B), seed=9)
+    out = oracle.verify(vw)
+    for b in range(B):
+        ua, ud = py_uniforms(9, 0, b)
+        lhs = ua * qf[1]
+        acc_margin = abs(lhs - pf[1]) / max(lhs, pf[1])
+        if lhs <= pf[1]:
+            # accepted: the bonus token's draw margin joins in (CDF .5, .8, 1 with position 1's draw word)
+            ud1 = py_uniforms(9, 1, b)[1]
+            e = np.array([0.0, pf[0], pf[0] + pf[1], 1.0])
+            j = int(np.searchsorted(e, ud1, side="right"))
+            expect = min(acc_margin, abs(e[min(j, 3)] - ud1), abs(e[j - 1] - ud1))
+        else:
+            expect = min(acc_margin, min(abs(1.0 - ud), abs(0.0 - ud)))      # residual (1, 0, 0): one step from 0 to 1
+        assert abs(out["margin"][b] - expect) < 1e-7, (b, out["margin"][b], expect)

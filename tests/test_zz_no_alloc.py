@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 def test_static_scratch_topk_matches_workspace_topk_twice():
     import torch
-    from paper_2607_20475_b200 import binding
+    from paper_2607_20475_b200 import harness as binding
 
     binding.lib()
     B, V = binding.STATIC_MAX_ROWS, 70001
@@ -33,7 +33,7 @@ def test_static_scratch_topk_matches_workspace_topk_twice():
 
 def test_static_scratch_rejects_more_rows_than_it_holds():
     import torch
-    from paper_2607_20475_b200 import binding
+    from paper_2607_20475_b200 import harness as binding
 
     B, V, k = binding.STATIC_MAX_ROWS + 1, 4096, 4
     x = torch.zeros((B, V), dtype=torch.float32, device="cuda")
