@@ -100,7 +100,7 @@ static Layout layout_for(long long rows, int V, bool dense) {
 
 static int g_sm_count[64];
 
-static int configure_once(int *sm_count) {
+static int configure_once(int *sm_count, int *device) {
     static std::once_flag once[64];
     static cudaError_t result[64];
     static int clusters[64];
@@ -115,6 +115,8 @@ static int configure_once(int *sm_count) {
         };
         set((const void *)sonic_merge_kernel, MERGE_SMEM);
         set((const void *)sonic_dense_collect_kernel, DENSE_DYN_SMEM);
+        set((const void *)sonic_dense_stage2_kernel, DENSE_DYN_SMEM);
+        set((const void *)sonic_dense_finish_kernel, DENSE_DYN_SMEM);
         set((const void *)sonic_stream_kernel<0>, STREAM_SMEM_F32);
         set((const void *)sonic_stream_kernel<1>, STREAM_SMEM_BF16);
         if (r == cudaSuccess) r = cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
@@ -140,22 +142,65 @@ static int configure_once(int *sm_count) {
     if (result[dev] != cudaSuccess) return fail_cuda(result[dev], "kernel configuration");
     if (clusters[dev] < 1) return fail(SONIC_ECUDA, "no 8-CTA cluster of the cluster kernel fits on this device");
     *sm_count = g_sm_count[dev] > 0 ? g_sm_count[dev] : 1;
+    *device = dev;
     return SONIC_OK;
 }
 
-// One call = a chain of kernels on the caller's stream, each a programmatic dependent of the one before (it may
-// begin launching while its predecessor runs and waits for it inside the kernel; the paper overlaps its two stages
-// the same way, Section 3.5):
-//   stream kernel -> merge kernel (+ stage 2 of the histogram path) -> [collect pass] -> [residual pass]
-//   -> cluster kernel (rows no other path finished; usually none) -> [verification scan]
+// Per host thread and device: one internal stream and two events, so that the histogram passes (rows with top-k off)
+// run beside the merges (rows with top-k) instead of behind them.  A call forks the stream from the caller's after
+// the streaming kernel and joins it before the call's last kernel; under stream capture it is captured with the
+// caller's stream.  Created by the thread's first call on a device outside a capture; whenever the stream cannot
+// be used safely (not created yet and the caller is capturing; still part of another, open capture) the call runs all
+// of its kernels on the caller's stream instead, with the same results.
+struct SideStream {
+    cudaStream_t s = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool tried = false, ok = false;
+    ~SideStream() {
+        if (join) cudaEventDestroy(join);
+        if (fork) cudaEventDestroy(fork);
+        if (s) cudaStreamDestroy(s);
+    }
+};
+static thread_local SideStream g_side[64];
+
+static SideStream *side_stream_for(int dev, cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone, ss = cudaStreamCaptureStatusNone;
+    unsigned long long cid = 0, sid = 0;
+    if (cudaStreamGetCaptureInfo(st, &cs, &cid) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (cs == cudaStreamCaptureStatusInvalidated) return nullptr;
+    SideStream &S = g_side[dev];
+    if (!S.tried) {
+        if (cs != cudaStreamCaptureStatusNone) return nullptr;          // (nothing is created while a capture is open)
+        S.tried = true;
+        S.ok = cudaStreamCreateWithFlags(&S.s, cudaStreamNonBlocking) == cudaSuccess &&
+               cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&S.join, cudaEventDisableTiming) == cudaSuccess;
+        if (!S.ok) cudaGetLastError();
+    }
+    if (!S.ok) return nullptr;
+    if (cudaStreamGetCaptureInfo(S.s, &ss, &sid) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (ss == cudaStreamCaptureStatusInvalidated) return nullptr;
+    if (ss == cudaStreamCaptureStatusActive && !(cs == cudaStreamCaptureStatusActive && cid == sid)) return nullptr;   // busy in another capture
+    return &S;
+}
+
+// One call = a chain of kernels on the caller's stream.  Up to the residual pass each is a programmatic dependent
+// of the one before (it may begin launching while its predecessor runs; the paper overlaps its two stages the
+// same way, Section 3.5):
+//   stream kernel -> merge kernel (rows with top-k)
+//                 \-> [histogram pass -> its row step -> collect pass -> its row step -> residual pass]   (rows with top-k off)
+//   -> cluster kernel (an ordinary launch after all of it: rows no other path finished; usually none) -> [verification scan]
+// The second line runs on the thread's internal stream beside the merges when that stream can be used, else behind
+// them on the caller's stream.
 static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, int B_requests) {
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
     const bool dense = (P.op != OP_TOPK);
     const Layout L = layout_for(P.rows, P.V, dense);
     if (ws_bytes < L.total) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows of this vocabulary size");
-    int sm_count = 1;
-    int rc = configure_once(&sm_count);
+    int sm_count = 1, dev = 0;
+    int rc = configure_once(&sm_count, &dev);
     if (rc != SONIC_OK) return rc;
     unsigned char *base = reinterpret_cast<unsigned char *>(ws);
     P.error = reinterpret_cast<unsigned int *>(base);
@@ -199,30 +244,63 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     cfg.stream = st;
     cfg.attrs = &pdl;
     cfg.numAttrs = 1;
-    // the passes of the histogram path take (row, tile) items in a loop: two CTAs per SM at most
-    // (a tile is cut into up to four parts when a call has few rows of that class: up to four CTAs per tile)
-    const int dense_ctas = dense ? (int)(4ll * nitems < 2ll * sm_count ? 4ll * nitems : 2ll * sm_count) : 0;
-    cfg.gridDim = dim3(P.rows + dense_ctas);
+    // Fork: the histogram passes go to the thread's internal stream (if it can be used), behind the streaming
+    // kernel and beside the merges.  After the fork every exit joins that stream again (also the failing ones: the
+    // caller's stream, or its capture, must not be left with a branch that was never joined).
+    SideStream *side = dense ? side_stream_for(dev, st) : nullptr;
+    if (side) {
+        if ((e = cudaEventRecord(side->fork, st)) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+        if ((e = cudaStreamWaitEvent(side->s, side->fork, 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
+    }
+    auto unwind = [&](int code) {
+        if (side && cudaEventRecord(side->join, side->s) == cudaSuccess) cudaStreamWaitEvent(st, side->join, 0);
+        return code;
+    };
+    cfg.gridDim = dim3(P.rows);
     cfg.blockDim = dim3(MERGE_THREADS);
     cfg.dynamicSmemBytes = MERGE_SMEM;
     e = cudaLaunchKernelEx(&cfg, sonic_merge_kernel, P, tiles);
-    if (e != cudaSuccess) return fail_cuda(e, "merge kernel launch");
+    if (e != cudaSuccess) return unwind(fail_cuda(e, "merge kernel launch"));
     if (dense) {
-        cfg.gridDim = dim3(dense_ctas);
-        cfg.blockDim = dim3(DENSE_THREADS);
-        cfg.dynamicSmemBytes = DENSE_DYN_SMEM;
-        e = cudaLaunchKernelEx(&cfg, sonic_dense_collect_kernel, P, tiles);
-        if (e != cudaSuccess) return fail_cuda(e, "collect pass launch");
+        // the passes of the histogram path take (row, tile part) items in a loop: two CTAs per SM at most (a tile is
+        // cut into up to four parts when a call has few rows of that class: up to four CTAs per tile)
+        const int dense_ctas = (int)(4ll * nitems < 2ll * sm_count ? 4ll * nitems : 2ll * sm_count);
+        cudaLaunchConfig_t dcfg = cfg;
+        dcfg.stream = side ? side->s : st;
+        dcfg.gridDim = dim3(dense_ctas);
+        dcfg.blockDim = dim3(DENSE_THREADS);
+        dcfg.dynamicSmemBytes = DENSE_DYN_SMEM;
+        cudaLaunchConfig_t fcfg = dcfg;              // row-level steps: one CTA per row, one per SM at most
+        fcfg.gridDim = dim3(P.rows < sm_count ? P.rows : sm_count);
+        // Stage 2 never waits for its predecessor in the stream.  On the internal stream it is an ordinary launch
+        // behind the fork; on the caller's stream it is a programmatic dependent of the merge kernel, whose CTAs let
+        // it go only after their own wait for the streaming kernel.
+        cudaLaunchConfig_t d2cfg = dcfg;
+        if (side) { d2cfg.attrs = nullptr; d2cfg.numAttrs = 0; }
+        e = cudaLaunchKernelEx(&d2cfg, sonic_dense_stage2_kernel, P, tiles);
+        if (e != cudaSuccess) return unwind(fail_cuda(e, "histogram pass launch"));
+        e = cudaLaunchKernelEx(&dcfg, sonic_dense_collect_kernel, P, tiles);
+        if (e != cudaSuccess) return unwind(fail_cuda(e, "collect pass launch"));
+        e = cudaLaunchKernelEx(&fcfg, sonic_dense_finish_kernel, P, tiles);
+        if (e != cudaSuccess) return unwind(fail_cuda(e, "row finish launch"));
         if (P.op == OP_VERIFY && P.K > 0) {
-            cfg.dynamicSmemBytes = 0;
-            e = cudaLaunchKernelEx(&cfg, sonic_dense_resid_kernel, P, tiles);
-            if (e != cudaSuccess) return fail_cuda(e, "residual pass launch");
+            dcfg.dynamicSmemBytes = 0;
+            e = cudaLaunchKernelEx(&dcfg, sonic_dense_resid_kernel, P, tiles);
+            if (e != cudaSuccess) return unwind(fail_cuda(e, "residual pass launch"));
         }
     }
+    if (side) {
+        if ((e = cudaEventRecord(side->join, side->s)) != cudaSuccess) return fail_cuda(e, "cudaEventRecord");
+        if ((e = cudaStreamWaitEvent(st, side->join, 0)) != cudaSuccess) return fail_cuda(e, "cudaStreamWaitEvent");
+    }
+    // The cluster kernel is an ordinary launch: it starts when everything before it is complete (the merges as well
+    // as the histogram passes, which ran beside them).
     const int clusters = P.rows < EXACT_CLUSTERS ? P.rows : EXACT_CLUSTERS;
     cfg.gridDim = dim3(clusters * CL);
     cfg.blockDim = dim3(EX_THREADS);
     cfg.dynamicSmemBytes = EXACT_SMEM;
+    cfg.attrs = nullptr;
+    cfg.numAttrs = 0;
     if (P.dtype == SONIC_DTYPE_F32) e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<0>, P);
     else e = cudaLaunchKernelEx(&cfg, sonic_exact_kernel<1>, P);
     if (e != cudaSuccess) return fail_cuda(e, "cluster kernel launch");

@@ -186,18 +186,32 @@ __device__ __forceinline__ void dense_load_keys(const KParams &P, const DenseIte
     for (int k = 0; k < DENSE_NV; ++k) kv[k] = (k < nv) ? src[k] : make_uint4(KEY_NEG_INF, KEY_NEG_INF, KEY_NEG_INF, KEY_NEG_INF);
 }
 
-// Ticket of a pass: true in every thread of the row's last CTA to arrive (whose reads then see what the others wrote).
-__device__ __forceinline__ bool dense_arrive(unsigned int *ticket, int items, DenseShared &sm, int tid) {
+// Ticket of a pass: a CTA reports `cnt` finished items of a row at once; true in every thread of the CTA whose report
+// completes the row's `items` (its reads then see what the others wrote).
+__device__ __forceinline__ bool dense_arrive(unsigned int *ticket, int cnt, int items, DenseShared &sm, int tid) {
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned int t = atomicAdd(ticket, 1u);
-        sm.last = (t == (unsigned int)(items - 1)) ? 1 : 0;
+        const unsigned int t = atomicAdd(ticket, (unsigned int)cnt);
+        sm.last = (t + (unsigned int)cnt == (unsigned int)items) ? 1 : 0;
         if (sm.last) __threadfence();
     }
     __syncthreads();
     return sm.last != 0;
 }
+
+// The items of a pass are dealt in contiguous ranges, so that a CTA's items mostly belong to one row: the row's
+// parameters are loaded once, its ticket is drawn once, and the rows a CTA turns out to complete are finished after
+// all of its items (another row's items never wait behind a finish).
+struct DenseRange { int lo, hi; };
+__device__ __forceinline__ DenseRange dense_range(int n_items, int cta, int ncta) {
+    const int per = (n_items + ncta - 1) / ncta;
+    DenseRange r;
+    r.lo = min(n_items, cta * per);
+    r.hi = min(n_items, r.lo + per);
+    return r;
+}
+constexpr int DENSE_FIN_MAX = 8;              // rows one CTA can have to finish (a range spans few rows)
 
 // ---------------------------------------------------------------- pass H
 // Mass histogram of one item, added to the row's histogram in global memory.
@@ -238,11 +252,14 @@ __device__ __forceinline__ void dense_hist_item(const KParams &P, const DenseIte
     }
 }
 
-// Last arriver of pass H: the crossing bin of top-p against the min-p threshold, as the key interval pass C works with.
-__device__ __forceinline__ void dense_hist_finish(const KParams &P, const RowCfg &c, int row, DenseShared &sm,
-                                                  unsigned long long *h, int tid, uint32_t Mkey, float scale) {
+// Row step of pass H: the crossing bin of top-p against the min-p threshold, as the key interval pass C works with
+// (in every thread: klo, khi, tk, target).  Every CTA of pass C that meets the row computes it for itself from the
+// row's histogram (16 KB, one round of loads); `store` (the CTA of the row's first item) leaves it for the row's finish.
+struct DenseCut { uint32_t tk, klo, khi; unsigned long long target; };
+__device__ __forceinline__ DenseCut dense_hist_finish(const KParams &P, const RowCfg &c, int row, DenseShared &sm,
+                                                      unsigned long long *h, int tid, uint32_t Mkey, float scale, bool store) {
     const unsigned long long *hist = P.hist + (size_t)row * DBINS;
-    for (int i = tid; i < DBINS; i += DENSE_THREADS) h[i] = __ldcg(&hist[i]);
+    for (int i = tid; i < DBINS; i += DENSE_THREADS) h[i] = hist[i];
     __syncthreads();
     // thread t owns bins DBINS-1-4t .. DBINS-4-4t (from the top)
     constexpr int BPT = DBINS / DENSE_THREADS;
@@ -268,27 +285,34 @@ __device__ __forceinline__ void dense_hist_finish(const KParams &P, const RowCfg
         sm.digit = found;
     }
     __syncthreads();
-    if (tid < 32) {
+    if (tid < 64) {
+        // two warps: the lower key of the bin, and the lower key of the bin above it
         const float Mf = unkey(Mkey);
         const int b_p = sm.digit;
         uint32_t tk = 0u;
         int b_m = -1;
         if (c.z & M_MIN_P) { tk = minp_key(Mf, c.theta); b_m = dense_digit(max(tk, KEY_NEG_INF + 1u), Mf, scale); }
-        uint32_t klo, khi;
         if (b_m > b_p) {
             // the min-p threshold lies above the bin top-p would cut in: the cut is the threshold itself
-            klo = 0xFFFFFFFFu; khi = tk - 1u; target = 0ull;
+            if (tid == 0) { sm.bc64[0] = ((unsigned long long)0xFFFFFFFFu << 32) | (tk - 1u); sm.bc64[1] = 0ull; sm.base = tk; }
         } else {
-            klo = dense_bin_lower_key(b_p, Mkey, Mf, scale, tid);
-            khi = dense_bin_lower_key(b_p + 1, Mkey, Mf, scale, tid) - 1u;
-        }
-        if (tid == 0) {
-            DenseRow *dr = P.drow + row;
-            dr->Mkey = Mkey; dr->tk = tk; dr->klo = klo; dr->khi = khi; dr->target = target;
-            __threadfence();
-            dr->state = 1u;
+            const uint32_t k = dense_bin_lower_key(b_p + (tid >> 5), Mkey, Mf, scale, tid & 31);
+            if (tid == 32) sm.kmax = k - 1u;                    // khi
+            if (tid == 0) { sm.kmin = k; sm.bc64[1] = target; sm.base = tk; }     // klo
         }
     }
+    __syncthreads();
+    DenseCut r;
+    if (sm.bc64[1] == 0ull) { r.klo = (uint32_t)(sm.bc64[0] >> 32); r.khi = (uint32_t)sm.bc64[0]; }
+    else { r.klo = sm.kmin; r.khi = sm.kmax; }
+    r.tk = sm.base; r.target = sm.bc64[1];
+    __syncthreads();
+    if (store && tid == 0) {
+        DenseRow *dr = P.drow + row;
+        dr->Mkey = Mkey; dr->tk = r.tk; dr->klo = r.klo; dr->khi = r.khi; dr->target = r.target;
+        dr->state = 1u;
+    }
+    return r;
 }
 
 // ---------------------------------------------------------------- in-tile search
@@ -782,93 +806,143 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
     return true;
 }
 
-// Pass C for one item whose cut parameters are known; the row's last CTA finishes it.
-__device__ __forceinline__ void dense_collect_item(const KParams &P, const RowCfg &c, const DenseItem &it, int tiles, const uint4 (&kv)[DENSE_NV],
-                                                   uint32_t Mkey, uint32_t klo, uint32_t khi, unsigned long long target, uint32_t tk,
-                                                   DenseShared &sm, unsigned long long *dyn, int tid) {
-    uint2 cells = make_uint2(0u, 0u);
-    draw_cells(P, c, cells.x, cells.y);           // (inputs only: off the chain that follows the ticket)
-    if (cells.x == 0x7fffffffu) return;
-    DSTAMP(40);
-#ifdef SONIC_DTRACE2
-    if (it.tile == 0 && it.part == 0) { dense_collect_part(P, it, kv, unkey(Mkey), 0xFFFFFFFFu, khi, sm, dyn, tid); __syncthreads(); }
-#endif
-    dense_collect_part(P, it, kv, unkey(Mkey), klo, khi, sm, dyn, tid);
-    DSTAMP(2);
-    if (!dense_arrive(&P.drow[it.row].ticket_c, tiles * it.sub, sm, tid)) return;
-    const bool ok = dense_finish(P, c, it.row, tiles, sm, dyn, tid, Mkey, klo <= khi, target, tk, cells);
-    if (!ok && tid == 0) { P.rs[it.row].status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
+// Row-level parameters of a pass, derived by every CTA that needs them from what the earlier kernels left.
+struct DenseRowPar {
+    int kind;                                  // 0 nothing to do, 1 histogram items (pass H), 2 collect items (pass C)
+    uint32_t Mkey, tk, klo, khi;
+    unsigned long long target;
+    float scale;
+};
+
+// What the streaming kernel left about a row, and what follows from it for the stage at hand.
+//   stage 2: top-p rows take pass H; the others know their cut from the row maximum (min-p: the elements at or
+//            above the threshold key; neither: every finite element - no bin, no list) and take pass C at once;
+//   stage 3: top-p rows take pass C with the crossing bin found from the row's histogram (computed here, by every
+//            CTA that meets the row; dyn holds the bins meanwhile);
+//   stage 4 (the row's finish): top-p rows read what stage 3 stored, the others are as in stage 2.
+// `first` marks the one CTA that speaks for the row (emits the rows without a token in stage 2, stores the cut in stage 3).
+__device__ __forceinline__ DenseRowPar dense_row_par(const KParams &P, int row, int tiles, DenseShared &sm, unsigned long long *dyn, int tid,
+                                                     const int stage, const bool first, RowCfg &c) {
+    DenseRowPar r;
+    r.kind = 0; r.tk = 0u; r.klo = 0u; r.khi = 0u; r.target = 0ull; r.scale = 0.0f;
+    const CfgRaw raw = fetch_cfg(P, row);
+    const DenseRow *dr = P.drow + row;
+    uint32_t s_tk = 0u, s_klo = 0u, s_khi = 0u, s_state = 0u;
+    unsigned long long s_target = 0ull;
+    if (stage == 4) { s_state = __ldcg(&dr->state); s_tk = __ldcg(&dr->tk); s_klo = __ldcg(&dr->klo); s_khi = __ldcg(&dr->khi); s_target = __ldcg(&dr->target); }
+    dense_row_stats(P, row, tiles, sm, tid);
+    __syncthreads();
+    r.Mkey = sm.Mkey;
+    const uint32_t mkey = sm.mkey;
+    const unsigned int Nf = sm.Nf;
+    bool bad = sm.bad != 0u;
+    __syncthreads();
+    c = resolve_cfg(P, row, raw);
+    bad = bad || c.bad;
+    if (bad || Nf == 0u) {
+        if (stage == 2 && first && tid == 0) emit_row(P, c, row, -1, 0.0f, (bad ? F_BADPARAM : F_NO_TOKEN) | F_DENSE, 0, 0.0f);
+    } else if (c.z & M_TOP_P) {
+        if (stage == 2) {
+            r.kind = 1; r.scale = dense_scale(r.Mkey, mkey, Nf);
+        } else if (stage == 3) {
+            const DenseCut cut = dense_hist_finish(P, c, row, sm, dyn, tid, r.Mkey, dense_scale(r.Mkey, mkey, Nf), first);
+            r.kind = 2; r.tk = cut.tk; r.klo = cut.klo; r.khi = cut.khi; r.target = cut.target;
+        } else if (s_state == 1u) {
+            r.kind = 2; r.tk = s_tk; r.klo = s_klo; r.khi = s_khi; r.target = s_target;
+        }
+    } else if (stage != 3) {
+        r.kind = 2;
+        r.tk = (c.z & M_MIN_P) ? minp_key(unkey(r.Mkey), c.theta) : 0u;
+        r.klo = 0xFFFFFFFFu; r.khi = r.tk ? r.tk - 1u : KEY_NEG_INF;
+    }
+    return r;
 }
 
-// Stage 2 of the histogram path, run by the extra CTAs of the merge kernel's launch: pass H for rows with top-p,
-// pass C (and the row's finish) for the others, whose cut is a key threshold known from the row maximum.
-__device__ void dense_stage2(const KParams &P, int tiles, int cta, int ncta, unsigned long long *dyn) {
-    __shared__ DenseShared sm;
+// The item loop of stages 2 and 3: the (row, tile part) items of the call's rows of this class are dealt in
+// contiguous ranges, so that a CTA's items mostly belong to one row whose parameters it derives once.  No CTA waits
+// for another: the rows are finished in the kernel that follows (sonic_dense_finish_kernel).
+__device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta, int ncta, unsigned long long *dyn, DenseShared &sm, const int stage) {
     const int tid = threadIdx.x;
     const int nd = (int)__ldcg(&P.error[WS_NDENSE]);
     const int sub = dense_pick_sub(nd, tiles, ncta);
-    for (int item = cta; item < nd * tiles * sub; item += ncta) {
+    const int per_row = tiles * sub;
+    const DenseRange rg = dense_range(nd * per_row, cta, ncta);
+    int cur_row = -1;
+    DenseRowPar par;
+    par.kind = 0;
+    for (int item = rg.lo; item < rg.hi; ++item) {
         const DenseItem it = dense_item(P.dlist, item, tiles, sub);
-        const int row = it.row;
         uint4 kv[DENSE_NV];
         dense_load_keys(P, it, tid, kv);
-        const RowCfg c = load_cfg(P, row);
-        dense_row_stats(P, row, tiles, sm, tid);
-        __syncthreads();
-        const uint32_t Mkey = sm.Mkey, mkey = sm.mkey;
-        const unsigned int Nf = sm.Nf;
-        const bool bad = c.bad || sm.bad;
-        __syncthreads();
-        if (bad || Nf == 0u) {
-            if (it.tile == 0 && it.part == 0 && tid == 0) emit_row(P, c, row, -1, 0.0f, (bad ? F_BADPARAM : F_NO_TOKEN) | F_DENSE, 0, 0.0f);
-            continue;
+        if (it.row != cur_row) {
+            cur_row = it.row;
+            RowCfg c;
+            par = dense_row_par(P, it.row, tiles, sm, dyn, tid, stage, it.tile == 0 && it.part == 0, c);
         }
-        const float Mf = unkey(Mkey);
-        if (c.z & M_TOP_P) {
-            const float scale = dense_scale(Mkey, mkey, Nf);
+        if (par.kind == 1) {
             unsigned int *hm0 = reinterpret_cast<unsigned int *>(dyn), *hm1 = hm0 + DBINS;
-            dense_hist_item(P, it, kv, Mf, scale, hm0, hm1, tid);
-            if (dense_arrive(&P.drow[row].ticket_h, tiles * sub, sm, tid)) dense_hist_finish(P, c, row, sm, dyn, tid, Mkey, scale);
-        } else {
-            // min-p: the elements at or above the threshold key; neither: every finite element.  No bin, no list.
-            const uint32_t tk = (c.z & M_MIN_P) ? minp_key(Mf, c.theta) : 0u;
-            const uint32_t khi = tk ? tk - 1u : KEY_NEG_INF;
-            dense_collect_item(P, c, it, tiles, kv, Mkey, 0xFFFFFFFFu, khi, 0ull, tk, sm, dyn, tid);
+            dense_hist_item(P, it, kv, unkey(par.Mkey), par.scale, hm0, hm1, tid);
+        } else if (par.kind == 2) {
+            dense_collect_part(P, it, kv, unkey(par.Mkey), par.klo, par.khi, sm, dyn, tid);
         }
         __syncthreads();
-        KERNEL_T1(6);
     }
 }
 
-// Stage 3: pass C for the rows whose crossing bin pass H has found.
+// Stage 2 never waits for its predecessor in the stream: on the library's internal stream it is an ordinary launch
+// behind the streaming kernel; on the caller's stream it is a programmatic dependent of the merge kernel, whose CTAs
+// let their dependents go only after their own wait for the streaming kernel, so when a CTA of this grid starts,
+// the streaming kernel is complete and its results are visible.
+__global__ void __launch_bounds__(DENSE_THREADS, 2)
+sonic_dense_stage2_kernel(const KParams P, const int tiles) {
+    extern __shared__ __align__(16) unsigned char dense_dyn_raw[];
+    __shared__ DenseShared sm;
+    pdl_launch_dependents();
+    KERNEL_T0(6);
+    dense_items(P, tiles, (int)blockIdx.x, (int)gridDim.x, reinterpret_cast<unsigned long long *>(dense_dyn_raw), sm, 2);
+    KERNEL_T1(6);
+}
+
 __global__ void __launch_bounds__(DENSE_THREADS, 2)
 sonic_dense_collect_kernel(const KParams P, const int tiles) {
+    extern __shared__ __align__(16) unsigned char dense_dyn_raw[];
+    __shared__ DenseShared sm;
+    pdl_launch_dependents();
+    pdl_wait_primary();
+    KERNEL_T0(3);
+    dense_items(P, tiles, (int)blockIdx.x, (int)gridDim.x, reinterpret_cast<unsigned long long *>(dense_dyn_raw), sm, 3);
+    KERNEL_T1(3);
+}
+
+// The rows' finish, one CTA per row of the class (a programmatic dependent of pass C, whose completion is the only
+// synchronisation a row needs).
+__global__ void __launch_bounds__(DENSE_THREADS)
+sonic_dense_finish_kernel(const KParams P, const int tiles) {
     extern __shared__ __align__(16) unsigned char dense_dyn_raw[];
     __shared__ DenseShared sm;
     unsigned long long *dyn = reinterpret_cast<unsigned long long *>(dense_dyn_raw);
     const int tid = threadIdx.x;
     pdl_launch_dependents();
-    DSTAMP(30);
     pdl_wait_primary();
-    DSTAMP(31);
-    KERNEL_T0(3);
+    KERNEL_T0(8);
     const int nd = (int)__ldcg(&P.error[WS_NDENSE]);
-    const int sub = dense_pick_sub(nd, tiles, (int)gridDim.x);
-    for (int item = blockIdx.x; item < nd * tiles * sub; item += gridDim.x) {
-        const DenseItem it = dense_item(P.dlist, item, tiles, sub);
-        const DenseRow *dr = P.drow + it.row;
-        DSTAMP(0);
-        uint4 kv[DENSE_NV];
-        dense_load_keys(P, it, tid, kv);
-        if (__ldcg(&dr->state) != 1u) continue;          // no top-p (finished in stage 2), or no token
-        const RowCfg c = load_cfg(P, it.row);
-        const uint32_t Mkey = __ldcg(&dr->Mkey), tk = __ldcg(&dr->tk), klo = __ldcg(&dr->klo), khi = __ldcg(&dr->khi);
-        const unsigned long long target = __ldcg(&dr->target);
-        DSTAMP(1);
-        dense_collect_item(P, c, it, tiles, kv, Mkey, klo, khi, target, tk, sm, dyn, tid);
+    for (int i = blockIdx.x; i < nd; i += gridDim.x) {
+        const int row = __ldcg(&P.dlist[i]);
+        RowCfg c;
+        // (the Philox cells need the request's seed and offset only: their loads go out with the row's other loads)
+        const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
+        const unsigned long long seed = P.seed ? P.seed[req] : 0ull, off = P.offset ? P.offset[req] : 0ull;
+        const DenseRowPar par = dense_row_par(P, row, tiles, sm, dyn, tid, 4, false, c);
+        if (par.kind == 0) continue;
+        uint32_t r4[4];
+        const unsigned long long pos = off + (unsigned long long)c.l;
+        philox4x32_10((uint32_t)pos, (uint32_t)(pos >> 32), (uint32_t)c.b, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), r4);
+        const uint2 cells = make_uint2(r4[0] >> 8, r4[1] >> 8);
+        const bool ok = dense_finish(P, c, row, tiles, sm, dyn, tid, par.Mkey, par.klo <= par.khi, par.target, par.tk, cells);
+        if (!ok && tid == 0) { P.rs[row].status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
         __syncthreads();
-        KERNEL_T1(3);
     }
+    KERNEL_T1(8);
 }
 
 // Stage 4 (verification calls): the residual max(0, p - q) of the positions whose draft was rejected.  The
@@ -905,13 +979,14 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
             const int base_idx = tile * CTA_TILE + tid * DENSE_EPT + 4 * k;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
+                // (no branch per element: the sixteen chains of a thread overlap)
                 const int idx = base_idx + u;
-                if ((((unsigned long long)key4[u] << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc) {
-                    const double w = exp((double)unkey(key4[u]) - Md);
-                    const double r = w * inv_Wt - (double)__ldg(q + idx);
-                    S += w;
-                    if (r > 0.0) { R += r; Pp += w; }
-                }
+                const bool in = (((unsigned long long)key4[u] << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc;
+                const double w = in ? exp((double)unkey(key4[u]) - Md) : 0.0;
+                const double r = w * inv_Wt - (double)(in ? __ldg(q + idx) : 0.0f);
+                S += w;
+                R += (r > 0.0) ? r : 0.0;
+                Pp += (r > 0.0) ? w : 0.0;
             }
         }
         // fixed reduction order: lanes by butterfly, warps in order
@@ -928,20 +1003,21 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
             for (int w = 0; w < DENSE_WARPS; ++w) { r += sm.redd[0][w]; p += sm.redd[1][w]; s += sm.redd[2][w]; }
             dt[tile].R = r; dt[tile].Pp = p; dt[tile].S = s;
         }
-        if (!dense_arrive(&dr->ticket_r, tiles, sm, tid)) continue;
+        if (!dense_arrive(&dr->ticket_r, 1, tiles, sm, tid)) continue;
         // ---- the row's last CTA: corrected tile residuals, the tile of the draw, the element
-        if (tid == 0) {
+        if (tid < 32) {
+            // a tile's three sums per lane (one round of loads), added up in tile order by every lane alike
+            double sj = 0.0, rj0 = 0.0, pj = 0.0;
+            if (tid < tiles) { sj = __ldcg(&dt[tid].S); rj0 = __ldcg(&dt[tid].R); pj = __ldcg(&dt[tid].Pp); }
             double Wd = 0.0;
-            for (int j = 0; j < tiles; ++j) Wd += __ldcg(&dt[j].S);
+            for (int j = 0; j < tiles; ++j) Wd += __shfl_sync(0xFFFFFFFFu, sj, j);
             const double corr = inv_Wt - 1.0 / Wd;
+            double rj = rj0 - corr * pj;
+            rj = (tid < tiles && rj > 0.0) ? rj : 0.0;
+            reinterpret_cast<double *>(sm.wt)[tid] = rj;
             double Rtot = 0.0;
-            for (int j = 0; j < tiles; ++j) {
-                double rj = __ldcg(&dt[j].R) - corr * __ldcg(&dt[j].Pp);
-                rj = rj > 0.0 ? rj : 0.0;
-                reinterpret_cast<double *>(sm.wt)[j] = rj;
-                Rtot += rj;
-            }
-            sm.bcd[0] = Wd; sm.bcd[1] = Rtot;
+            for (int j = 0; j < tiles; ++j) Rtot += __shfl_sync(0xFFFFFFFFu, rj, j);
+            if (tid == 0) { sm.bcd[0] = Wd; sm.bcd[1] = Rtot; }
         }
         __syncthreads();
         const double Wd = sm.bcd[0], Rtot = sm.bcd[1];
@@ -960,8 +1036,8 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
             if (jt < 0) { cum = 0.0; for (int j = 0; j < tiles; ++j) { if (rj[j] > 0.0) { jt = j; before = cum; } cum += rj[j]; } }
             const double inv_Wd = 1.0 / Wd;
             auto wf = [=](uint32_t key, int idx) -> double {
-                if (!((((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc)) return 0.0;
-                const double r = exp((double)unkey(key) - Md) * inv_Wd - (double)__ldg(q + idx);
+                const bool in = (((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc;
+                const double r = (in ? exp((double)unkey(key) - Md) : 0.0) * inv_Wd - (double)(in ? __ldg(q + idx) : 0.0f);
                 return r > 0.0 ? r : 0.0;
             };
             double rw;

@@ -1432,21 +1432,14 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
 // One CTA per row of the streaming classes: combines the tile records and
 // finishes the row (global top-k, truncation epilogue, token selection, or the
 // per-position verification result).  Rows it cannot prove are flagged for the
-// cluster kernel.  The CTAs past the row count run stage 2 of the histogram path
-// (rows with top-k off) beside them.
-__global__ void __launch_bounds__(MERGE_THREADS, 2)
+// cluster kernel.
+__global__ void __launch_bounds__(MERGE_THREADS)
 sonic_merge_kernel(const KParams P, const int tiles) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ MergeShared<MERGE_THREADS> s_merge;
     const int row = blockIdx.x;
     const int tid = threadIdx.x;
-    pdl_launch_dependents();                   // the next kernel of the call may start launching; it waits for this grid
     KERNEL_T0(1);
-    if (row >= P.rows) {
-        pdl_wait_primary();
-        dense_stage2(P, tiles, row - P.rows, (int)gridDim.x - P.rows, reinterpret_cast<unsigned long long *>(smem_raw));
-        return;
-    }
     const RowCfg c = load_cfg(P, row);         // inputs only: independent of the streaming kernel
     const bool other = (c.cls == CLS_EXACT || c.cls == CLS_DENSE);
     if (other && row != 0) return;
@@ -1454,6 +1447,10 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     uint2 cells = make_uint2(0u, 0u);
     if (P.op != OP_TOPK && c.cls == CLS_TOPK) draw_cells(P, c, cells.x, cells.y);
     pdl_wait_primary();                        // tile records and candidates of the streaming kernel
+    // The next kernel of the call (stage 2 of the histogram path) does not wait for this grid: it needs the
+    // streaming kernel's results only, and those are complete once every CTA here is past its wait (the first
+    // row's CTA never leaves before it).  So it is let go after the wait, and runs beside the merges.
+    pdl_launch_dependents();
     if (row == 0 && tid == 0) P.error[WS_QUEUE] = 0u;    // the streaming kernel is done with its work counter
     if (other) return;
     RowState *rs = P.rs + row;
