@@ -51,6 +51,7 @@ struct DenseShared {
     unsigned long long comp[DENSE_THREADS];          // listed elements (fast path: at most one per thread)
     unsigned long long wt[DENSE_THREADS];            // their weights in ranking order
     unsigned long long chunk[DENSE_THREADS];         // support mass per chunk of 512 elements (tile-major)
+    unsigned int sub[5][DENSE_THREADS];              // medium path of the finish: per sub-bin count, mass words, smallest and largest key
     unsigned long long bc64[4];
     double bcd[2];
     unsigned int nstage, kmin, kmax, base;
@@ -611,30 +612,148 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
     unsigned int n_in = 0u;
     bool chunks_final = true;                     // the per-chunk masses include the listed elements that are in
     if (listed && nb > 0u) {
-        const unsigned long long rest = max(target > C_above ? target - C_above : 1ull, 1ull);
-        if (nb <= (unsigned int)DENSE_THREADS && !overflow) {
+        unsigned long long rest = max(target > C_above ? target - C_above : 1ull, 1ull);
+        // Listed elements that are in for sure although they sit in the crossing bin (the medium path below finds
+        // them above the sub-bin the cut falls into): their mass and number
+        unsigned long long sure_mass = 0ull;
+        unsigned int sure_n = 0u;
+        bool small_ready = (nb <= (unsigned int)DENSE_THREADS && !overflow);
+        unsigned int n_small = nb;
+        uint32_t tie_v = 0u;                      // medium / crowded path: the cut falls among the ties of this key
+        bool tie_path = false, in_smem = false, no_target = false;     // no_target: top-p does not decide inside the short list
+        unsigned int tie_n = 0u;
+        if (!small_ready && nb <= (unsigned int)MEMBER_CAP && !overflow) {
+            // Medium path: up to MEMBER_CAP listed elements (low-precision logits: a few values, hundreds of ties
+            // each).  One level of 512 sub-bins uniform over the listed keys' span separates the values; the
+            // sub-bin the cut falls into then holds few elements (ranked like a short list) or the ties of one key.
+            in_smem = true;
+            const unsigned long long *gm = P.members + (size_t)row * MEMBER_CAP;
+            for (int i = tid; i < (int)nb; i += DENSE_THREADS) dyn[i] = __ldcg(&gm[i]);
+            const uint32_t kmin = __ldcg(&dr->kmin), kmax = __ldcg(&dr->kmax);
+            const unsigned long long span = (unsigned long long)(kmax - kmin) + 1ull;
+            unsigned int *scnt = sm.sub[0], *slo = sm.sub[1], *shi = sm.sub[2], *smin = sm.sub[3], *smax = sm.sub[4];
+            scnt[tid] = 0u; slo[tid] = 0u; shi[tid] = 0u; smin[tid] = 0xFFFFFFFFu; smax[tid] = 0u;
+            __syncthreads();
+            auto subbin = [=](uint32_t key) -> int { return (int)(((unsigned long long)(key - kmin) * (unsigned long long)DENSE_THREADS) / span); };
+            for (int i = tid; i < (int)nb; i += DENSE_THREADS) {
+                const uint32_t key = (uint32_t)(dyn[i] >> 32);
+                const int sb = subbin(key);
+                const unsigned long long w1 = qweight(key, Mf);
+                // lanes holding the same key (ties: same sub-bin, same weight) add once
+                const unsigned int peers = __match_any_sync(__activemask(), key);
+                if ((tid & 31) == __ffs(peers) - 1) {
+                    const unsigned int np = __popc(peers);
+                    const unsigned long long w = w1 * np;
+                    atomicAdd(&scnt[sb], np);
+                    const unsigned int lo = (unsigned int)w, hi = (unsigned int)(w >> 32);
+                    unsigned int carry = 0;
+                    if (lo) { const unsigned int old = atomicAdd(&slo[sb], lo); carry = (old + lo < old) ? 1u : 0u; }
+                    if (hi + carry) atomicAdd(&shi[sb], hi + carry);
+                    atomicMin(&smin[sb], key); atomicMax(&smax[sb], key);
+                }
+            }
+            __syncthreads();
+            // thread t owns sub-bin 511 - t (from the top): mass and number of the listed elements above it
+            const int sbm = DENSE_THREADS - 1 - tid;
+            const unsigned long long mmass = (unsigned long long)slo[sbm] | ((unsigned long long)shi[sbm] << 32);
+            unsigned long long tot;
+            const unsigned long long pre = dense_block_scan<unsigned long long>(mmass, sm.red64, tid, tot);
+            const unsigned int mcnt = scnt[sbm];
+            unsigned int cincl = mcnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, cincl, o); if (lane >= o) cincl += up; }
+            if (lane == 31) sm.red32[0][warp] = cincl;
+            if (tid == 0) sm.flag = 0;
+            __syncthreads();
+            unsigned int coff = 0u;
+            for (int w = 0; w < warp; ++w) coff += sm.red32[0][w];
+            const unsigned int cpre = coff + cincl - mcnt;
+            {
+                // the sub-bin where the running mass reaches what is missing ...
+                const unsigned long long r = min(rest, max(tot, 1ull));
+                if (mmass > 0ull && pre < r && r <= pre + mmass) sm.flag = sbm;
+            }
+            __syncthreads();
+            // ... against the sub-bin of the min-p threshold: the higher one decides (DENSE_THREADS: above every listed key)
+            int xb = sm.flag;
+            bool by_mass = true;
+            if (tk) {
+                const int sbt = (tk > kmax) ? DENSE_THREADS : (tk >= kmin ? subbin(tk) : -1);
+                if (sbt > xb) { xb = sbt; by_mass = false; }
+            }
+            if (xb >= DENSE_THREADS) {
+                // no listed element passes min-p: nothing of the bin is in
+                small_ready = true; n_small = 0u; no_target = true;
+                sm.comp[tid] = 0ull;
+                __syncthreads();
+            } else {
+                if (sbm == xb) { sm.bc64[2] = pre; sm.cnt_above = cpre; }
+                __syncthreads();
+                sure_mass = sm.bc64[2];
+                sure_n = sm.cnt_above;
+                if (by_mass) rest = (rest > sure_mass) ? rest - sure_mass : 1ull; else no_target = true;
+                const unsigned int cx = scnt[xb];
+                const uint32_t xmin = smin[xb], xmax = smax[xb];
+                __syncthreads();
+            if (cx <= (unsigned int)DENSE_THREADS) {
+                // gather the sub-bin's elements as the short list
+                if (tid == 0) sm.nstage = 0u;
+                sm.comp[tid] = 0ull;
+                __syncthreads();
+                for (int i = tid; i < (int)nb; i += DENSE_THREADS) {
+                    const unsigned long long m = dyn[i];
+                    if (subbin((uint32_t)(m >> 32)) == xb) sm.comp[atomicAdd(&sm.nstage, 1u)] = m;
+                }
+                __syncthreads();
+                n_small = cx;
+                small_ready = true;
+            } else if (xmin == xmax) {
+                tie_path = true; tie_v = xmin; tie_n = cx;
+            } else {
+                return false;
+            }
+            // the elements above the sub-bin are in: their mass goes to their tiles and chunks
+            for (int i = tid; i < (int)nb; i += DENSE_THREADS) {
+                const unsigned long long m = dyn[i];
+                const uint32_t key = (uint32_t)(m >> 32);
+                if (subbin(key) > xb && m >= cutc) {
+                    const unsigned long long w = qweight(key, Mf);
+                    const uint32_t idx = ~(uint32_t)m;
+                    if (w) { atomicAdd(&sm.tile_mass[idx / CTA_TILE], w); atomicAdd(&sm.chunk[idx / DENSE_CHUNK], w); }
+                }
+            }
+            __syncthreads();
+            }
+        } else if (!small_ready) {
+            // a crowded bin: resolvable here only if it holds one value repeated (low-precision logits)
+            const uint32_t kmin = __ldcg(&dr->kmin), kmax = __ldcg(&dr->kmax);
+            if (kmin != kmax) return false;
+            tie_path = true; tie_v = kmin; tie_n = nb;
+        }
+        if (small_ready) {
             // at most one listed element per thread: ranks by warp sorts and binary searches, then the running mass
             // in ranking order
             int rank;
-            const unsigned long long key = rank_keys<DENSE_THREADS, BlockSync>(sm.comp, (int)nb, tid, rank);
+            const unsigned long long key = rank_keys<DENSE_THREADS, BlockSync>(sm.comp, (int)n_small, tid, rank);
             const unsigned long long wk = key ? qweight((uint32_t)(key >> 32), Mf) : 0ull;
             __syncthreads();                      // every search has read the runs
             if (key) { sm.comp[rank] = key; sm.wt[rank] = wk; }
+            if (tid == 0) { sm.bc64[0] = 0ull; sm.bc64[1] = 0ull; }
             __syncthreads();
             DSTAMP(5);
-            const bool have = (unsigned int)tid < nb;
+            const bool have = (unsigned int)tid < n_small;
             const unsigned long long mine_c = have ? sm.comp[tid] : 0ull, mine_w = have ? sm.wt[tid] : 0ull;
             unsigned long long total_m;
             const unsigned long long pre = dense_block_scan<unsigned long long>(mine_w, sm.red64, tid, total_m);
-            if (target) {
-                // the element at which the running mass first reaches what is still missing above the bin
+            if (target && !no_target) {
+                // the element at which the running mass first reaches what is still missing above it
                 const unsigned long long r = min(rest, max(total_m, 1ull));
                 if (mine_w > 0ull && pre < r && r <= pre + mine_w) sm.bc64[0] = mine_c;
                 __syncthreads();
                 cutc = max(cutc, sm.bc64[0]);
             }
             DSTAMP(6);
-            // what of the bin is in: a prefix of the ranking; its mass goes to its tiles and chunks for the draw
+            // what of the list is in: a prefix of the ranking; its mass goes to its tiles and chunks for the draw
             const bool inc = have && mine_c >= cutc;
             if (inc && mine_w) {
                 const uint32_t idx = ~(uint32_t)mine_c;
@@ -644,68 +763,32 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
             n_in = (unsigned int)__syncthreads_count(inc ? 1 : 0);
             if (have && (unsigned int)tid + 1u == n_in) sm.bc64[1] = pre + mine_w;
             __syncthreads();
-            mass_in = n_in ? sm.bc64[1] : 0ull;
-        } else if (nb <= (unsigned int)MEMBER_CAP && !overflow) {
-            // many listed elements: a full sort, weights recomputed along the ranking
+            mass_in = (n_in ? sm.bc64[1] : 0ull) + sure_mass;
+            n_in += sure_n;
+        } else if (tie_path) {
+            // the cut falls among tie_n elements of one key: the first m of them in index order are in
             chunks_final = false;
-            const unsigned long long *gm = P.members + (size_t)row * MEMBER_CAP;
-            for (int i = tid; i < (int)nb; i += DENSE_THREADS) dyn[i] = __ldcg(&gm[i]);
-            __syncthreads();
-            dense_sort_members(dyn, (int)nb, tid);
-            const int ept = ((int)nb + DENSE_THREADS - 1) / DENSE_THREADS;
-            const int lo = min((int)nb, tid * ept), hi = min((int)nb, lo + ept);
-            unsigned long long mine = 0ull;
-            for (int j = lo; j < hi; ++j) mine += qweight((uint32_t)(dyn[j] >> 32), Mf);
-            unsigned long long total_m;
-            const unsigned long long pre = dense_block_scan<unsigned long long>(mine, sm.red64, tid, total_m);
-            if (target) {
-                const unsigned long long r = min(rest, max(total_m, 1ull));
-                if (mine > 0ull && pre < r && r <= pre + mine) {
-                    unsigned long long cum = pre;
-                    bool done = false;
-                    for (int j = lo; j < hi; ++j) {
-                        cum += qweight((uint32_t)(dyn[j] >> 32), Mf);
-                        if (!done && cum >= r) { sm.bc64[0] = dyn[j]; done = true; }
-                    }
-                }
-                __syncthreads();
-                cutc = max(cutc, sm.bc64[0]);
-            }
-            unsigned long long ms = 0ull;
-            unsigned int ns = 0u;
-            for (int j = lo; j < hi; ++j) {
-                const unsigned long long m = dyn[j];
-                if (m >= cutc) {
-                    const unsigned long long w = qweight((uint32_t)(m >> 32), Mf);
-                    ms += w; ++ns;
-                    if (w) atomicAdd(&sm.tile_mass[(~(uint32_t)m) / CTA_TILE], w);
-                }
-            }
-            ms = dense_warp_sum(ms);
-            ns = __reduce_add_sync(0xFFFFFFFFu, ns);
-            __syncthreads();
-            if (lane == 0) { sm.red64[warp] = ms; sm.red32[0][warp] = ns; }
-            __syncthreads();
-#pragma unroll
-            for (int w = 0; w < DENSE_WARPS; ++w) { mass_in += sm.red64[w]; n_in += sm.red32[0][w]; }
-            __syncthreads();
-        } else {
-            // a crowded bin: resolvable here only if it holds one value repeated (low-precision logits)
-            chunks_final = false;
-            const uint32_t kmin = __ldcg(&dr->kmin), kmax = __ldcg(&dr->kmax);
-            if (kmin != kmax) return false;
-            const uint32_t v = kmin;
+            const uint32_t v = tie_v;
             const unsigned long long wv = qweight(v, Mf);
-            unsigned long long m = nb;
+            unsigned long long m = tie_n;
             if (tk && v < tk) m = 0ull;
-            if (target && m > 0ull && wv > 0ull) {
+            if (target && !no_target && m > 0ull && wv > 0ull) {
                 const unsigned long long need = (rest + wv - 1ull) / wv;
                 m = min(m, max(need, 1ull));
             }
-            // the first m ties in index order: which tile holds the m-th, and where in it
+            // ties per tile: from the row's tile records when the whole bin is this key, else counted from the list
+            if (in_smem) {
+                if (tid < MAX_TILES) sm.tile_nb[tid] = 0u;
+                __syncthreads();
+                for (int i = tid; i < (int)nb; i += DENSE_THREADS) {
+                    const unsigned long long mm = dyn[i];
+                    if ((uint32_t)(mm >> 32) == v) atomicAdd(&sm.tile_nb[(~(uint32_t)mm) / CTA_TILE], 1u);
+                }
+                __syncthreads();
+            }
             int jt = -1;
             unsigned long long before = 0ull;
-            if (m > 0ull && m < (unsigned long long)nb) {
+            if (m > 0ull && m < (unsigned long long)tie_n) {
                 unsigned long long cum = 0ull;
                 for (int j = 0; j < tiles; ++j) {
                     const unsigned long long t = sm.tile_nb[j];
@@ -730,8 +813,8 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
                     left -= t;
                 }
             }
-            mass_in = m * wv;
-            n_in = (unsigned int)m;
+            mass_in = m * wv + sure_mass;
+            n_in = (unsigned int)m + sure_n;
             __syncthreads();
         }
     }
