@@ -634,7 +634,8 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
             unsigned int *scnt = sm.sub[0], *slo = sm.sub[1], *shi = sm.sub[2], *smin = sm.sub[3], *smax = sm.sub[4];
             scnt[tid] = 0u; slo[tid] = 0u; shi[tid] = 0u; smin[tid] = 0xFFFFFFFFu; smax[tid] = 0u;
             __syncthreads();
-            auto subbin = [=](uint32_t key) -> int { return (int)(((unsigned long long)(key - kmin) * (unsigned long long)DENSE_THREADS) / span); };
+            const unsigned long long mult = ((unsigned long long)DENSE_THREADS << 32) / span;      // (no division per element)
+            auto subbin = [=](uint32_t key) -> int { return min(DENSE_THREADS - 1, (int)(((unsigned long long)(key - kmin) * mult) >> 32)); };
             for (int i = tid; i < (int)nb; i += DENSE_THREADS) {
                 const uint32_t key = (uint32_t)(dyn[i] >> 32);
                 const int sb = subbin(key);
