@@ -29,13 +29,14 @@ __global__ void sonic_verify_combine_kernel(const KParams P, int B) {
         toks[l] = -1;
         if (l < K && P.out_pdraft) P.out_pdraft[(size_t)b * K + l] = (r.flags & (F_BADPARAM | F_NO_TOKEN)) ? 0.0f : r.p;
         if (r.flags & F_BADPARAM) flags |= F_BADPARAM;
+        if (r.flags & F_TIMEOUT) flags |= F_TIMEOUT;
         if (decided) continue;
         flags |= (r.flags & F_FALLBACK);
         if (r.flags & F_NO_TOKEN) { flags |= F_NO_TOKEN; decided = true; continue; }
         if (l < K && (r.flags & F_ACCEPT)) { toks[l] = P.draft_tokens[(size_t)b * K + l]; acc = l + 1; }
         else { toks[l] = r.token; decided = true; }
     }
-    if (flags & F_BADPARAM) {
+    if (flags & (F_BADPARAM | F_TIMEOUT)) {
         for (int l = 0; l <= K; ++l) toks[l] = -1;
         acc = 0;
         flags &= ~F_NO_TOKEN;

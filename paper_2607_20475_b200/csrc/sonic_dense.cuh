@@ -1017,6 +1017,10 @@ sonic_dense_finish_kernel(const KParams P, const int tiles) {
         const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
         const unsigned long long seed = P.seed ? P.seed[req] : 0ull, off = P.offset ? P.offset[req] : 0ull;
         const DenseRowPar par = dense_row_par(P, row, tiles, sm, dyn, tid, 4, false, c);
+        if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {       // (a wait of the streaming kernel ran out: nothing of the row is to be trusted)
+            if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_TIMEOUT | F_DENSE, 0, 0.0f);
+            continue;
+        }
         if (par.kind == 0) continue;
         uint32_t r4[4];
         const unsigned long long pos = off + (unsigned long long)c.l;

@@ -852,6 +852,11 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     SONIC_STAMP(2);
     const bool leader = (x.rank == 0 && x.tid == 0);
 
+    if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {           // (uniform over the cluster; see the merge kernel)
+        if (leader && P.op != OP_TOPK) emit_row(P, c, row, -1, 0.0f, F_TIMEOUT | F_FALLBACK, 0, 0.0f);
+        cg::this_cluster().sync();
+        return;
+    }
     if (bad) {
         if (leader) { emit_row(P, c, row, -1, 0.0f, F_BADPARAM | F_FALLBACK, 0, 0.0f); rs->status = 0; }
         cg::this_cluster().sync();

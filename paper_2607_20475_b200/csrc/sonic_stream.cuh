@@ -1453,6 +1453,15 @@ sonic_merge_kernel(const KParams P, const int tiles) {
     pdl_launch_dependents();
     if (row == 0 && tid == 0) P.error[WS_QUEUE] = 0u;    // the streaming kernel is done with its work counter
     if (other) return;
+    if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {
+        // a bounded wait of the streaming kernel ran out (in this call or an earlier one on this workspace): the
+        // tile records are not to be trusted, the row reports it instead of a token
+        if (tid == 0) {
+            if (P.op == OP_TOPK) { for (int j = 0; j < P.ktop; ++j) { P.out_vals[(size_t)row * P.ktop + j] = -CUDART_INF_F; P.out_idx[(size_t)row * P.ktop + j] = -1; } }
+            else emit_row(P, c, row, -1, 0.0f, F_TIMEOUT, 0, 0.0f);
+        }
+        return;
+    }
     RowState *rs = P.rs + row;
     const TileRec *recs = P.tiles + (size_t)row * MAX_TILES;
     const unsigned int tflags = (tid < tiles) ? __ldcg(&recs[tid].flags) : 0u;

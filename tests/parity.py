@@ -3,20 +3,55 @@
 Integer results (top-k index sets, greedy tokens, accept lengths) must be
 bit-exact.  Sampled / accepted tokens must be bit-exact unless the oracle's
 margin for the row (relative distance of a floating-point decision to its
-threshold) is below 1e-6; such rows are counted and reported.  Probabilities
-agree within 1e-5 relative for fp32 inputs and 2e-3 for bf16 inputs.
+threshold) is below 1e-6.  Such a row admits two outcomes, not any outcome: it
+is counted, reported, and still checked for being one of the admissible ones
+(support within one element of the oracle's, token inside the oracle's ranking
+prefix of that length and next to the oracle's token in index order, its
+probability the oracle's for that token).  Probabilities agree within 1e-5
+relative for fp32 inputs and 2e-3 for bf16 inputs.
 """
 from __future__ import annotations
+
+import math
 
 import numpy as np
 
 from paper_2607_20475_b200 import workloads as wl
 
 MARGIN = 1e-6
-FLAG_MASK = 0x3     # NO_TOKEN | BADPARAM (FALLBACK is a diagnostic of the CUDA path only)
+FLAG_MASK = 0x3     # NO_TOKEN | BADPARAM (the other bits are diagnostics of the CUDA path only)
 
 
-def compare_sample(got, ref, w, max_near=None):
+def _default_max_near(rows: int) -> int:
+    """At most a quarter of the rows (three for the smallest cases) may sit within the margin: rows with top-k off and a
+    nucleus of 10^4 to 10^5 tokens, each about 1e-5 of the mass, land there about one time in five.  Near-margin rows
+    are not skipped: each must still be one of its two admissible outcomes."""
+    return max(3, int(math.ceil(0.25 * rows)))
+
+
+def _admissible_near_row(oracle, w, b, got_token, got_support, got_prob, ref_token, ref_support, rtol):
+    """A near-margin row: one decision (a top-p or min-p cut, or the draw) may have gone the other way."""
+    if abs(int(got_support) - int(ref_support)) > 1:
+        return f"support {got_support} vs {ref_support}"
+    y = oracle.processed_row(w, b).astype(np.float64)
+    order = np.argsort(-y, kind="stable")
+    n = int(max(got_support, ref_support))
+    prefix = order[:n]
+    if got_token not in prefix:
+        return f"token {got_token} outside the ranking prefix of length {n}"
+    ids = np.sort(prefix)
+    pos_got, pos_ref = int(np.searchsorted(ids, got_token)), int(np.searchsorted(ids, ref_token))
+    if abs(pos_got - pos_ref) > 1:
+        return f"token {got_token} is not next to the oracle's {ref_token} in index order"
+    keep = order[:int(got_support)]
+    wts = np.exp(y[keep] - y[order[0]])
+    p = math.exp(y[got_token] - y[order[0]]) / wts.sum()
+    if abs(got_prob - p) > 10 * rtol * p + 1e-12:
+        return f"probability {got_prob} vs {p}"
+    return None
+
+
+def compare_sample(got, ref, w, max_near=None, oracle=None):
     B = w.B
     near = ref["margin"] < MARGIN
     rtol = 2e-3 if w.dtype == wl.DTYPE_BF16 else 1e-5
@@ -24,6 +59,9 @@ def compare_sample(got, ref, w, max_near=None):
         (np.nonzero((got["flags"] & FLAG_MASK) != (ref["flags"] & FLAG_MASK))[0][:10])
     greedy = (w.mode & wl.GREEDY) != 0
     bad = []
+    if oracle is None:
+        from oracle import oracle as _o      # (tests only)
+        oracle = _o
     for b in range(B):
         if greedy[b] or not near[b]:
             if got["token"][b] != ref["token"][b] or got["support"][b] != ref["support"][b]:
@@ -32,10 +70,15 @@ def compare_sample(got, ref, w, max_near=None):
             elif ref["token"][b] >= 0:
                 assert abs(got["prob"][b] - ref["prob"][b]) <= rtol * ref["prob"][b] + 1e-12, \
                     (b, got["prob"][b], ref["prob"][b])
+        elif ref["token"][b] >= 0:
+            why = _admissible_near_row(oracle, w, b, int(got["token"][b]), int(got["support"][b]), float(got["prob"][b]),
+                                       int(ref["token"][b]), int(ref["support"][b]), rtol)
+            if why:
+                bad.append((b, "near-margin row, not an admissible outcome: " + why, float(ref["margin"][b]), hex(int(w.mode[b]))))
     assert not bad, f"{len(bad)} rows differ (row, got, ref, got_support, ref_support, margin, mode): {bad[:8]}"
-    n_near = int(near.sum())
-    if max_near is not None:
-        assert n_near <= max_near, f"{n_near} near-margin rows"
+    n_near = int((near & ~greedy).sum())
+    limit = _default_max_near(B) if max_near is None else max_near
+    assert n_near <= limit, f"{n_near} near-margin rows of {B} (limit {limit})"
     return n_near
 
 
@@ -43,17 +86,33 @@ def compare_verify(got, ref, vw, max_near=None):
     near = ref["margin"] < MARGIN
     assert np.array_equal(got["flags"] & FLAG_MASK, ref["flags"] & FLAG_MASK)
     bad = []
+    K = vw.K
+    greedy = (vw.sample.mode & wl.GREEDY) != 0
     for b in range(vw.B):
-        if near[b] and not (vw.sample.mode[b] & wl.GREEDY):
+        g_tok, r_tok = got["tokens"][b], ref["tokens"][b]
+        if near[b] and not greedy[b]:
+            # one decision may have gone the other way: the outputs must still be well formed (accepted drafts, one
+            # more token, then -1) and agree with the oracle up to the first position where they part
+            a = int(got["accept_len"][b])
+            ok = 0 <= a <= K and np.array_equal(g_tok[:a], vw.draft_tokens[b, :a]) and (g_tok[a + 1:] == -1).all() \
+                and 0 <= g_tok[a] < vw.V
+            first = next((l for l in range(K + 1) if g_tok[l] != r_tok[l]), K + 1)
+            ok = ok and first >= min(a, int(ref["accept_len"][b]))
+            if not ok:
+                bad.append((b, "near-margin request, malformed", g_tok.tolist(), r_tok.tolist(), float(ref["margin"][b])))
             continue
-        if got["accept_len"][b] != ref["accept_len"][b] or not np.array_equal(got["tokens"][b], ref["tokens"][b]):
-            bad.append((b, got["tokens"][b].tolist(), ref["tokens"][b].tolist(), float(ref["margin"][b])))
+        if got["accept_len"][b] != ref["accept_len"][b] or not np.array_equal(g_tok, r_tok):
+            bad.append((b, g_tok.tolist(), r_tok.tolist(), float(ref["margin"][b])))
     assert not bad, f"{len(bad)} requests differ: {bad[:6]}"
-    assert np.allclose(got["p_draft"], ref["p_draft"], rtol=1e-5, atol=1e-9), \
-        np.abs(got["p_draft"] - ref["p_draft"]).max()
-    n_near = int(near.sum())
-    if max_near is not None:
-        assert n_near <= max_near
+    sure = ~(near & ~greedy)
+    assert np.allclose(got["p_draft"][sure], ref["p_draft"][sure], rtol=1e-5, atol=1e-9), \
+        np.abs(got["p_draft"][sure] - ref["p_draft"][sure]).max()
+    # (a near-margin request: a cut that went the other way moves every probability of the position by about the
+    #  mass of one element)
+    assert np.allclose(got["p_draft"][~sure], ref["p_draft"][~sure], rtol=1e-4, atol=2e-6)
+    n_near = int((near & ~greedy).sum())
+    limit = _default_max_near(vw.B) if max_near is None else max_near
+    assert n_near <= limit, f"{n_near} near-margin requests of {vw.B} (limit {limit})"
     return n_near
 
 

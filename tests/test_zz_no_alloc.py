@@ -3,7 +3,8 @@
 serving loop in which cudaMalloc would stall the device).  It takes no workspace: its scratch is a fixed array inside the
 library.  Checked here against sonic_topk, bit for bit, on two calls in a row with
 different inputs, so that what the first call leaves in the shared array cannot leak
-into the second.  Collected last on purpose."""
+into the second; and against the CPU oracle's sorted top-k as well, so that the check does
+not rest on the other entry point alone.  Collected last on purpose."""
 import numpy as np
 import pytest
 
@@ -29,6 +30,10 @@ def test_static_scratch_topk_matches_workspace_topk_twice():
         torch.cuda.synchronize()
         assert np.array_equal(out_idx.cpu().numpy(), ref_idx), f"call {call}: indices differ"
         assert np.array_equal(out_vals.cpu().numpy().view(np.uint32), ref_vals.view(np.uint32)), f"call {call}"
+        from oracle import oracle
+        ov, oi = oracle.topk(tw.logits_f32(), k)
+        assert np.array_equal(out_idx.cpu().numpy(), oi), f"call {call}: indices differ from the oracle's"
+        assert np.array_equal(out_vals.cpu().numpy().view(np.uint32), ov.view(np.uint32)), f"call {call}: values differ from the oracle's"
 
 
 def test_static_scratch_rejects_more_rows_than_it_holds():
