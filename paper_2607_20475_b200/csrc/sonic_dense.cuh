@@ -27,7 +27,7 @@ namespace sonic {
 
 #ifdef SONIC_DTRACE
 __device__ __forceinline__ unsigned int dtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
-#define DSTAMP(i) do { if (threadIdx.x == 0) P.error[64 + (i)] = dtimer(); } while (0)
+#define DSTAMP(i) do { if (threadIdx.x == 0 && blockIdx.x == 0) P.error[64 + (i)] = dtimer(); } while (0)
 #else
 #define DSTAMP(i) do { } while (0)
 #endif
@@ -330,8 +330,6 @@ __device__ int dense_tile_find(const KParams &P, int row, int tile, T rest, WF w
     if (tid == 0) { sm.flag = -1; sm.digit = -1; }
     T s = T(0);
     int lastpos = -1;
-    if (kv[0].x == 0x12345u && kv[3].w == 0x54321u) lastpos = -2;     // (trace builds: the loads have landed)
-    DSTAMP(20);
 #pragma unroll
     for (int k = 0; k < DENSE_NV; ++k) {
         const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
@@ -342,10 +340,8 @@ __device__ int dense_tile_find(const KParams &P, int row, int tile, T rest, WF w
             if (w > T(0)) lastpos = first + k * 4 + u;
         }
     }
-    DSTAMP(21);
     T total;
     const T pre = dense_block_scan<T>(s, wtot, tid, total);
-    DSTAMP(22);
     // weight of the thread's first element whose running sum exceeds `rest` (want_last: of its last positive element)
     auto walk = [&](bool want_last, int &found, T &fw) {
         T cum = pre;
@@ -381,7 +377,6 @@ __device__ int dense_tile_find(const KParams &P, int row, int tile, T rest, WF w
         }
         __syncthreads();
     }
-    DSTAMP(23);
     w_out = *reinterpret_cast<T *>(&sm.bc64[3]);
     const int res = sm.flag;
     __syncthreads();
@@ -402,11 +397,6 @@ __device__ __forceinline__ void dense_collect_part(const KParams &P, const Dense
     const int base_idx = it.first(tid);
     const int nv = it.nv();
     const bool any_members = klo <= khi;
-    DSTAMP(41);
-#ifdef SONIC_DTRACE
-    if (kv[0].x == 0xdeadbeefu && kv[0].w == 0x12345u) am = 1ull;
-    DSTAMP(46);
-#endif
     // the weights first, without a branch per element (the chains of a thread's elements overlap) ...
 #pragma unroll
     for (int k = 0; k < DENSE_NV; ++k) {
@@ -443,7 +433,6 @@ __device__ __forceinline__ void dense_collect_part(const KParams &P, const Dense
             }
         }
     }
-    DSTAMP(42);
     am = dense_warp_sum(am);
     an = __reduce_add_sync(0xFFFFFFFFu, an);
     bn = __reduce_add_sync(0xFFFFFFFFu, bn);
@@ -464,7 +453,6 @@ __device__ __forceinline__ void dense_collect_part(const KParams &P, const Dense
         P.dtile[(size_t)it.row * MAX_TILES + it.tile].ch[it.part * nchunks + tid] = r;
     }
     const unsigned int cnt = sm.nstage;
-    DSTAMP(43);
     if (cnt == 0u) return;
     if (tid == 0) {
         DenseRow *dr = P.drow + it.row;
@@ -568,7 +556,6 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
     const int lane = tid & 31, warp = tid >> 5;
     DenseRow *dr = P.drow + row;
     DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
-    DSTAMP(3);
     // everything the other CTAs left, requested at once: a chunk record per thread, the first DENSE_THREADS listed
     // elements (one per thread, whatever their number turns out to be), their count and the overflow mark
     unsigned int nm = 0u, overflow = 0u;
@@ -599,7 +586,6 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
         if (tid == 0) { sm.bc64[0] = 0ull; sm.bc64[1] = 0ull; }
     }
     __syncthreads();
-    DSTAMP(4);
     unsigned long long C_above = 0ull;
     unsigned int cnt_above = 0u;
 #pragma unroll
@@ -741,7 +727,6 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
             if (key) { sm.comp[rank] = key; sm.wt[rank] = wk; }
             if (tid == 0) { sm.bc64[0] = 0ull; sm.bc64[1] = 0ull; }
             __syncthreads();
-            DSTAMP(5);
             const bool have = (unsigned int)tid < n_small;
             const unsigned long long mine_c = have ? sm.comp[tid] : 0ull, mine_w = have ? sm.wt[tid] : 0ull;
             unsigned long long total_m;
@@ -753,7 +738,6 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
                 __syncthreads();
                 cutc = max(cutc, sm.bc64[0]);
             }
-            DSTAMP(6);
             // what of the list is in: a prefix of the ranking; its mass goes to its tiles and chunks for the draw
             const bool inc = have && mine_c >= cutc;
             if (inc && mine_w) {
@@ -821,7 +805,6 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
     }
     const unsigned long long W = C_above + mass_in;
     const int support = (int)(cnt_above + n_in);
-    DSTAMP(7);
     const uint32_t a_acc = cells.x, a_draw = cells.y;
     uint32_t flags = F_DENSE;
     float p_draft = 0.0f;
@@ -858,7 +841,6 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
         if (tid < 32) {
             unsigned long long qt;
             const int token = dense_warp_draw(P, row, tiles, sm, cutc, Mf, T, lane, qt);
-            DSTAMP(10);
             if (tid == 0) emit_row(P, c, row, token, (float)((double)qt / (double)W), flags, support, 0.0f);
         }
         return true;
@@ -954,6 +936,7 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
     int cur_row = -1;
     DenseRowPar par;
     par.kind = 0;
+    DSTAMP((stage - 2) * 16 + 0);
     for (int item = rg.lo; item < rg.hi; ++item) {
         const DenseItem it = dense_item(P.dlist, item, tiles, sub);
         uint4 kv[DENSE_NV];
@@ -963,6 +946,7 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
             RowCfg c;
             par = dense_row_par(P, it.row, tiles, sm, dyn, tid, stage, it.tile == 0 && it.part == 0, c);
         }
+        DSTAMP((stage - 2) * 16 + 1 + 2 * min(item - rg.lo, 6));
         if (par.kind == 1) {
             unsigned int *hm0 = reinterpret_cast<unsigned int *>(dyn), *hm1 = hm0 + DBINS;
             dense_hist_item(P, it, kv, unkey(par.Mkey), par.scale, hm0, hm1, tid);
@@ -970,6 +954,7 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
             dense_collect_part(P, it, kv, unkey(par.Mkey), par.klo, par.khi, sm, dyn, tid);
         }
         __syncthreads();
+        DSTAMP((stage - 2) * 16 + 2 + 2 * min(item - rg.lo, 6));
     }
 }
 

@@ -46,6 +46,10 @@ __device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned int 
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Announces `bytes` of a copy to the barrier's current phase without arriving on it (the arrival follows later).
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned int bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, unsigned int bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
@@ -1034,15 +1038,21 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
         int item = current_item();
         STREAM_STAMP(1);
         bool prepared = false;
-        auto issue_copy = [&](int row, int tile, int s) {         // lane 0: the tile's bulk copy (the arrival on full[s])
+        // lane 0: the tile's bulk copy, with the arrival on full[s] (arrive == true) or with the bytes announced only
+        // (the arrival then follows once the stage's description is written)
+        auto issue_copy = [&](int row, int tile, int s, bool arrive) {
             const int first = tile * CTA_TILE;
             const int elems = min(CTA_TILE, ((P.V - first) + VEC - 1) / VEC * VEC);
             const unsigned int bytes = (unsigned int)elems * ELT;
             const unsigned char *src = reinterpret_cast<const unsigned char *>(P.logits) +
                                        ((size_t)row * (size_t)P.row_stride + (size_t)first) * ELT;
-            mbar_arrive_expect_tx(&sh.full[s], bytes);
+            if (arrive) mbar_arrive_expect_tx(&sh.full[s], bytes); else mbar_expect_tx(&sh.full[s], bytes);
             bulk_load(stages + (size_t)s * STAGE_BYTES, src, bytes, &sh.full[s], l2_policy);
         };
+        // The CTA's first tile is requested at once, before its row's parameters and lists are known (they take two
+        // rounds of global loads): the copy's latency hides behind them.  (A row of the cluster kernel's class gets
+        // a copy nobody reads: such rows are rare.)
+        if (item >= 0 && lane == 0) issue_copy(item / tiles, item % tiles, 0, false);
         for (;; ++n) {
             const int s = n % NSTAGE;
             if (n >= NSTAGE) {
@@ -1077,8 +1087,8 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
                 m.bad = bad_now;
                 m.next_row = (nxt >= 0) ? nxt / tiles : -1;
                 m.next_tile = (nxt >= 0) ? nxt % tiles : -1;
-                if (c.cls == CLS_EXACT) mbar_arrive(&sh.full[s]);      // nothing is copied for rows of the exact class
-                else issue_copy(row, tile, s);
+                if (n == 0 || c.cls == CLS_EXACT) mbar_arrive(&sh.full[s]);     // (the first tile's copy is under way; nothing is copied for rows of the cluster kernel's class)
+                else issue_copy(row, tile, s, true);
             }
             __syncwarp();
             // hit buffer (n + 1) % (NSTAGE + 1) was last used by tile n - NSTAGE, which the consumers have left
