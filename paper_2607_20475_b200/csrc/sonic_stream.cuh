@@ -1443,7 +1443,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
 // finishes the row (global top-k, truncation epilogue, token selection, or the
 // per-position verification result).  Rows it cannot prove are flagged for the
 // cluster kernel.
-__global__ void __launch_bounds__(MERGE_THREADS)
+__global__ void __launch_bounds__(MERGE_THREADS, 2)
 sonic_merge_kernel(const KParams P, const int tiles) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ MergeShared<MERGE_THREADS> s_merge;
