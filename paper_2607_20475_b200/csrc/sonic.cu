@@ -286,8 +286,11 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
         if (e != cudaSuccess) return unwind(fail_cuda(e, "row finish launch"));
         if (P.op == OP_VERIFY && P.K > 0) {
             dcfg.dynamicSmemBytes = 0;
+            fcfg.dynamicSmemBytes = 0;
             e = cudaLaunchKernelEx(&dcfg, sonic_dense_resid_kernel, P, tiles);
             if (e != cudaSuccess) return unwind(fail_cuda(e, "residual pass launch"));
+            e = cudaLaunchKernelEx(&fcfg, sonic_dense_resid_finish_kernel, P, tiles);
+            if (e != cudaSuccess) return unwind(fail_cuda(e, "residual draw launch"));
         }
     }
     if (side) {

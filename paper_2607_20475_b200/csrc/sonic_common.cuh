@@ -413,6 +413,28 @@ __device__ __forceinline__ unsigned long long qweight(uint32_t key, float Mf) {
     return __float2ull_rn(w * 1099511627776.0f);
 }
 
+// exp(d) for d <= 0 in fp32 with a relative error below 1e-7 and no bias to speak of (mean 4e-10): d * log2(e) is
+// split into its nearest integer and a fraction in [-1/2, 1/2] by one fused multiply-add (so the error does not grow
+// with |d|), 2^fraction is a degree-6 polynomial, the integer goes into the exponent field.  Used where fp64 is too
+// slow to weigh every element (the residual pass) and ex2.approx is too coarse.
+__device__ __forceinline__ float exp_accurate(float d) {
+    d = fmaxf(d, -80.0f);
+    const float L1 = 1.44269502162933349609375f;        // fp32(log2 e)
+    const float L2 = 1.925963033500011e-08f;            // log2 e - L1
+    const float MAGIC = 12582912.0f;                     // 1.5 * 2^23: adding it leaves the nearest integer in the low mantissa bits
+    const float r = fmaf(d, L1, MAGIC);
+    const int ei = __float_as_int(r) - 0x4B400000;       // round(d * log2 e), >= -116
+    const float f = fmaf(d, L2, fmaf(d, L1, -__fsub_rn(r, MAGIC)));
+    float p = 0.00015337577497120947f;
+    p = fmaf(p, f, 0.0013399859890341759f);
+    p = fmaf(p, f, 0.009618519805371761f);
+    p = fmaf(p, f, 0.05550329014658928f);
+    p = fmaf(p, f, 0.24022646248340607f);
+    p = fmaf(p, f, 0.6931471824645996f);
+    p = fmaf(p, f, 1.0f);                                // 2^f in [0.7071, 1.4143]
+    return __int_as_float(__float_as_int(p) + (ei << 23));
+}
+
 // floor(W * u) for the draw's uniform u = (2 a + 1) / 2^25, exactly.
 __device__ __forceinline__ unsigned long long draw_target(unsigned long long W, uint32_t a_draw) {
     const unsigned long long mul = 2ull * a_draw + 1ull;

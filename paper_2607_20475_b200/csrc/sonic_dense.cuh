@@ -1020,10 +1020,91 @@ sonic_dense_finish_kernel(const KParams P, const int tiles) {
 
 // Stage 4 (verification calls): the residual max(0, p - q) of the positions whose draft was rejected.  The
 // support's total weight W is known here only in fixed point (relative error up to 1e-7 on peaked rows, too
-// coarse where p - q cancels), so a tile accumulates, in fp64, the residual sum R~ taken with that W~, the sum Pp of
-// the weights whose residual is positive, and the plain sum S of the weights; with W = sum of S the row's last
-// CTA corrects each tile's residual to R~ - (1/W~ - 1/W) * Pp (exact up to the elements whose residual changes
+// coarse where p - q cancels), so an item accumulates, in fp64, the residual sum R~ taken with that W~, the sum Pp of
+// the weights whose residual is positive, and the plain sum S of the weights; with W = sum of S the row's finish
+// corrects each tile's residual to R~ - (1/W~ - 1/W) * Pp (exact up to the elements whose residual changes
 // sign between W~ and W, each of which contributes less than 1e-7 of its own probability).
+// Weights: an element that carries more than 2^-7 of the support's mass (at most 128 per row, usually a handful) is
+// weighed with the fp64 exponential: its residual is a difference of two numbers of that size.  The others use an
+// fp32 exponential of relative error below 1e-7 with no bias; independent errors of that size on probabilities
+// below 2^-7 add up to less than 1e-8 in the cumulative sums.
+// The draft's probabilities of 16 consecutive elements (first a multiple of 16), independent of the keys: an element
+// outside the support has weight 0 and so a residual <= 0 whatever q is; indices past the row's end are clamped.
+__device__ __forceinline__ void resid_load_q(const float *q, int first, int V, float (&qv)[DENSE_EPT]) {
+    if (first + DENSE_EPT <= V && ((reinterpret_cast<uintptr_t>(q + first) & 15) == 0)) {
+        const float4 *s4 = reinterpret_cast<const float4 *>(q + first);
+#pragma unroll
+        for (int k = 0; k < DENSE_NV; ++k) {
+            const float4 v = __ldg(s4 + k);
+            qv[4 * k] = v.x; qv[4 * k + 1] = v.y; qv[4 * k + 2] = v.z; qv[4 * k + 3] = v.w;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < DENSE_EPT; ++e) qv[e] = __ldg(q + min(first + e, V - 1));
+    }
+}
+
+__device__ __forceinline__ double resid_weight(uint32_t key, float Mf, double Md, float big) {
+    const float y = unkey(key);
+    const float w32 = exp_accurate(__fsub_rn(y, Mf));
+    return (w32 > big) ? exp((double)y - Md) : (double)w32;
+}
+
+// The element of one tile at which the running sum of the residuals first exceeds `rest` (the tile's last element of
+// positive residual if rounding keeps the sum below it; -1 if the tile has none).  Whole CTA; a thread holds its 16
+// residuals in registers.
+__device__ int resid_tile_find(const KParams &P, int row, int tile, const float *q, unsigned long long cutc, float Mf, double Md,
+                               float big, double inv_W, double rest, DenseShared &sm, int tid) {
+    const int first = tile * CTA_TILE + tid * DENSE_EPT;
+    const uint4 *src = reinterpret_cast<const uint4 *>(P.ykeys + (size_t)row * ((size_t)P.ytiles * CTA_TILE) + first);
+    uint4 kv[DENSE_NV];
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) kv[k] = src[k];
+    float qv[DENSE_EPT];
+    resid_load_q(q, first, P.V, qv);
+    if (tid == 0) { sm.flag = -1; sm.digit = -1; }
+    double r[DENSE_EPT];
+    double s = 0.0;
+    int lastpos = -1;
+#pragma unroll
+    for (int k = 0; k < DENSE_NV; ++k) {
+        const uint32_t key4[4] = {kv[k].x, kv[k].y, kv[k].z, kv[k].w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e = 4 * k + u;
+            const bool in = (((unsigned long long)key4[u] << 32) | (uint32_t)(~(uint32_t)(first + e))) >= cutc;
+            const double w = in ? resid_weight(key4[u], Mf, Md, big) : 0.0;
+            const double v = w * inv_W - (double)qv[e];
+            r[e] = v > 0.0 ? v : 0.0;
+            s += r[e];
+            if (v > 0.0) lastpos = first + e;
+        }
+    }
+    double total;
+    const double pre = dense_block_scan<double>(s, sm.redd[0], tid, total);
+    if (s > 0.0 && pre <= rest && rest < pre + s) {
+        double cum = pre;
+        int found = -1;
+#pragma unroll
+        for (int e = 0; e < DENSE_EPT; ++e) {
+            cum += r[e];
+            if (r[e] > 0.0 && found < 0 && cum > rest) found = first + e;
+        }
+        sm.flag = found < 0 ? lastpos : found;
+    }
+    __syncthreads();
+    if (sm.flag < 0) {
+        if (lastpos >= 0) atomicMax(&sm.digit, lastpos);
+        __syncthreads();
+        if (tid == 0) sm.flag = sm.digit;
+        __syncthreads();
+    }
+    const int res = sm.flag;
+    __syncthreads();
+    return res;
+}
+
+// One CTA's items: contiguous ranges over the rows of the residual list, a tile per item.
 __global__ void __launch_bounds__(DENSE_THREADS, 2)
 sonic_dense_resid_kernel(const KParams P, const int tiles) {
     __shared__ DenseShared sm;
@@ -1032,19 +1113,33 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
     pdl_wait_primary();
     KERNEL_T0(4);
     const int nr = (int)__ldcg(&P.error[WS_NRESID]);
-    for (int item = blockIdx.x; item < nr * tiles; item += gridDim.x) {
+    const DenseRange rg = dense_range(nr * tiles, (int)blockIdx.x, (int)gridDim.x);
+    int cur_row = -1;
+    unsigned long long cutc = 0ull;
+    float Mf = 0.0f, big = 0.0f;
+    double Md = 0.0, inv_Wt = 0.0;
+    const float *q = nullptr;
+    for (int item = rg.lo; item < rg.hi; ++item) {
         const DenseItem it = dense_item(P.rlist, item, tiles, 1);
         const int row = it.row, tile = it.tile;
-        DenseRow *dr = P.drow + row;
-        DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
         uint4 kv[DENSE_NV];
         dense_load_keys(P, it, tid, kv);
-        const RowCfg c = load_cfg(P, row);
-        const unsigned long long cutc = __ldcg(&dr->cutc), Wq = __ldcg(&dr->W);
-        const uint32_t Mkey = __ldcg(&dr->Mkey);
-        const double Md = (double)unkey(Mkey);
-        const double inv_Wt = 1099511627776.0 / (double)Wq;                 // 1 / W~
-        const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)P.V;
+        {
+            const int b = row / (P.K + 1), l = row - b * (P.K + 1);
+            q = P.draft_probs + ((size_t)b * P.K + l) * (size_t)P.V;
+        }
+        float qv[DENSE_EPT];
+        resid_load_q(q, tile * CTA_TILE + tid * DENSE_EPT, P.V, qv);
+        if (row != cur_row) {
+            cur_row = row;
+            const DenseRow *dr = P.drow + row;
+            cutc = __ldcg(&dr->cutc);
+            const unsigned long long Wq = __ldcg(&dr->W);
+            Mf = unkey(__ldcg(&dr->Mkey));
+            Md = (double)Mf;
+            inv_Wt = 1099511627776.0 / (double)Wq;                      // 1 / W~
+            big = (float)((double)Wq * (1.0 / 1099511627776.0) * (1.0 / 128.0));
+        }
         double R = 0.0, Pp = 0.0, S = 0.0;
 #pragma unroll
         for (int k = 0; k < DENSE_NV; ++k) {
@@ -1052,11 +1147,10 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
             const int base_idx = tile * CTA_TILE + tid * DENSE_EPT + 4 * k;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                // (no branch per element: the sixteen chains of a thread overlap)
                 const int idx = base_idx + u;
                 const bool in = (((unsigned long long)key4[u] << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc;
-                const double w = in ? exp((double)unkey(key4[u]) - Md) : 0.0;
-                const double r = w * inv_Wt - (double)(in ? __ldg(q + idx) : 0.0f);
+                const double w = in ? resid_weight(key4[u], Mf, Md, big) : 0.0;
+                const double r = w * inv_Wt - (double)qv[4 * k + u];
                 S += w;
                 R += (r > 0.0) ? r : 0.0;
                 Pp += (r > 0.0) ? w : 0.0;
@@ -1074,10 +1168,37 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
         if (tid == 0) {
             double r = 0.0, p = 0.0, s = 0.0;
             for (int w = 0; w < DENSE_WARPS; ++w) { r += sm.redd[0][w]; p += sm.redd[1][w]; s += sm.redd[2][w]; }
-            dt[tile].R = r; dt[tile].Pp = p; dt[tile].S = s;
+            DenseTile *dt = P.dtile + (size_t)row * MAX_TILES + tile;
+            dt->R = r; dt->Pp = p; dt->S = s;
         }
-        if (!dense_arrive(&dr->ticket_r, 1, tiles, sm, tid)) continue;
-        // ---- the row's last CTA: corrected tile residuals, the tile of the draw, the element
+        __syncthreads();
+    }
+    KERNEL_T1(4);
+}
+
+// The residual draw, one CTA per row of the residual list (a programmatic dependent of the kernel above).
+__global__ void __launch_bounds__(DENSE_THREADS)
+sonic_dense_resid_finish_kernel(const KParams P, const int tiles) {
+    __shared__ DenseShared sm;
+    const int tid = threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait_primary();
+    KERNEL_T0(9);
+    const int nr = (int)__ldcg(&P.error[WS_NRESID]);
+    for (int i = blockIdx.x; i < nr; i += gridDim.x) {
+        const int row = __ldcg(&P.rlist[i]);
+        DenseRow *dr = P.drow + row;
+        DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
+        const RowCfg c = load_cfg(P, row);
+        const unsigned long long cutc = __ldcg(&dr->cutc), Wq = __ldcg(&dr->W);
+        const uint32_t Mkey = __ldcg(&dr->Mkey);
+        const float Mf = unkey(Mkey);
+        const double Md = (double)Mf;
+        const double inv_Wt = 1099511627776.0 / (double)Wq;
+        const float big = (float)((double)Wq * (1.0 / 1099511627776.0) * (1.0 / 128.0));
+        const float *q = P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)P.V;
+        uint32_t a_acc, a_draw;
+        draw_cells(P, c, a_acc, a_draw);
         if (tid < 32) {
             // a tile's three sums per lane (one round of loads), added up in tile order by every lane alike
             double sj = 0.0, rj0 = 0.0, pj = 0.0;
@@ -1094,8 +1215,6 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
         }
         __syncthreads();
         const double Wd = sm.bcd[0], Rtot = sm.bcd[1];
-        uint32_t a_acc, a_draw;
-        draw_cells(P, c, a_acc, a_draw);
         int token = -1;
         if (Rtot > 0.0) {
             const double target = cell_to_u(a_draw) * Rtot;
@@ -1108,14 +1227,8 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
             }
             if (jt < 0) { cum = 0.0; for (int j = 0; j < tiles; ++j) { if (rj[j] > 0.0) { jt = j; before = cum; } cum += rj[j]; } }
             const double inv_Wd = 1.0 / Wd;
-            auto wf = [=](uint32_t key, int idx) -> double {
-                const bool in = (((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc;
-                const double r = (in ? exp((double)unkey(key) - Md) : 0.0) * inv_Wd - (double)(in ? __ldg(q + idx) : 0.0f);
-                return r > 0.0 ? r : 0.0;
-            };
-            double rw;
             __syncthreads();
-            if (jt >= 0) token = dense_tile_find<double>(P, row, jt, target - before, wf, sm.redd[0], sm, tid, rw);
+            if (jt >= 0) token = resid_tile_find(P, row, jt, q, cutc, Mf, Md, big, inv_Wd, target - before, sm, tid);
         }
         if (token < 0) {
             // empty residual (p <= q on the whole support, by rounding): draw from p itself
@@ -1128,7 +1241,6 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
                 if (!hit && t > 0ull && cum + t > T) { jt = j; before = cum; hit = true; }
                 cum += t;
             }
-            const float Mf = unkey(Mkey);
             auto wf = [=](uint32_t key, int idx) -> unsigned long long {
                 const unsigned long long wq = qweight(key, Mf);
                 return ((((unsigned long long)key << 32) | (uint32_t)(~(uint32_t)idx)) >= cutc) ? wq : 0ull;
@@ -1139,8 +1251,8 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
         }
         if (tid == 0) emit_row(P, c, row, token, 0.0f, F_DENSE, __ldcg(&dr->support), __ldcg(&dr->p_draft));
         __syncthreads();
-        KERNEL_T1(4);
     }
+    KERNEL_T1(9);
 }
 
 }  // namespace sonic
