@@ -5,8 +5,11 @@ A "step" is one fused call (sonic_sample on the heterogeneous-batch workload c2
 by default) over one batch of seeded synthetic input.  Inputs rotate over enough
 distinct copies that their total footprint exceeds twice the L2 capacity, so
 every call reads its logits from HBM.  Calls are captured in CUDA graphs and
-timed with CUDA events on the launching stream; with N > 1 (torchrun) every rank
-runs an independent replica on its own GPU and the slowest rank's time counts.
+timed with CUDA events on the launching stream: a timed block is exactly
+`--steps` calls, and blocks are repeated until `--min-time-ms` of device time has
+been measured (mean and minimum over the blocks are printed).  With N > 1
+(torchrun) every rank runs an independent replica on its own GPU and the slowest
+rank's time counts.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
@@ -29,9 +32,35 @@ if ROOT not in sys.path:
 from paper_2607_20475_b200 import workloads as wl  # noqa: E402
 
 METRIC = "us_per_fused_sample_call"
-# DRAM bytes (read + write) of one call's kernels from the ncu captures summarised under profiles/ (per workload)
-NCU_TRAFFIC = {"c2": 17.93e6, "c3": 143.1e6}
 L2_BYTES = 126 * 1024 * 1024
+PROFILE_TRAFFIC = os.path.join(ROOT, "profiles", "dram_traffic_per_call.txt")
+
+
+def profiled_traffic(name: str):
+    """DRAM bytes (read + write) of one call's kernels and their serialised times, from the ncu summary committed
+    under profiles/ (lines `<workload> total <bytes>` and `<workload> kernel <name> <launches per call> <us> <bytes>`).
+    Returns (bytes or None, {kernel: {...}}, source file or None)."""
+    if not os.path.exists(PROFILE_TRAFFIC):
+        return None, {}, None
+    total, kernels = None, {}
+    for ln in open(PROFILE_TRAFFIC):
+        f = ln.split()
+        if len(f) >= 3 and f[0] == name and f[1] == "total":
+            total = float(f[2])
+        elif len(f) >= 6 and f[0] == name and f[1] == "kernel":
+            kernels[f[2]] = {"launches_per_call": float(f[3]), "us_per_call_under_ncu": float(f[4]), "dram_bytes_per_call": float(f[5])}
+    return total, kernels, os.path.relpath(PROFILE_TRAFFIC, ROOT)
+
+
+def launches_per_call(name: str, w) -> int:
+    """Kernels one call enqueues.  Sampling: streaming, merge, histogram pass, collect pass, row finish, cluster kernel.
+    Verification adds the residual pass, the residual draw and the combine kernel.  (sonic_topk: streaming, merge,
+    cluster kernel.)"""
+    if name == "c4":
+        return 9 if w.K > 0 else 7
+    if name.startswith("c5"):
+        return 3
+    return 6
 
 
 def peaks():
@@ -255,6 +284,10 @@ def build_device_copies(name, copies, binding):
             if ws is None:
                 ws = binding.new_workspace(w.B, w.V)
             devs.append(binding.DeviceSample(w, ws=ws))
+    # one eager call per copy: results exist for the row counts, and nothing of the library is set up for the
+    # first time inside a capture
+    for d in devs:
+        d.run()
     torch.cuda.synchronize()
     return devs
 
@@ -270,6 +303,7 @@ def capture(devs, calls):
 
 
 def time_graph_steps(graph_full, per_graph, graph_rem, rem, steps):
+    """Device time (s) of exactly `steps` calls: CUDA events on the launching stream, synchronised on both sides."""
     import torch
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -281,6 +315,15 @@ def time_graph_steps(graph_full, per_graph, graph_rem, rem, steps):
     end.record()
     torch.cuda.synchronize()
     return start.elapsed_time(end) / 1000.0
+
+
+def time_blocks(graph_full, per_graph, graph_rem, rem, steps, min_time_s, max_blocks=400):
+    """Timed blocks of exactly `steps` calls each, repeated until their device time adds up to `min_time_s`.
+    Returns the list of block times (s)."""
+    blocks = [time_graph_steps(graph_full, per_graph, graph_rem, rem, steps)]
+    while sum(blocks) < min_time_s and len(blocks) < max_blocks:
+        blocks.append(time_graph_steps(graph_full, per_graph, graph_rem, rem, steps))
+    return blocks
 
 
 def time_graph_min(graph, per_graph, reps=12):
@@ -317,10 +360,14 @@ def time_warm_l2(dev, calls=8, reps=12):
 
 
 def fallback_rows(name, devs):
-    """Rows (requests for c4) per call, over the input copies, that report the exact kernel (diagnostic flag bit 2)."""
-    per_copy = [int((d.results()["flags"][:(d.vw.B if name == "c4" else None)] & 4).astype(bool).sum()) for d in devs]
-    return {"mean_per_call": float(np.mean(per_copy)), "max_per_call": int(max(per_copy)),
-            "unit": "requests" if name == "c4" else "rows"}
+    """Rows (requests for c4) per call, over the input copies, that report the cluster kernel (diagnostic flag bit 2)
+    and the histogram path (bit 3)."""
+    out = {}
+    for key, bit in (("cluster", 4), ("dense", 8)):
+        per_copy = [int((d.results()["flags"][:(d.vw.B if name == "c4" else None)] & bit).astype(bool).sum()) for d in devs]
+        out[key] = {"mean_per_call": float(np.mean(per_copy)), "max_per_call": int(max(per_copy)),
+                    "unit": "requests" if name == "c4" else "rows"}
+    return out
 
 
 def measure_floor(calls=64, reps=20):
@@ -434,18 +481,30 @@ def run_sonic(args, rank, world, local_rank):
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    elapsed = time_graph_steps(g_full, per_graph, g_rem, rem, steps)
+    if args.profile_run:
+        args.min_time_ms = 0.0
+    blocks = time_blocks(g_full, per_graph, g_rem, rem, steps, args.min_time_ms / 1000.0)
     # keep the sampler busy long enough to see clocks under load
-    t_end = time.time() + 0.6
+    t_end = time.time() + (0.3 if args.min_time_ms > 0 else 0.0)
     while rank == 0 and time.time() < t_end:
         g_full.replay()
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    elapsed = max_over_ranks(elapsed, world, "cuda")
+    # every rank's mean over its blocks; the job's time is the slowest rank's
+    elapsed = max_over_ranks(float(np.mean(blocks)), world, "cuda")
     clocks = sampler.stop() if rank == 0 else None
 
-    us_call = elapsed / steps * 1e6                     # per replica
+    us_call = elapsed / steps * 1e6                     # per replica, mean over the blocks
+    us_call_best_block = min(blocks) / steps * 1e6
+    if args.profile_run:
+        # under a profiler: the timed calls only (no end-to-end leg, probes or CPU baseline), a short line
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": job_value(us_call, world), "unit": "us", "steps": steps,
+                              "profile_run": True, "config": config_dict(name, w0, copies, bytes_call, world)}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     e2e_us, h2d, d2h = e2e_measure(name, devs[0], steps=min(steps, 40))
     e2e_us = max_over_ranks(e2e_us, world, "cuda")
     floor_us = measure_floor() if rank == 0 else None
@@ -463,7 +522,9 @@ def run_sonic(args, rank, world, local_rank):
         B = w0.B
         rows = B * (w0.K + 1) if name == "c4" else B
         achieved = bytes_call / (us_call * 1e-6) / 1e9
-        launches_per_call = 5 if name == "c4" else 4     # exact (first round), stream, merge, exact (second round) [, verify combine]
+        n_launch = launches_per_call(name, w0)
+        traffic, per_kernel, traffic_src = profiled_traffic(name)
+        in_dtype = "bf16" if w0_dtype(w0) == wl.DTYPE_BF16 else "f32"
         cpu_us, cpu_desc, cpu_rows, cpu_near = oracle_time(name, w0, budget_s=15.0)
         cpu_all = oracle_time_all_cores(name, w0, budget_s=6.0)
         probe = read_probe()
@@ -471,26 +532,35 @@ def run_sonic(args, rank, world, local_rank):
             "metric": METRIC, "value": job_value(us_call, world), "unit": "us", "n_gpus": world, "steps": steps,
             "warmup": max(3, args.warmup), "ms_per_step": us_call / 1000.0, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
+            "dtype": "f32", "input_dtype": in_dtype, "data": "synthetic",
             "config": config_dict(name, w0, copies, bytes_call, world),
+            "timed": {"blocks": len(blocks), "calls_per_block": steps, "device_ms_total": sum(blocks) * 1e3,
+                      "us_per_call_mean": us_call, "us_per_call_min_block": us_call_best_block,
+                      "note": "value is the mean over the blocks; every block is exactly `steps` calls between two CUDA events"},
             "rows_per_s": rows * world / (us_call * 1e-6),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC.get(name), "peak_source": which, "kernel": "whole call",
-                         "note": "algorithmic bytes of the call / CUDA-event time of the whole call (stream, merge and both "
-                                 "launches of the exact kernel, overlapped through a forked side stream and programmatic "
-                                 "dependent launch); the per-kernel split is in profiles/"},
+                         "traffic": traffic, "algorithmic_bytes": int(bytes_call), "measured_dram_bytes": traffic,
+                         "measured_dram_bytes_source": traffic_src, "peak_source": which, "kernel": "whole call",
+                         "dominant_kernel": "sonic_stream_kernel",
+                         "per_kernel": per_kernel,
+                         "note": "achieved = algorithmic bytes of the call (logits + mask words + lists, read once) / CUDA-event "
+                                 "time of the whole call: the streaming kernel moves the bytes, the merges and the histogram "
+                                 "passes of the same call run behind it, partly beside each other on a forked stream, "
+                                 "so a call has no single kernel's duration.  per_kernel: serialised "
+                                 "times and DRAM bytes under ncu from the committed profile (compare shares)."},
             "cpu_baseline": {"value": cpu_us, "unit": "us", "cores": 1, "kind": "oracle", "sample": cpu_desc},
             "cpu_baseline_all_cores": None if cpu_all is None else
                 {"value": cpu_all[0], "unit": "us", "cores": cpu_all[1], "kind": "oracle", "sample": cpu_all[2]},
             "read_probe": dict(probe, frac_of_read_probe=achieved / probe["gbs"]),
             "e2e": {"value": job_value(e2e_us, world), "unit": "us", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
-            "gpu_launches": launches_per_call * steps,
+            "gpu_launches": n_launch * steps * len(blocks),
+            "gpu_launches_per_call": n_launch,
             "empty_graph_node_us": floor_us,
             "us_per_call_min": min_us,
             "warm_l2": {"us_per_call": warm_us, "input_fits_l2": bool(bytes_call < L2_BYTES),
                         "note": "one input copy replayed back to back"},
-            "rows": {"per_call": rows, "exact_kernel": fb,
-                     "near_margin": {"count": cpu_near, "of": cpu_rows, "unit": fb["unit"],
+            "rows": {"per_call": rows, "cluster_kernel": fb["cluster"], "histogram_path": fb["dense"],
+                     "near_margin": {"count": cpu_near, "of": cpu_rows, "unit": fb["cluster"]["unit"],
                                      "note": "decision margin below 1e-6 in the oracle, on the cpu_baseline sample"}},
             "clocks": clocks,
             "also": extra,
@@ -532,9 +602,51 @@ def quick_topk(k, binding, reps=10):
             "frac": nbytes / us / 1e3 / peak, "copies": 2, "k": k}
 
 
+def topk_all(binding, min_time_s=0.05):
+    """sonic_topk on all of configuration 5: three regimes x six k (B=256, V=262144, fp32; two input copies > 2x L2)."""
+    import torch
+    peak, _ = peaks()
+    table = {}
+    for regime in wl.TOPK_REGIMES:
+        tw = wl.config5(regime)
+        ws = binding.new_workspace(tw.B, tw.V)
+        first = binding.DeviceTopK(tw, 1, ws=ws)
+        second_logits = first.logits.clone()
+        nbytes = tw.logits.nbytes
+        for k in wl.TOPK_KS:
+            devs = [binding.DeviceTopK(tw, k, ws=ws, logits=first.logits), binding.DeviceTopK(tw, k, ws=ws, logits=second_logits)]
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for d in devs:
+                    d.run()
+            for _ in range(3):
+                g.replay()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps, total = 0, 0.0
+            torch.cuda.synchronize()
+            while total < min_time_s and reps < 400:
+                s.record()
+                for _ in range(5):
+                    g.replay()
+                e.record()
+                torch.cuda.synchronize()
+                total += s.elapsed_time(e) * 1e-3
+                reps += 5
+            us = total * 1e6 / (reps * 2)
+            table[f"{regime}_k{k}"] = {"us_per_call": round(us, 2), "achieved_gbs": round(nbytes / us / 1e3, 1),
+                                       "frac": round(nbytes / us / 1e3 / peak, 4)}
+            del devs, g
+        del first, second_logits, ws
+        torch.cuda.empty_cache()
+    return {"workload": "c5: sonic_topk, B=256, V=262144, fp32, regimes x k", "algorithmic_bytes": int(nbytes),
+            "copies": 2, "table": table}
+
+
 def quick_measure(name, binding, reps=30):
     """Short cold-input timing of another configuration (not the headline line)."""
     import torch
+    if name == "c5":
+        return topk_all(binding)
     if name.startswith("c5k"):
         return quick_topk(int(name[3:]), binding)
     w0 = make_workload(name)
@@ -542,22 +654,27 @@ def quick_measure(name, binding, reps=30):
     copies = int(min(8, max(2, np.ceil(2.0 * L2_BYTES / bytes_call))))
     devs = build_device_copies(name, copies, binding)
     g = capture(devs, copies)
-    for _ in range(2):
+    for _ in range(3):
         g.replay()
     s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    blocks = []
     torch.cuda.synchronize()
-    s.record()
-    for _ in range(reps):
-        g.replay()
-    e.record()
-    torch.cuda.synchronize()
-    us = s.elapsed_time(e) * 1000.0 / (reps * copies)
+    while sum(blocks) < 0.1 and len(blocks) < 200:           # >= 100 ms of device time
+        s.record()
+        for _ in range(reps):
+            g.replay()
+        e.record()
+        torch.cuda.synchronize()
+        blocks.append(s.elapsed_time(e) * 1e-3)
+    us = float(np.mean(blocks)) * 1e6 / (reps * copies)
     peak, which = peaks()
     gbs = bytes_call / (us * 1e-6) / 1e9
+    traffic, per_kernel, src = profiled_traffic(name)
     del devs, g
     torch.cuda.empty_cache()
-    return {"us_per_call": us, "algorithmic_bytes": int(bytes_call), "achieved_gbs": gbs, "frac": gbs / peak,
-            "copies": copies}
+    return {"us_per_call": us, "us_per_call_min_block": min(blocks) * 1e6 / (reps * copies), "blocks": len(blocks),
+            "algorithmic_bytes": int(bytes_call), "measured_dram_bytes": traffic, "achieved_gbs": gbs, "frac": gbs / peak,
+            "copies": copies, "gpu_launches_per_call": launches_per_call(name, w0)}
 
 
 def run_sweep():
@@ -606,7 +723,12 @@ def main():
     ap.add_argument("--impl", default="sonic", choices=["sonic", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4"])
     ap.add_argument("--sweep", action="store_true", help="time the V x B x entropy x dtype sweep instead (one GPU)")
-    ap.add_argument("--also", default="c1,c3,c4,c5k1,c5k64", help="other configurations to time briefly (comma separated, '' for none)")
+    ap.add_argument("--min-time-ms", type=float, default=500.0,
+                    help="repeat the timed block of --steps calls until this much device time is measured (0: one block)")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="run the warm-up and one timed block only and print a short line (for use under ncu; never a bench value)")
+    ap.add_argument("--also", default="c1,c3,c4,c5", help="other configurations to time briefly (comma separated, '' for none; "
+                    "c5 = sonic_topk over all regimes and k, c5k<k> = one k of the 'normal' regime)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -18,8 +18,9 @@
  *   0x200 min-p                 0x400 top-k log-probabilities (reserved, ignored)
  * A parameter array may be NULL when no request sets the bit that reads it.
  * Parameter domains: tau > 0 finite; k >= 0; p, theta in (0, 1]; rep_penalty alpha > 0 finite (the paper states
- * alpha >= 1), freq_penalty and pres_penalty finite (the paper states >= 0), bias values finite; a set bit with a
- * parameter outside its domain gives SONIC_FLAG_BADPARAM for that row.
+ * alpha >= 1), freq_penalty and pres_penalty finite (the paper states >= 0); a set bit with a parameter outside
+ * its domain gives SONIC_FLAG_BADPARAM for that row (greedy rows too, for tau and the penalty coefficients).
+ * Bias values and logits must not be NaN or +inf (a precondition, not checked; -inf logits are masked entries).
  */
 #ifndef SONIC_H
 #define SONIC_H
@@ -68,7 +69,16 @@ size_t sonic_workspace_bytes(int max_rows, int max_vocab, int max_topk);
  * (a tile copy that never completed) ran out.  Every row of such a call, and of later calls on that workspace,
  * reports SONIC_FLAG_TIMEOUT with token -1 until the workspace is initialised again with this function.
  *
- * Streams: every kernel of a call is enqueued on the caller's `stream`; the library creates no stream or event. */
+ * Streams: a call's kernels are ordered on the caller's `stream` (everything enqueued before the call precedes
+ * them, everything after follows them).  Per host thread and device the library keeps ONE internal non-blocking stream
+ * and two events, created by this function or by the thread's first sampling call outside a stream capture:
+ * sonic_sample / sonic_verify fork it from `stream` behind their first kernel and join it back before their last
+ * one, so that rows with and without top-k are finished side by side.  Under stream capture the fork is captured
+ * with the caller's stream (one graph, no dependency outside it).  Whenever the internal stream cannot be used -
+ * it does not exist yet and the caller is capturing, or it still belongs to another capture that is open - the
+ * call runs all of its kernels on `stream` alone: same results, about a third slower on mixed batches.  So: call
+ * this function (or one eager sampling call) on a thread before that thread captures, and do not keep two captures
+ * open on one thread at the same time if both should get the two-stream schedule.  sonic_topk uses no other stream. */
 int sonic_workspace_init(void *workspace, size_t bytes, void *stream);
 
 /*

@@ -305,6 +305,11 @@ static int bad_params(const oracle_args *a, int b)
 {
     uint32_t z = a->mode[b];
     if (z & ORACLE_TEMPERATURE) { float t = a->temperature[b]; if (!(t > 0.0f) || !isfinite(t)) return 1; }
+    /* penalty coefficients (Appendix "Repetition Penalties": alpha >= 1, beta >= 0, gamma >= 0): a divisor that is
+     * not positive and finite, or a coefficient that is not finite, is outside the domain like any other parameter */
+    if (z & ORACLE_REPETITION) { float al = a->rep_penalty[b]; if (!(al > 0.0f) || !isfinite(al)) return 1; }
+    if ((z & ORACLE_FREQUENCY) && !isfinite(a->freq_penalty[b])) return 1;
+    if ((z & ORACLE_PRESENCE) && !isfinite(a->pres_penalty[b])) return 1;
     if (z & ORACLE_GREEDY) return 0;
     if ((z & ORACLE_TOP_K) && a->top_k[b] < 0) return 1;
     if (z & ORACLE_TOP_P) { float p = a->top_p[b]; if (!(p > 0.0f && p <= 1.0f)) return 1; }

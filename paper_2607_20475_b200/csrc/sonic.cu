@@ -369,6 +369,12 @@ int sonic_workspace_init(void *workspace, size_t bytes, void *stream) {
     if (bytes < layout_for(1, 1, true).total) return fail(SONIC_EWORKSPACE, "workspace smaller than one row");
     cudaError_t e = cudaMemsetAsync(workspace, 0, WS_HEADER, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail_cuda(e, "cudaMemsetAsync");
+    // The calling thread's internal stream is created here already (if this is not inside a capture), so that a
+    // thread whose very first sampling call is captured still gets the two-stream schedule.  Best effort: a call
+    // that finds no usable internal stream runs on the caller's stream alone.
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) (void)side_stream_for(dev, (cudaStream_t)stream);
+    else cudaGetLastError();
     g_err[0] = 0;
     return SONIC_OK;
 }

@@ -300,6 +300,11 @@ __device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const C
     c.bias_len = (z & M_BIAS) ? min(max(v_bl, 0), P.bias_stride) : 0;
     bool greedy = (z & M_GREEDY) != 0;
     if (c.temp && !(c.tau > 0.0f && c.tau < CUDART_INF_F)) c.bad = true;
+    // penalty coefficients (Appendix "Repetition Penalties" states alpha >= 1 and beta, gamma >= 0): a divisor that is not
+    // positive and finite, or a coefficient that is not finite, would turn logits into NaN or +-inf
+    if ((z & M_REPETITION) && !(c.alpha > 0.0f && c.alpha < CUDART_INF_F)) c.bad = true;
+    if ((z & M_FREQUENCY) && !(fabsf(c.beta) < CUDART_INF_F)) c.bad = true;
+    if ((z & M_PRESENCE) && !(fabsf(c.gamma) < CUDART_INF_F)) c.bad = true;
     if (!greedy) {
         if ((z & M_TOP_K) && c.k < 0) c.bad = true;
         if ((z & M_TOP_P) && !(c.p > 0.0f && c.p <= 1.0f)) c.bad = true;

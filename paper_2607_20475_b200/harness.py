@@ -131,10 +131,11 @@ class DeviceVerify:
 
 
 class DeviceTopK:
-    def __init__(self, tw: wl.TopKWorkload, k: int, device="cuda", ws: Optional[torch.Tensor] = None):
+    def __init__(self, tw: wl.TopKWorkload, k: int, device="cuda", ws: Optional[torch.Tensor] = None,
+                 logits: Optional[torch.Tensor] = None):
         self.tw = tw
         self.k = k
-        self.logits = _dev(_padded_logits(tw.logits, tw.dtype), device)
+        self.logits = _dev(_padded_logits(tw.logits, tw.dtype), device) if logits is None else logits   # (shared between holders of several k)
         self.out_vals = torch.zeros((tw.B, k), dtype=torch.float32, device=device)
         self.out_idx = torch.full((tw.B, k), -7, dtype=torch.int32, device=device)
         self.ws = new_workspace(tw.B, tw.V, device) if ws is None else ws

@@ -135,6 +135,25 @@ def test_edge_rows(sonic, oracle):
     assert got["token"][3] == 7 and got["token"][9] == 0 and got["token"][2] == 12345
 
 
+def test_penalty_coefficients_outside_their_domain(sonic, oracle):
+    # Appendix "Repetition Penalties": alpha >= 1, beta >= 0, gamma >= 0.  A divisor that is not positive and finite, or a
+    # coefficient that is not finite, is a bad parameter (greedy rows too); a clear bit hides any value
+    V = 9000
+    rng = np.random.default_rng(12)
+    x = rng.standard_normal((9, V)).astype(np.float32) * 2
+    inf, nan = np.inf, np.nan
+    R, F, Pn = wl.REPETITION, wl.FREQUENCY, wl.PRESENCE
+    mode = [R | wl.TOP_K, R | wl.GREEDY, R | wl.TOP_P, F | wl.TOP_K, Pn | wl.MIN_P, F | wl.GREEDY, wl.TOP_K, R | F | Pn | wl.TOP_K, R | wl.TOP_K]
+    w = make_sample(x, mode, top_k=[5, 0, 0, 7, 0, 0, 5, 9, 5], top_p=[1, 1, .8, 1, 1, 1, 1, 1, 1], min_p=[0, 0, 0, 0, .1, 0, 0, 0, 0],
+                    rep=[0.0, -2.0, nan, 1.0, 1.0, 1.0, nan, 0.5, inf], freq=[0, 0, 0, inf, 0, nan, inf, -0.25, 0],
+                    pres=[0, 0, 0, 0, -inf, 0, nan, -0.5, 0],
+                    hist=[{3: 1, 77: 2}] * 9, seed=np.arange(9) + 40)
+    got, ref, n = run_sample(sonic, oracle, w)
+    bad = (got["flags"] & 2) != 0
+    assert list(bad) == [True, True, True, True, True, True, False, False, True]
+    assert np.all(got["token"][bad] == -1)
+
+
 def test_temperature_ties_in_topk(sonic, oracle):
     # distinct logits that collide after the temperature division: the boundary group of the top-k
     # must be broken by index exactly as the definition does

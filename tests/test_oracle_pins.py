@@ -283,6 +283,21 @@ def test_no_token_and_bad_parameters():
     assert out["flags"].tolist() == [1, 0, 2]
 
 
+def test_penalty_coefficients_outside_their_domain_are_bad_parameters():
+    # Appendix "Repetition Penalties" states alpha >= 1, beta >= 0, gamma >= 0; a coefficient that would make a logit NaN
+    # or infinite (divisor not positive and finite, coefficient not finite) is reported like any bad parameter,
+    # for greedy rows as well; a clear mode bit hides the value
+    x = np.linspace(-1.0, 1.0, 12, dtype=np.float32)[None, :].repeat(7, 0)
+    R, F, Pn = wl.REPETITION, wl.FREQUENCY, wl.PRESENCE
+    out = oracle.sample(make_sample(x, [R | wl.GREEDY, R, F | wl.GREEDY, Pn, wl.GREEDY, R | F | Pn | wl.GREEDY, R | wl.GREEDY],
+                                    rep=[0.0, np.nan, 1.0, 1.0, np.nan, 0.5, np.inf], freq=[0, 0, np.inf, 0, np.inf, -1.0, 0],
+                                    pres=[0, 0, 0, np.nan, np.nan, -1.0, 0], hist=[{11: 1}] * 7))
+    assert out["flags"].tolist() == [2, 2, 2, 2, 0, 0, 2]
+    assert out["token"].tolist()[:4] == [-1, -1, -1, -1] and out["token"][4] == 11 and out["token"][6] == -1
+    # row 5: alpha = 0.5 is inside (0, inf): x[11] = 1.0 / 0.5 + 1 + 1 = 4
+    assert out["token"][5] == 11
+
+
 # ----------------------------------------------------------- verification
 def _verify_workload(p_rows, q_rows, drafts, mode, seed, **kw):
     """p_rows [B, K+1, V] target probabilities, q_rows [B, K, V] draft probabilities."""
