@@ -59,6 +59,7 @@ constexpr int WS_NDENSE = 4;                   // rows of the current call on th
 constexpr int WS_NRESID = 5;                   // verification rows of the current call whose draft was rejected (length of the residual list)
 constexpr int WS_EXACT_LEFT = 6;               // clusters of the cluster kernel that have run out of rows
 constexpr int WS_NEXACT = 7;                   // rows of the current call that belong to the cluster kernel by class
+constexpr int WS_TEST_WITHHOLD = 100;          // test-only builds (SONIC_TEST_WITHHOLD): 1 + the work item whose tile copy is withheld
 constexpr int WS_HEADER_WORDS = 128;
 constexpr uint32_t ST_FAILED = 0x1;           // streaming / histogram path could not finish the row
 constexpr unsigned int ERR_TIMEOUT = 0x1;     // workspace header: a bounded mbarrier wait expired

@@ -1046,6 +1046,22 @@ sonic_exact_kernel(const KParams P) {
     const int nwords = (P.rows + 31) >> 5;
     // (the passes that read the two lists are complete: their lengths go back to zero for the next call)
     if (blockIdx.x == 0 && x.tid == 0) { P.error[WS_NDENSE] = 0u; P.error[WS_NRESID] = 0u; }
+    if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {
+        // A bounded wait of the streaming kernel ran out (in this call or an earlier one on this workspace): nothing
+        // the call computed is to be trusted.  This is the call's last kernel over the rows, behind both chains, so
+        // here every row is made to say so (rows whose first tile was never processed are on no other path's list).
+        for (int row = blockIdx.x * EX_THREADS + x.tid; row < P.rows; row += gridDim.x * EX_THREADS) {
+            if (P.op == OP_TOPK) {
+                for (int j = 0; j < P.ktop; ++j) { P.out_vals[(size_t)row * P.ktop + j] = -CUDART_INF_F; P.out_idx[(size_t)row * P.ktop + j] = -1; }
+            } else {
+                RowCfg c0;
+                c0.b = row; c0.l = 0;
+                emit_row(P, c0, row, -1, 0.0f, F_TIMEOUT, 0, 0.0f);
+            }
+        }
+        KERNEL_T1(2);
+        return;
+    }
     // both counters stay as they are until the last cluster has left (below), so every CTA reads the same values
     if (__ldcg(&P.error[WS_FAILED_ROWS]) == 0u && __ldcg(&P.error[WS_NEXACT]) == 0u) { KERNEL_T1(2); return; }
     for (int i = x.tid; i < nwords; i += EX_THREADS) need[i] = 0u;

@@ -36,7 +36,10 @@ template <> struct VecTraits<0> { static constexpr int VEC = 4, NV = 8, NSTAGE =
 template <> struct VecTraits<1> { static constexpr int VEC = 8, NV = 4, NSTAGE = 2, ELT = 2; };
 
 constexpr int STREAM_CTA_THREADS = STREAM_THREADS + 32;      // eight consumer warps + the producer warp
-constexpr unsigned int WAIT_LIMIT = 1u << 22;                // try_wait rounds before a wait gives up
+#ifndef SONIC_WAIT_LIMIT
+#define SONIC_WAIT_LIMIT (1u << 22)
+#endif
+constexpr unsigned int WAIT_LIMIT = SONIC_WAIT_LIMIT;        // try_wait rounds before a wait gives up (a test-only build shortens it)
 
 // ---------------------------------------------------------------- mbarrier / bulk-copy primitives
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -1047,6 +1050,11 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             const unsigned char *src = reinterpret_cast<const unsigned char *>(P.logits) +
                                        ((size_t)row * (size_t)P.row_stride + (size_t)first) * ELT;
             if (arrive) mbar_arrive_expect_tx(&sh.full[s], bytes); else mbar_expect_tx(&sh.full[s], bytes);
+#ifdef SONIC_TEST_WITHHOLD
+            // test-only build: the bytes of one chosen tile are announced but its copy is never issued, so the waits
+            // on this stage run out (consumers, then the producer) and the call reports it
+            if (__ldcg(&P.error[WS_TEST_WITHHOLD]) == (unsigned int)(row * tiles + tile) + 1u) return;
+#endif
             bulk_load(stages + (size_t)s * STAGE_BYTES, src, bytes, &sh.full[s], l2_policy);
         };
         // The CTA's first tile is requested at once, before its row's parameters and lists are known (they take two
