@@ -53,10 +53,10 @@ extern "C" {
 #define SONIC_FLAG_TIMEOUT   0x10u  /* a bounded wait inside the streaming kernel expired: token is -1 (see sonic_workspace_init) */
 
 /* Bytes of workspace that serve every call over at most max_rows logit rows (B for sonic_sample / sonic_topk,
- * B*(K+1) for sonic_verify) of at most max_vocab entries each.  max_topk is accepted for forward compatibility
- * (the candidate slots are sized for every supported k) and ignored.  Pure host arithmetic.
- * Per row: 1.3 KB of control words, 8 bytes per candidate slot (min(32768, V rounded up to 8192)), and for the rows
- * with top-k off 4 bytes per vocabulary entry (the processed logits as ordered keys) plus 48 KB of histogram and list. */
+ * B*(K+1) for sonic_verify) of at most max_vocab entries each, and every sonic_topk call with k <= max_topk.  Pure
+ * host arithmetic.  Per row: 1.3 KB of control words, 8 bytes per candidate slot (min(32768, V rounded up to 8192);
+ * twice as many for sonic_topk with k > 2048), and for sampling and verification 4 bytes per vocabulary entry (the
+ * processed logits of rows with top-k off as ordered keys) plus 58 KB of histogram and lists. */
 size_t sonic_workspace_bytes(int max_rows, int max_vocab, int max_topk);
 
 /* Zeroes the workspace header (the first 512 bytes: work counters and the sticky error word) once after allocation
@@ -169,7 +169,7 @@ int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, 
  *
  * Same inputs, outputs and results as sonic_topk, for at most SONIC_STATIC_MAX_ROWS rows
  * per call; larger B is rejected with SONIC_ESHAPE.  The scratch memory is a fixed array
- * of about 2.1 MB inside the library image (SONIC_STATIC_MAX_ROWS rows of candidate
+ * of about 4.2 MB inside the library image (SONIC_STATIC_MAX_ROWS rows of candidate
  * slots and control words); every GPU that loads the library holds it until the process
  * exits.  The function calls no cudaMalloc, cudaFree or other allocating routine, and
  * all of its kernels go to `stream`.

@@ -74,11 +74,14 @@ struct Layout {
     int ytiles;
 };
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
-static Layout layout_for(long long rows, int V, bool dense) {
+// Candidate slots per row: CAND_CAP, twice that for sonic_topk with k beyond 2048 (its tiles bring up to ~1100
+// candidates each at k = 4096, V = 2^18, where an even share of CAND_CAP is 1024), never more than the row has elements.
+static size_t slot_cap(int op, int ktop) { return (op == OP_TOPK && ktop > 2048) ? 2 * (size_t)CAND_CAP : (size_t)CAND_CAP; }
+static Layout layout_for(long long rows, int V, bool dense, size_t cap = CAND_CAP) {
     Layout L;
     memset(&L, 0, sizeof(L));
     const int tiles = (V + CTA_TILE - 1) / CTA_TILE;
-    const size_t slots = (size_t)tiles * CTA_TILE < CAND_CAP ? (size_t)tiles * CTA_TILE : CAND_CAP;
+    const size_t slots = (size_t)tiles * CTA_TILE < cap ? (size_t)tiles * CTA_TILE : cap;
     L.cand_stride = (unsigned int)slots;
     L.ytiles = tiles;
     size_t off = WS_HEADER;
@@ -198,7 +201,7 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
     if (!ws) return fail(SONIC_EINVAL, "workspace is NULL");
     if (((uintptr_t)ws & 255) != 0) return fail(SONIC_EINVAL, "workspace must be 256-byte aligned");
     const bool dense = (P.op != OP_TOPK);
-    const Layout L = layout_for(P.rows, P.V, dense);
+    const Layout L = layout_for(P.rows, P.V, dense, slot_cap(P.op, P.ktop));
     if (ws_bytes < L.total) return fail(SONIC_EWORKSPACE, "workspace too small for this many rows of this vocabulary size");
     int sm_count = 1, dev = 0;
     int rc = configure_once(&sm_count, &dev);
@@ -356,11 +359,14 @@ using namespace sonic;
 extern "C" {
 
 size_t sonic_workspace_bytes(int max_rows, int max_vocab, int max_topk) {
-    (void)max_topk;                            // the candidate slots are sized for every supported k
     if (max_rows < 1) max_rows = 1;
     if (max_vocab < 1) max_vocab = 1;
     if (max_vocab > SONIC_MAX_VOCAB) max_vocab = SONIC_MAX_VOCAB;
-    return layout_for(max_rows, max_vocab, true).total;
+    // the larger of the two layouts a call can have: sampling / verification (with the histogram path's regions), and
+    // sonic_topk with its slots for max_topk
+    const size_t a = layout_for(max_rows, max_vocab, true).total;
+    const size_t b = layout_for(max_rows, max_vocab, false, slot_cap(OP_TOPK, max_topk)).total;
+    return a > b ? a : b;
 }
 
 int sonic_workspace_init(void *workspace, size_t bytes, void *stream) {
@@ -437,7 +443,7 @@ int sonic_topk(const void *logits, int dtype, int B, int V, int64_t row_stride, 
 // the library image.  In host code this name is only a stand-in for the symbol; the device
 // address the kernels need comes from cudaGetSymbolAddress (below), never from `&`.
 constexpr size_t STATIC_WS_BYTES = WS_HEADER + 256 * 4 +
-    (size_t)SONIC_STATIC_MAX_ROWS * (sizeof(RowState) + sizeof(PosResult) + sizeof(TileRec) * MAX_TILES + (size_t)CAND_CAP * 8);
+    (size_t)SONIC_STATIC_MAX_ROWS * (sizeof(RowState) + sizeof(PosResult) + sizeof(TileRec) * MAX_TILES + 2 * (size_t)CAND_CAP * 8);
 static __device__ __align__(256) unsigned char g_static_workspace[STATIC_WS_BYTES];
 
 static int static_workspace_address(void **out) {

@@ -245,7 +245,81 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         csync();
         // every proven key is at least (cutoff key << 32): the search starts from the range the keys can span
         unsigned long long lo = max(1ull, (unsigned long long)(c.temp ? tykey : tkey) << 32), hi = kmax + 1ull;   // count(>= lo) >= k > count(>= hi) = 0
-        for (int it = 0; it < 24 && hi - lo > 1ull; ++it) {
+        bool bracketed = false;
+        {
+            // First a bracket from one counting pass: 2048 bins over the keys the proven candidates span, counted from
+            // the top; the bin in which the count reaches k gives a floor that keeps at least k, and usually no more
+            // than the buffer holds (the search below then has nothing left to do).
+            int *hist = reinterpret_cast<int *>(buf);            // (what was packed so far is dropped: it is packed again below)
+            int *redi = reinterpret_cast<int *>(sh.scratch);
+            const uint32_t klo = (uint32_t)(lo >> 32), khi = (uint32_t)(kmax >> 32);
+            const uint32_t span = khi - klo;
+            const int shift = span < 2048u ? 0 : (32 - __clz(span)) - 11;
+            for (int i = tid; i < 2048; i += THREADS) hist[i] = 0;
+            csync();
+            for (int ta = warp; ta < tiles; ta += 2 * NW) {
+                const int tb = ta + NW;
+                const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
+                const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
+                const unsigned long long *pa = P.cand + (size_t)row * P.cand_stride + (size_t)ta * cap_t;
+                const unsigned long long *pb = P.cand + (size_t)row * P.cand_stride + (size_t)tb * cap_t;
+                for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
+                    unsigned long long cd[GB];
+#pragma unroll
+                    for (int u = 0; u < HB; ++u) {
+                        const int j = j0 + u * 32 + lane;
+                        cd[u] = (j < na) ? __ldcg(pa + j) : 0ull;
+                        cd[HB + u] = (j < nb) ? __ldcg(pb + j) : 0ull;
+                    }
+#pragma unroll
+                    for (int u = 0; u < GB; ++u) {
+                        const int j = j0 + (u % HB) * 32 + lane;
+                        const bool valid = (u < HB) ? (j < na) : (j < nb);
+                        const unsigned long long out = proven_key(cd[u], valid ? 0 : total);
+                        if (out >= lo) atomicAdd(&hist[(khi - (uint32_t)(out >> 32)) >> shift], 1);
+                    }
+                }
+            }
+            csync();
+            static_assert(2048 % THREADS == 0, "bins per thread");
+            constexpr int BPT = 2048 / THREADS;
+            int v[BPT], s = 0;
+#pragma unroll
+            for (int j = 0; j < BPT; ++j) { v[j] = hist[tid * BPT + j]; s += v[j]; }
+            int incl = s;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (lane == 31) redi[warp] = incl;
+            if (tid == 0) redi[40] = -1;
+            csync();
+            int pre = incl - s;
+            for (int w = 0; w < warp; ++w) pre += redi[w];
+            if (pre < c.k && pre + s >= c.k) {
+                int run = pre;
+#pragma unroll
+                for (int j = 0; j < BPT; ++j) {
+                    if (run < c.k && run + v[j] >= c.k) { redi[40] = tid * BPT + j; redi[41] = run; redi[42] = run + v[j]; }
+                    run += v[j];
+                }
+            }
+            csync();
+            const int b = redi[40], above = redi[41], kept = redi[42];
+            csync();
+            if (b >= 0) {
+                // bin b holds the keys khi - ((b + 1) << shift) + 1 .. khi - (b << shift)
+                const unsigned long long width = 1ull << shift;
+                const unsigned long long down = (unsigned long long)(b + 1) * width - 1ull;
+                const uint32_t kb = (down >= (unsigned long long)span) ? klo : khi - (uint32_t)down;
+                lo = max(lo, (unsigned long long)kb << 32);                                    // count(>= lo) = kept >= k
+                if (b > 0) hi = ((unsigned long long)(khi - (uint32_t)((unsigned long long)b * width) + 1u)) << 32;   // count(>= hi) = above < k
+                (void)above;
+                bracketed = kept <= MERGE_CAP;
+            }
+        }
+        for (int it = 0; it < 24 && !bracketed && hi - lo > 1ull; ++it) {
             const unsigned long long step = (hi - lo) >> 3;
             unsigned long long th[7];
 #pragma unroll
