@@ -175,6 +175,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             const int tb = ta + NW;
             const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
             const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
+            const bool single = tb >= tiles;            // no second tile for this warp: all load slots go to the first
             const unsigned long long *pa = P.cand + (size_t)row * P.cand_stride + (size_t)ta * cap_t;
             const unsigned long long *pb = P.cand + (size_t)row * P.cand_stride + (size_t)tb * cap_t;
             if (max(na, nb) <= 32) {
@@ -195,13 +196,13 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 if (ob >= floor_key) { const int pos = base + __popc(ma) + __popc(mb & below); if (pos < MERGE_CAP) buf[pos] = ob; }
                 continue;
             }
-            for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
+            for (int j0 = 0; j0 < max(na, nb); j0 += (single ? 32 * GB : 32 * HB)) {
                 unsigned long long cd[GB];
 #pragma unroll
                 for (int u = 0; u < HB; ++u) {
-                    const int j = j0 + u * 32 + lane;
+                    const int j = j0 + u * 32 + lane, j2 = j + 32 * HB;
                     cd[u] = (j < na) ? __ldcg(pa + j) : 0ull;
-                    cd[HB + u] = (j < nb) ? __ldcg(pb + j) : 0ull;
+                    cd[HB + u] = single ? ((j2 < na) ? __ldcg(pa + j2) : 0ull) : ((j < nb) ? __ldcg(pb + j) : 0ull);
                 }
                 // filter all of the batch, then reserve room with ONE shared-memory atomic per warp and batch
                 // (every warp adds to the same counter: per-candidate or per-slot atomics would queue up there)
@@ -210,8 +211,8 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 int nkeep = 0;
 #pragma unroll
                 for (int u = 0; u < GB; ++u) {
-                    const int j = j0 + (u % HB) * 32 + lane;
-                    const bool valid = (u < HB) ? (j < na) : (j < nb);
+                    const int j = j0 + (u % HB) * 32 + lane + ((single && u >= HB) ? 32 * HB : 0);
+                    const bool valid = (u < HB || single) ? (j < na) : (j < nb);
                     out[u] = proven_key(cd[u], valid ? 0 : total);
                     kmax = max(kmax, out[u]);
                     km[u] = __ballot_sync(0xFFFFFFFFu, out[u] >= floor_key);
@@ -261,20 +262,21 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 const int tb = ta + NW;
                 const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
                 const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
+                const bool single = tb >= tiles;            // no second tile for this warp: all load slots go to the first
                 const unsigned long long *pa = P.cand + (size_t)row * P.cand_stride + (size_t)ta * cap_t;
                 const unsigned long long *pb = P.cand + (size_t)row * P.cand_stride + (size_t)tb * cap_t;
-                for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
+                for (int j0 = 0; j0 < max(na, nb); j0 += (single ? 32 * GB : 32 * HB)) {
                     unsigned long long cd[GB];
 #pragma unroll
                     for (int u = 0; u < HB; ++u) {
-                        const int j = j0 + u * 32 + lane;
+                        const int j = j0 + u * 32 + lane, j2 = j + 32 * HB;
                         cd[u] = (j < na) ? __ldcg(pa + j) : 0ull;
-                        cd[HB + u] = (j < nb) ? __ldcg(pb + j) : 0ull;
+                        cd[HB + u] = single ? ((j2 < na) ? __ldcg(pa + j2) : 0ull) : ((j < nb) ? __ldcg(pb + j) : 0ull);
                     }
 #pragma unroll
                     for (int u = 0; u < GB; ++u) {
-                        const int j = j0 + (u % HB) * 32 + lane;
-                        const bool valid = (u < HB) ? (j < na) : (j < nb);
+                        const int j = j0 + (u % HB) * 32 + lane + ((single && u >= HB) ? 32 * HB : 0);
+                        const bool valid = (u < HB || single) ? (j < na) : (j < nb);
                         const unsigned long long out = proven_key(cd[u], valid ? 0 : total);
                         if (out >= lo) atomicAdd(&hist[(khi - (uint32_t)(out >> 32)) >> shift], 1);
                     }
@@ -330,20 +332,21 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 const int tb = ta + NW;
                 const int na = sh.tcnt[ta + 1] - sh.tcnt[ta];
                 const int nb = (tb < tiles) ? sh.tcnt[tb + 1] - sh.tcnt[tb] : 0;
+                const bool single = tb >= tiles;            // no second tile for this warp: all load slots go to the first
                 const unsigned long long *pa = P.cand + (size_t)row * P.cand_stride + (size_t)ta * cap_t;
                 const unsigned long long *pb = P.cand + (size_t)row * P.cand_stride + (size_t)tb * cap_t;
-                for (int j0 = 0; j0 < max(na, nb); j0 += 32 * HB) {
+                for (int j0 = 0; j0 < max(na, nb); j0 += (single ? 32 * GB : 32 * HB)) {
                     unsigned long long cd[GB];
 #pragma unroll
                     for (int u = 0; u < HB; ++u) {
-                        const int j = j0 + u * 32 + lane;
+                        const int j = j0 + u * 32 + lane, j2 = j + 32 * HB;
                         cd[u] = (j < na) ? __ldcg(pa + j) : 0ull;
-                        cd[HB + u] = (j < nb) ? __ldcg(pb + j) : 0ull;
+                        cd[HB + u] = single ? ((j2 < na) ? __ldcg(pa + j2) : 0ull) : ((j < nb) ? __ldcg(pb + j) : 0ull);
                     }
 #pragma unroll
                     for (int u = 0; u < GB; ++u) {
-                        const int j = j0 + (u % HB) * 32 + lane;
-                        const bool valid = (u < HB) ? (j < na) : (j < nb);
+                        const int j = j0 + (u % HB) * 32 + lane + ((single && u >= HB) ? 32 * HB : 0);
+                        const bool valid = (u < HB || single) ? (j < na) : (j < nb);
                         const unsigned long long out = proven_key(cd[u], valid ? 0 : total);
 #pragma unroll
                         for (int q = 0; q < 7; ++q) cnt[q] += (out >= th[q]) ? 1 : 0;
