@@ -715,6 +715,60 @@ def run_sweep():
                       "peak_source": which, "table": table}))
 
 
+TIMELINE_KERNELS = {0: "sonic_stream_kernel", 1: "sonic_merge_kernel", 6: "sonic_dense_stage2_kernel",
+                    3: "sonic_dense_collect_kernel", 8: "sonic_dense_finish_kernel", 4: "sonic_dense_resid_kernel",
+                    9: "sonic_dense_resid_finish_kernel", 2: "sonic_exact_kernel", 5: "sonic_verify_combine_kernel"}
+
+
+def run_timeline(names, reps=5):
+    """Per-kernel timeline of ONE call inside a replayed CUDA graph, from the trace variant of the library (every kernel
+    leaves the earliest start and the latest end of its CTAs, globaltimer, in the workspace header).  One input copy
+    (warm L2 where it fits); the figures show how the kernels of a call overlap, they are not a bench value.
+    Prints one JSON line: {workload: {kernel: [start_us, end_us] (median of `reps` replays, from the first start)}}."""
+    import torch
+    from paper_2607_20475_b200 import build as _build
+    _build.LIB = _build.build_trace()               # before the binding loads a library: this process uses the trace variant
+    from paper_2607_20475_b200 import harness as binding
+    binding.lib()
+    out = {}
+    for name in names:
+        if name.startswith("c5k"):
+            dev = binding.DeviceTopK(wl.config5("normal"), int(name[3:]))
+        elif name == "c4":
+            dev = binding.DeviceVerify(make_workload(name))
+        else:
+            dev = binding.DeviceSample(make_workload(name))
+        hdr = dev.ws[:512].view(torch.int32)
+        dev.run()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            dev.run()
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        runs = []
+        for _ in range(reps):
+            init = torch.zeros(24, dtype=torch.int32, device="cuda")
+            init[0::2] = -1                                     # starts take a minimum, ends a maximum
+            hdr[48:72] = init
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            h = hdr.cpu().numpy().astype(np.int64) & 0xFFFFFFFF
+            t0 = min(int(h[48 + 2 * k]) for k in TIMELINE_KERNELS if h[48 + 2 * k] != 0xFFFFFFFF)
+            runs.append({nm: [((int(h[48 + 2 * k]) - t0) & 0xFFFFFFFF) / 1000.0, ((int(h[49 + 2 * k]) - t0) & 0xFFFFFFFF) / 1000.0]
+                         for k, nm in TIMELINE_KERNELS.items() if h[48 + 2 * k] != 0xFFFFFFFF and h[49 + 2 * k] != 0})
+        kernels = {}
+        for nm in runs[0]:
+            if all(nm in r for r in runs):
+                kernels[nm] = [round(float(np.median([r[nm][0] for r in runs])), 2), round(float(np.median([r[nm][1] for r in runs])), 2)]
+        out[name] = {"kernels": kernels, "call_end_us": max(v[1] for v in kernels.values())}
+        del dev, g
+        torch.cuda.empty_cache()
+    print(json.dumps({"timeline": out, "unit": "us from the first kernel's start", "build": "-DSONIC_TRACE variant, one input copy"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -727,6 +781,9 @@ def main():
                     help="repeat the timed block of --steps calls until this much device time is measured (0: one block)")
     ap.add_argument("--profile-run", action="store_true",
                     help="run the warm-up and one timed block only and print a short line (for use under ncu; never a bench value)")
+    ap.add_argument("--timeline", default=None,
+                    help="print the per-kernel timeline of one call of the given workloads (comma separated: c1..c4, c5k<k>) "
+                         "from the trace variant of the library, instead of a bench line (one GPU)")
     ap.add_argument("--also", default="c1,c3,c4,c5", help="other configurations to time briefly (comma separated, '' for none; "
                     "c5 = sonic_topk over all regimes and k, c5k<k> = one k of the 'normal' regime)")
     args = ap.parse_args()
@@ -739,6 +796,10 @@ def main():
         if args.warmup == 16:
             args.warmup = 1
         run_reference(args, rank, world)
+        return
+    if args.timeline:
+        if rank == 0:
+            run_timeline([n for n in args.timeline.split(",") if n])
         return
     if args.sweep:
         if rank == 0:

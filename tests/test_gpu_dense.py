@@ -105,6 +105,35 @@ def test_top_p_against_min_p_in_one_row(sonic, oracle):
     run(sonic, oracle, w)
 
 
+def test_top_p_just_below_and_just_above_a_cumulative_fraction_with_the_mass_in_the_ragged_tile(sonic, oracle):
+    # p set a hair below and a hair above the cumulative fraction of the n-th ranked token (relative distance 2e-5, far
+    # outside the near-margin band): the support is n, then n + 1.  The heavy tokens sit in the row's ragged last tile
+    # (V = 2 tiles + 300), so the cut element, most of the support and the drawn tokens are found there.
+    V = 2 * 8192 + 300
+    rng = np.random.default_rng(21)
+    base = (rng.standard_normal(V) * 1.5).astype(np.float32)
+    base[-300:] += np.float32(6.0)
+    y = base.astype(np.float64)
+    order = np.lexsort((np.arange(V), -y))
+    wts = np.exp(y[order] - y.max())
+    frac = np.cumsum(wts) / wts.sum()
+    rows, ps, want = [], [], []
+    for n in (1, 2, 17, 120, 299, 300, 301, 2000):
+        f = frac[n - 1]                                        # mass of the n best tokens
+        if frac[n] - f < 1e-4 * f:                             # (the next token must clear the band too)
+            continue
+        for p_, n_ in ((f * (1 - 2e-5), n), (f * (1 + 2e-5), n + 1)):
+            rows.append(base); ps.append(np.float32(p_)); want.append(n_)
+    B = len(rows)
+    assert B >= 10
+    w = make_sample(np.stack(rows), np.full(B, wl.TOP_P), top_p=ps, seed=np.arange(B) + 3, offset=np.arange(B) * 7)
+    got, ref, near = run(sonic, oracle, w, max_near=0)
+    assert near == 0
+    assert ref["support"].tolist() == want and got["support"].tolist() == want
+    assert np.all((got["flags"] & DENSE) != 0)
+    assert np.mean(got["token"] >= 2 * 8192) > 0.5            # drawn from the ragged tile
+
+
 def test_rows_without_token_and_bad_rows_of_the_class(sonic, oracle):
     V = 20000
     rng = np.random.default_rng(13)
