@@ -274,8 +274,8 @@ static int launch_all(KParams &P, void *ws, size_t ws_bytes, cudaStream_t st, in
         dcfg.gridDim = dim3(dense_ctas);
         dcfg.blockDim = dim3(DENSE_THREADS);
         dcfg.dynamicSmemBytes = DENSE_DYN_SMEM;
-        cudaLaunchConfig_t fcfg = dcfg;              // row-level steps: one CTA per row, one per SM at most
-        fcfg.gridDim = dim3(P.rows < sm_count ? P.rows : sm_count);
+        cudaLaunchConfig_t fcfg = dcfg;              // row-level steps: one CTA per row of the call (rows of other classes leave at once)
+        fcfg.gridDim = dim3(P.rows);
         // Stage 2 never waits for its predecessor in the stream.  On the internal stream it is an ordinary launch
         // behind the fork; on the caller's stream it is a programmatic dependent of the merge kernel, whose CTAs let
         // it go only after their own wait for the streaming kernel.

@@ -832,6 +832,7 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
             __threadfence();
             const unsigned int slot = atomicAdd(&P.error[WS_NRESID], 1u);
             P.rlist[slot] = row;
+            dr->state = 2u;                                  // the residual draw's CTA of this row has work
         }
         return true;
     }
@@ -983,8 +984,8 @@ sonic_dense_collect_kernel(const KParams P, const int tiles) {
     KERNEL_T1(3);
 }
 
-// The rows' finish, one CTA per row of the class (a programmatic dependent of pass C, whose completion is the only
-// synchronisation a row needs).
+// The rows' finish, one CTA per row of the call (those of other classes leave at once): a programmatic dependent of
+// pass C, whose completion is the only synchronisation a row needs.
 __global__ void __launch_bounds__(DENSE_THREADS)
 sonic_dense_finish_kernel(const KParams P, const int tiles) {
     extern __shared__ __align__(16) unsigned char dense_dyn_raw[];
@@ -992,28 +993,32 @@ sonic_dense_finish_kernel(const KParams P, const int tiles) {
     unsigned long long *dyn = reinterpret_cast<unsigned long long *>(dense_dyn_raw);
     const int tid = threadIdx.x;
     pdl_launch_dependents();
+    // One CTA per row of the call: the row is known at launch, so its parameters are read - and the CTAs of rows of
+    // other classes are gone - before the wait (inputs only; nothing here depends on the earlier kernels).
+    const int row = blockIdx.x;
+    {
+        const RowCfg c0 = load_cfg(P, row);
+        if (c0.cls != CLS_DENSE) return;
+    }
+    const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
+    const unsigned long long seed = P.seed ? P.seed[req] : 0ull, off = P.offset ? P.offset[req] : 0ull;
     pdl_wait_primary();
     KERNEL_T0(8);
-    const int nd = (int)__ldcg(&P.error[WS_NDENSE]);
-    for (int i = blockIdx.x; i < nd; i += gridDim.x) {
-        const int row = __ldcg(&P.dlist[i]);
+    {
         RowCfg c;
-        // (the Philox cells need the request's seed and offset only: their loads go out with the row's other loads)
-        const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
-        const unsigned long long seed = P.seed ? P.seed[req] : 0ull, off = P.offset ? P.offset[req] : 0ull;
         const DenseRowPar par = dense_row_par(P, row, tiles, sm, dyn, tid, 4, false, c);
-        if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {       // (a wait of the streaming kernel ran out: nothing of the row is to be trusted)
-            if (tid == 0) emit_row(P, c, row, -1, 0.0f, F_TIMEOUT | F_DENSE, 0, 0.0f);
-            continue;
+        if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {       // (a wait of the streaming kernel ran out: the call's last kernel reports it for every row)
+            KERNEL_T1(8);
+            return;
         }
-        if (par.kind == 0) continue;
-        uint32_t r4[4];
-        const unsigned long long pos = off + (unsigned long long)c.l;
-        philox4x32_10((uint32_t)pos, (uint32_t)(pos >> 32), (uint32_t)c.b, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), r4);
-        const uint2 cells = make_uint2(r4[0] >> 8, r4[1] >> 8);
-        const bool ok = dense_finish(P, c, row, tiles, sm, dyn, tid, par.Mkey, par.klo <= par.khi, par.target, par.tk, cells);
-        if (!ok && tid == 0) { P.rs[row].status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
-        __syncthreads();
+        if (par.kind != 0) {
+            uint32_t r4[4];
+            const unsigned long long pos = off + (unsigned long long)c.l;
+            philox4x32_10((uint32_t)pos, (uint32_t)(pos >> 32), (uint32_t)c.b, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), r4);
+            const uint2 cells = make_uint2(r4[0] >> 8, r4[1] >> 8);
+            const bool ok = dense_finish(P, c, row, tiles, sm, dyn, tid, par.Mkey, par.klo <= par.khi, par.target, par.tk, cells);
+            if (!ok && tid == 0) { P.rs[row].status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
+        }
     }
     KERNEL_T1(8);
 }
@@ -1182,11 +1187,16 @@ sonic_dense_resid_finish_kernel(const KParams P, const int tiles) {
     __shared__ DenseShared sm;
     const int tid = threadIdx.x;
     pdl_launch_dependents();
+    // one CTA per row of the call, as in the rows' finish: rows of other classes, and positions without a draft, leave
+    // before the wait; rows whose draft was accepted right after it
+    const int row = blockIdx.x;
+    {
+        const RowCfg c0 = load_cfg(P, row);
+        if (c0.cls != CLS_DENSE || c0.l >= P.K) return;
+    }
     pdl_wait_primary();
     KERNEL_T0(9);
-    const int nr = (int)__ldcg(&P.error[WS_NRESID]);
-    for (int i = blockIdx.x; i < nr; i += gridDim.x) {
-        const int row = __ldcg(&P.rlist[i]);
+    if (__ldcg(&(P.drow + row)->state) == 2u) {
         DenseRow *dr = P.drow + row;
         DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
         const RowCfg c = load_cfg(P, row);
