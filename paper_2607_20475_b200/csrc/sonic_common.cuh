@@ -341,14 +341,12 @@ __device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) { return r
 
 #ifdef SONIC_TRACE
 __device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
-#define STREAM_STAMP(i) do { if ((int)blockIdx.x == (int)P.error[121] && lane == 0) P.error[40 + (i)] = gtimer_lo(); } while (0)
 // kernel-level timeline: earliest start and latest end of kernel k (0 stream, 1 merge, 2 exact first launch, 3 exact second launch)
 #define KERNEL_T0(k) do { if (threadIdx.x == 0) atomicMin(&P.error[48 + 2 * (k)], gtimer_lo()); } while (0)
 #define KERNEL_T1(k) do { if (threadIdx.x == 0) atomicMax(&P.error[49 + 2 * (k)], gtimer_lo()); } while (0)
 #else
 #define KERNEL_T0(k) do { } while (0)
 #define KERNEL_T1(k) do { } while (0)
-#define STREAM_STAMP(i) do { } while (0)
 #endif
 
 // ---------------------------------------------------------------- Philox4x32-10

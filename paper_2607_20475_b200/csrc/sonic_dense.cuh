@@ -25,12 +25,6 @@
 
 namespace sonic {
 
-#ifdef SONIC_DTRACE
-__device__ __forceinline__ unsigned int dtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
-#define DSTAMP(i) do { if (threadIdx.x == 0 && blockIdx.x == 0) P.error[64 + (i)] = dtimer(); } while (0)
-#else
-#define DSTAMP(i) do { } while (0)
-#endif
 
 constexpr int DENSE_THREADS = 512;
 constexpr int DENSE_WARPS = DENSE_THREADS / 32;
@@ -937,7 +931,6 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
     int cur_row = -1;
     DenseRowPar par;
     par.kind = 0;
-    DSTAMP((stage - 2) * 16 + 0);
     for (int item = rg.lo; item < rg.hi; ++item) {
         const DenseItem it = dense_item(P.dlist, item, tiles, sub);
         uint4 kv[DENSE_NV];
@@ -947,7 +940,6 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
             RowCfg c;
             par = dense_row_par(P, it.row, tiles, sm, dyn, tid, stage, it.tile == 0 && it.part == 0, c);
         }
-        DSTAMP((stage - 2) * 16 + 1 + 2 * min(item - rg.lo, 6));
         if (par.kind == 1) {
             unsigned int *hm0 = reinterpret_cast<unsigned int *>(dyn), *hm1 = hm0 + DBINS;
             dense_hist_item(P, it, kv, unkey(par.Mkey), par.scale, hm0, hm1, tid);
@@ -955,7 +947,6 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
             dense_collect_part(P, it, kv, unkey(par.Mkey), par.klo, par.khi, sm, dyn, tid);
         }
         __syncthreads();
-        DSTAMP((stage - 2) * 16 + 2 + 2 * min(item - rg.lo, 6));
     }
 }
 

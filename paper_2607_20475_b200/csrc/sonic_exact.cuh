@@ -19,12 +19,6 @@
 namespace sonic {
 namespace cg = cooperative_groups;
 
-#ifdef SONIC_TRACE
-// debug builds: rank 0 / thread 0 of the cluster handling the traced row stamps the clock into the workspace header
-#define SONIC_STAMP(i) do { if (x.rank == 0 && x.tid == 0 && x.trace) x.tracep[8 + (i)] = (unsigned int)clock64(); } while (0)
-#else
-#define SONIC_STAMP(i) do { } while (0)
-#endif
 
 constexpr int EX_THREADS = 512;
 constexpr int EX_WARPS = EX_THREADS / 32;
@@ -64,8 +58,6 @@ struct ExactCtx {
     unsigned int *hcnt, *hm0, *hm1;            // per-bin count and 64-bit mass as two 32-bit words (32-bit adds, explicit carry)
     int rank, lo, len, per, tid, lane, warp;
     int phase;
-    int trace;
-    unsigned int *tracep;
     float Mf;                                  // largest processed logit
     float scale, inv_scale;                    // histogram bins per logit unit (a power of two) and its reciprocal
 };
@@ -345,9 +337,7 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
             }
         }
     }
-    if (first) SONIC_STAMP(17);
     cg::this_cluster().sync();
-    if (first) SONIC_STAMP(18);
     // CTA r reduces bins [r*bpr, (r+1)*bpr) over the cluster.  Remote shared-memory reads are slow, so
     // all of them are issued at once: thread t fetches (bin, rank) pairs t, t + EX_THREADS, ... into a
     // local staging area (the sort buffer, idle during histogram levels), then the owners add locally.
@@ -397,7 +387,6 @@ __device__ int hist_level(ExactCtx &x, const Cut &base, bool by_mass, bool first
     unsigned long long v[XV] = {sc, sm, 0, 0};
     unsigned long long all[CL][XV];
     allgather(x, v, all);                      // every remote histogram read precedes this barrier
-    if (first) SONIC_STAMP(19);
     if (by_mass && first) {
         unsigned long long Zq = 0;
         for (int r = 0; r < CL; ++r) Zq += all[r][1];
@@ -494,7 +483,6 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         return 2047 - (int)t;
     };
     const int a = hist_level(x, base, by_mass, true, p, HBINS, dig_a, target, in_bin, sortbuf);
-    SONIC_STAMP(4);
     // A bin is an interval of (M - y), hence of keys.  A conservative key interval (the exact one widened by a
     // margin that covers the roundings of the digit arithmetic and of this computation) lets the later passes
     // reject almost every element with two integer compares before the exact digit test.
@@ -567,7 +555,6 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
         if (gmin == gmax) { single = true; single_key = gmax; }
         else b = hist_level(x, base, by_mass, false, p, HBINS, dig_b, target, in_bin, sortbuf);
     }
-    SONIC_STAMP(5);
     uint32_t klo = klo_a, khi = khi_a;
     if (b >= 0 && a != 0) {                                      // (bin 0 of level 0 is open below: no finer band)
         const int n = 2047 - a, m = 2047 - b;
@@ -618,7 +605,6 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
                 if (off + i < (unsigned int)GATHER_CAP) dst[off + i] = sortbuf[i];
         }
         cg::this_cluster().sync();
-        SONIC_STAMP(6);
         unsigned long long v2[XV] = {0, 0, 0, 0};
         if (x.rank == 0) {
             const int nn = (int)min(n, (unsigned int)GATHER_CAP);
@@ -626,7 +612,6 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
             for (int i = nn + x.tid; i < m; i += EX_THREADS) sortbuf[i] = 0ull;
             __syncthreads();
             bitonic_sort_desc_cta<EX_THREADS>(sortbuf, m, x.tid);
-            SONIC_STAMP(7);
             // running count / mass in ranking order; each thread owns a contiguous chunk of the sorted list
             const int chunk = (nn + EX_THREADS - 1) / EX_THREADS;
             const int lo = min(nn, x.tid * chunk), hi = min(nn, lo + chunk);
@@ -656,7 +641,6 @@ __device__ Cut select_cut(ExactCtx &x, const Cut &base, bool by_mass, unsigned l
             v2[0] = sortbuf[max(0, x.sh->flag)];
         }
         allgather(x, v2, all);
-        SONIC_STAMP(8);
         Cut c;
         c.v = (uint32_t)(all[0][0] >> 32);
         c.idx = (int)(~(uint32_t)all[0][0]);
@@ -716,10 +700,6 @@ template <int DT>
 __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned long long *sortbuf) {
     const RowCfg c = load_cfg(P, row);
     RowState *rs = P.rs + row;
-#ifdef SONIC_TRACE
-    x.tracep = P.error;
-    x.trace = (row == (int)P.error[120]);
-#endif
     const int V = P.V;
     x.per = (((V + CL - 1) / CL) + 1023) & ~1023;
     x.lo = x.rank * x.per;
@@ -732,18 +712,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         for (int i = x.tid * 32; i < x.len; i += EX_THREADS * 32)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(q + x.lo + i));
     }
-    SONIC_STAMP(0);
-#ifdef SONIC_TRACE
-    SONIC_STAMP(12);
-    cg::this_cluster().sync();
-    SONIC_STAMP(13);
-    cg::this_cluster().sync();
-    SONIC_STAMP(14);
-    { unsigned long long tv[XV] = {1, 2, 3, 4}; unsigned long long ta[CL][XV]; allgather(x, tv, ta); if (ta[0][0] == 77) x.trace = 0; }
-    SONIC_STAMP(15);
-    __syncthreads();
-    SONIC_STAMP(16);
-#endif
 
     // ---- load the slice, mask, sparse patches, temperature, keys
     constexpr int VEC = VecTraits<DT>::VEC;
@@ -802,7 +770,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         }
     }
     bad = __syncthreads_or(bad);
-    SONIC_STAMP(1);
     uint32_t kmax = 0, kmin = 0xFFFFFFFFu;      // kmin over the finite elements
     unsigned int nfin32 = 0;
     for (int l0 = x.tid * 4; l0 < x.per; l0 += EX_THREADS * 4) {   // per is a multiple of 1024: whole float4s
@@ -849,7 +816,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         x.scale = ldexpf(1.0f, e);
         x.inv_scale = ldexpf(1.0f, -e);
     }
-    SONIC_STAMP(2);
     const bool leader = (x.rank == 0 && x.tid == 0);
 
     if (__ldcg(&P.error[WS_ERROR]) & ERR_TIMEOUT) {           // (uniform over the cluster; see the merge kernel)
@@ -913,9 +879,7 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     if (c.k > 0 && (unsigned long long)c.k < Nf) cut = select_cut(x, cut, false, (unsigned long long)c.k, 1.0f, sortbuf);
     const Cut cut_k = cut;
     if (c.z & M_TOP_P) {
-        SONIC_STAMP(3);
         Cut cp = select_cut(x, cut_k, true, 0ull, c.p, sortbuf);
-        SONIC_STAMP(9);
         if (tighter(cp, cut)) cut = cp;
     }
     if (c.z & M_MIN_P) {
@@ -944,7 +908,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     unsigned long long nS;
     ordered_totals<unsigned long long>(x, wq, inS, stq, nS);
     const unsigned long long Wq = stq.total;
-    SONIC_STAMP(10);
     const unsigned long long mul = 2ull * a_draw + 1ull;               // u = mul / 2^25
     const unsigned long long T = (__umul64hi(Wq, mul) << 39) | ((Wq * mul) >> 25);
     // A position that carries a draft token needs a draw from p only if the draft is rejected AND the residual is
@@ -952,7 +915,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
     const bool draft_pos = (P.op == OP_VERIFY && c.l < P.K);
     bool plain_draw = !draft_pos;
     int token = -1;
-    SONIC_STAMP(11);
 
     uint32_t flags = F_FALLBACK;
     float p_draft = 0.0f;
@@ -968,7 +930,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
         double Q = (d >= 0 && d < V) ? (double)__ldg(q + d) : 0.0;
         const bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);      // the same value in every CTA
         p_draft = (float)Pd;
-        SONIC_STAMP(20);
         if (accept) {
             // the request moves on with the draft token: neither the residual nor a draw of this position is read
             flags |= F_ACCEPT;
@@ -983,7 +944,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
             unsigned long long cdummy;
             ordered_totals<double>(x, wd, inS, std_, cdummy);
             const double Wd = std_.total;
-            SONIC_STAMP(21);
             const double inv_Wd = 1.0 / Wd;                        // p = w * (1 / W): one rounding more than w / W, far below the margins
             auto rd = [=](int i) -> double {
                 if (!(i < slen && member(scut, skeys[i], slo + i))) return 0.0;
@@ -1003,7 +963,6 @@ __device__ void exact_row(const KParams &P, const int row, ExactCtx &x, unsigned
                 ordered_totals<unsigned long long>(x, wq, inS, stq, ndummy);
                 plain_draw = true;
             }
-            SONIC_STAMP(22);
         }
     }
     double token_prob = 0.0;

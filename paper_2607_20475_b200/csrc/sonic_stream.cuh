@@ -102,11 +102,6 @@ struct MergeShared {
     alignas(16) double scratch[THREADS];      // also read as int4
 };
 
-#ifdef SONIC_TRACE
-#define MERGE_STAMP(i) do { if (tid == 0 && row == (int)P.error[120]) P.error[8 + (i)] = (unsigned int)clock64(); } while (0)
-#else
-#define MERGE_STAMP(i) do { } while (0)
-#endif
 
 constexpr int RANK_SORT_MAX = 512;            // at most this many candidates: sort by rank counting
 constexpr int WARP_EPILOGUE_MAX = 128;        // at most this many survivors of TopK: one warp finishes the row
@@ -124,7 +119,6 @@ template <int THREADS, typename Sync>
 __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int tiles,
                                unsigned long long *buf, MergeShared<THREADS> &sh, int tid, uint2 cells) {
     Sync csync;
-    MERGE_STAMP(0);
     const int cap_t = (int)(P.cand_stride / (unsigned)tiles);
     const TileRec *rec = P.tiles + (size_t)row * MAX_TILES;
     // tile records: the first warp takes one tile per lane; prefix of the counts and the largest cutoff by shuffles
@@ -148,7 +142,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     }
     csync();
     if (sh.found) return false;
-    MERGE_STAMP(1);
     const unsigned int tkey = sh.tkey;
     const bool complete = (tkey == KEY_NEG_INF);
     const bool strict = c.temp && !complete;            // keys are compared after the temperature division
@@ -231,9 +224,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 }
             }
         }
-        MERGE_STAMP(17);
         csync();
-        MERGE_STAMP(18);
         if (attempt == 1 || sh.count <= MERGE_CAP || sh.count < c.k) break;
         // More proven candidates than the buffer holds (large k): find a key floor that keeps between k and
         // MERGE_CAP of them by an eight-way search over the candidates in global memory, then pack again.
@@ -389,7 +380,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     }
     csync();
     const int Pn = sh.count;
-    MERGE_STAMP(2);
     if (Pn > MERGE_CAP) return false;
     int n;
     if (Pn >= c.k) n = c.k;
@@ -428,7 +418,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 hist[tid] = 0;
             }
             csync();
-            MERGE_STAMP(13);
             for (int i = tid; i < Pn; i += THREADS) {
                 const unsigned long long key = buf[i];
                 int bkt = 0;                                   // number of sampled keys <= key
@@ -438,7 +427,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 atomicAdd(&hist[bkt], 1);
             }
             csync();
-            MERGE_STAMP(14);
             if (tid < 32) {
                 int suf = hist[tid];                           // -> number of keys in buckets >= tid
 #pragma unroll
@@ -463,7 +451,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             const int cnt_lo = (int)res[2], cnt_hi = (int)res[3];
             tight = cnt_lo <= want_hi;
             csync();
-            MERGE_STAMP(15);
             // The bucket [lo, hi) holds the boundary.  If it is small, its keys are collected and ranked, which gives
             // the threshold that keeps exactly n (no search over key space, whose passes multiply when equal values
             // differ only in their index bits).
@@ -483,7 +470,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                     if (inb) list[base + __popc(mk & ((1u << (tid & 31)) - 1u))] = key;
                 }
                 csync();
-                MERGE_STAMP(16);
                 int rank;
                 const unsigned long long key = rank_keys<THREADS, Sync>(list, in_bucket, tid, rank);
                 csync();
@@ -494,7 +480,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 csync();
             }
         }
-        MERGE_STAMP(11);
         // eight-way search: seven interior thresholds per pass.  The warps add their counts into one of two sets
         // of totals in shared memory (the other set is cleared meanwhile), so a pass costs two block barriers
         // and every thread reads just the seven totals.
@@ -535,9 +520,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             }
             if (!done) hi = th[0];
             csync();
-#ifdef SONIC_TRACE
-            if (tid == 0 && row == (int)P.error[120]) P.error[28] += 1u;
-#endif
         }
         // keep the keys >= lo, packed to the front
         if (tid == 0) sh.count = 0;
@@ -577,10 +559,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         Pn2 = sh.count;
         csync();
     }
-    MERGE_STAMP(12);
-#ifdef SONIC_TRACE
-    if (tid == 0 && row == (int)P.error[120]) P.error[29] = Pn2;
-#endif
     const int PnAll = Pn;
     (void)PnAll;
 #define Pn Pn2
@@ -606,10 +584,6 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
     }
     (void)sorted;
 #undef Pn
-    MERGE_STAMP(3);
-#ifdef SONIC_TRACE
-    if (tid == 0 && row == (int)P.error[120]) { P.error[30] = Pn; P.error[31] = n; }
-#endif
 
     if (P.op == OP_TOPK) {
         for (int j = tid; j < n; j += THREADS) {
@@ -803,7 +777,6 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
     unsigned long long *ik = v.ik;
     const double W = cs[n - 1];                 // still the ranking-order cumulative sums here
     csync();
-    MERGE_STAMP(7);
     const uint32_t a_acc = cells.x, a_draw = cells.y;      // the row's Philox cells, drawn before the wait on the streaming kernel
     const double u_draw = cell_to_u(a_draw);
     uint32_t flags = 0;
@@ -883,14 +856,12 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
             if (cs[j] > target && (j == 0 || !(cs[j - 1] > target))) sh.pick = j;
         csync();
     }
-    MERGE_STAMP(8);
     if (tid == 0) {
         int j = sh.pick;
         int token = (int)(~(uint32_t)(ik[j] >> 32));
         float prob = (float)(w[(uint32_t)ik[j]] / W);
         emit_row(P, c, row, token, prob, flags, n, p_draft);
     }
-    MERGE_STAMP(9);
 }
 
 
@@ -900,9 +871,7 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
     epilogue_weights<NT>(n, buf, tid);
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
     csync();
-    MERGE_STAMP(4);
     n = epilogue_truncate<NT, Sync>(c, n, buf, sh, tid);
-    MERGE_STAMP(6);
     epilogue_index_order<NT, Sync>(n, buf, tid);
     epilogue_tail<NT, Sync>(P, c, row, n, buf, sh, tid, cells);
 }
@@ -914,11 +883,9 @@ __device__ void merge_epilogue_small(const KParams &P, const RowCfg &c, int row,
     epilogue_weights<THREADS>(n, buf, tid);
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
     __syncthreads();
-    MERGE_STAMP(4);
     if (tid < 32) epilogue_truncate_warp(c, n, buf, sh, tid);
     __syncthreads();
     n = sh.n_p;
-    MERGE_STAMP(6);
     epilogue_index_order<THREADS, BlockSync>(n, buf, tid);
     if (tid < 32) epilogue_tail<32, WarpSync>(P, c, row, n, buf, sh, tid, cells);
 }
@@ -979,7 +946,6 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
     ConsumerSync csync;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (warp == 0) STREAM_STAMP(0);
     KERNEL_T0(0);
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], STREAM_WARPS); }
@@ -1116,7 +1082,6 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
         int n = 0;
         Prep p_next{0, 0, 0};
         int item = current_item();
-        STREAM_STAMP(1);
         bool prepared = false;
         // lane 0: the tile's bulk copy, with the arrival on full[s] (arrive == true) or with the bytes announced only
         // (the arrival then follows once the stage's description is written)
@@ -1149,14 +1114,12 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             }
             if (item < 0) {                            // out of work: tell the consumers
                 if (lane == 0) { sh.meta[s].stop = 1; mbar_arrive(&sh.full[s]); }
-                STREAM_STAMP(5);
                 break;
             }
             const int row = item / tiles, tile = item - row * tiles;
             if (!prepared) {                           // the CTA's first tile: nothing was prepared ahead
                 p_next = prepare(row, tile, n % (NSTAGE + 1));
                 prepared = true;
-                STREAM_STAMP(2);
             }
             const RowCfg c = c_next;
             const Prep pr = p_next;
@@ -1198,7 +1161,7 @@ sonic_stream_kernel(const KParams P, const int tiles, const int nitems, const in
             if (lane == 0) atomicOr(P.error, ERR_TIMEOUT);
             return;
         }
-        if (sh.meta[s].stop) { if (warp == 0) STREAM_STAMP(6); KERNEL_T1(0); break; }
+        if (sh.meta[s].stop) { KERNEL_T1(0); break; }
         const int row = sh.meta[s].row, tile = sh.meta[s].tile;
         const int tile_base = tile * CTA_TILE;
         const int wbase = tile_base + warp * WARP_TILE;
