@@ -186,8 +186,8 @@ def test_many_short_rows_through_the_work_queue(sonic, oracle):
 
 
 def test_two_host_threads_share_the_device(sonic, oracle):
-    # two threads, each with its own stream and workspace, call into the library at the same time (the calls
-    # enqueue one at a time and share the library's internal side stream)
+    # two threads, each with its own stream and workspace, call into the library at the same time (each thread gets
+    # an internal stream of its own for the histogram passes)
     import threading
     import torch
     ws = [wl.config1(), wl.config1()]
