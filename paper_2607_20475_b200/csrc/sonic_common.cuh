@@ -341,7 +341,8 @@ __device__ __forceinline__ RowCfg load_cfg(const KParams &P, int row) { return r
 
 #ifdef SONIC_TRACE
 __device__ __forceinline__ unsigned int gtimer_lo() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned int)t; }
-// kernel-level timeline: earliest start and latest end of kernel k (0 stream, 1 merge, 2 exact first launch, 3 exact second launch)
+// kernel-level timeline (trace variant of the library only): earliest start and latest end of kernel k over its CTAs
+// (0 stream, 1 merge, 6 histogram pass, 3 collect pass, 8 row finish, 4 residual pass, 9 residual draw, 2 cluster kernel, 5 combine)
 #define KERNEL_T0(k) do { if (threadIdx.x == 0) atomicMin(&P.error[48 + 2 * (k)], gtimer_lo()); } while (0)
 #define KERNEL_T1(k) do { if (threadIdx.x == 0) atomicMax(&P.error[49 + 2 * (k)], gtimer_lo()); } while (0)
 #else

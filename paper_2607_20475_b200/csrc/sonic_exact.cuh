@@ -4,10 +4,12 @@
 // over count / probability-mass histograms, cluster-wide reductions going
 // through DSMEM and hardware cluster barriers (no flags, no spinning).
 //
-// It serves (a) rows whose answer needs the whole vocabulary by construction
-// (top-k off, or k beyond what the streaming path sorts) and (b) rows the
-// streaming path could not prove.  The paper bounds k at 128 and is lossy
-// beyond it (Section 3.3); this path removes that bound.
+// It is the last resort of a call: (a) rows with a top-k beyond what the
+// streaming path sorts, (b) rows the streaming path could not prove, (c) rows
+// of the histogram path whose crossing bin was too crowded.  Usually there is
+// none and the kernel returns at once.  (Rows with top-k off are finished by the
+// histogram passes, sonic_dense.cuh.)  The paper bounds k at 128 and is lossy
+// beyond it (Section 3.3); this path and the histogram path remove that bound.
 //
 // Probability mass is accumulated as 64-bit fixed point (2^-40 units of the
 // largest weight), so sums are order-independent and replays are bit-identical.
@@ -18,7 +20,6 @@
 
 namespace sonic {
 namespace cg = cooperative_groups;
-
 
 constexpr int EX_THREADS = 512;
 constexpr int EX_WARPS = EX_THREADS / 32;
@@ -49,7 +50,7 @@ struct ExactShared {
     unsigned int red_cnt[HBINS / CL];
     unsigned int ucount;
     int flag;
-    int ticket;                                      // first round: the ordinal of the cluster's next row
+    int ticket;                                      // the ordinal of the cluster's next row
 };
 
 struct ExactCtx {
