@@ -545,11 +545,15 @@ __device__ __forceinline__ int dense_warp_draw(const KParams &P, int row, int ti
 // Last arriver of pass C: the exact cut, the support's size and mass, then the draw or the accept test.
 // dyn: DENSE_DYN_SMEM bytes; cells: the row's two Philox cells.  Returns false if the row must go to the cluster kernel.
 __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int tiles, DenseShared &sm, unsigned long long *dyn, int tid,
-                             uint32_t Mkey, bool listed, unsigned long long target, uint32_t tk, uint2 cells) {
+                             uint32_t Mkey, bool listed, unsigned long long target, uint32_t tk, uint2 cells, int draft, float q_draft) {
     const float Mf = unkey(Mkey);
     const int lane = tid & 31, warp = tid >> 5;
     DenseRow *dr = P.drow + row;
     DenseTile *dt = P.dtile + (size_t)row * MAX_TILES;
+    // verification: the draft token's key goes out with the row's other loads (the token itself and its draft
+    // probability are inputs, read by the caller before the wait; draft = -1: no draft, or an id outside the vocabulary)
+    uint32_t key_draft = 0u;
+    if (draft >= 0) key_draft = __ldcg(&P.ykeys[(size_t)row * ((size_t)P.ytiles * CTA_TILE) + draft]);
     // everything the other CTAs left, requested at once: a chunk record per thread, the first DENSE_THREADS listed
     // elements (one per thread, whatever their number turns out to be), their count and the overflow mark
     unsigned int nm = 0u, overflow = 0u;
@@ -803,13 +807,12 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
     uint32_t flags = F_DENSE;
     float p_draft = 0.0f;
     if (P.op == OP_VERIFY && c.l < P.K) {
-        const int d = P.draft_tokens[(size_t)c.b * P.K + c.l];
+        const int d = P.draft_tokens[(size_t)c.b * P.K + c.l];        // (the value the caller read; an id outside the vocabulary is reported as it is)
         unsigned long long qd = 0ull;
         double Q = 0.0;
-        if (d >= 0 && d < P.V) {
-            const uint32_t kd = P.ykeys[(size_t)row * ((size_t)P.ytiles * CTA_TILE) + d];
-            if ((((unsigned long long)kd << 32) | (uint32_t)(~(uint32_t)d)) >= cutc) qd = qweight(kd, Mf);
-            Q = (double)__ldg(P.draft_probs + ((size_t)c.b * P.K + c.l) * (size_t)P.V + d);
+        if (draft >= 0) {
+            if ((((unsigned long long)key_draft << 32) | (uint32_t)(~(uint32_t)draft)) >= cutc) qd = qweight(key_draft, Mf);
+            Q = (double)q_draft;
         }
         const double Pd = (double)qd / (double)W;
         const bool accept = (Pd > 0.0) && (cell_to_u(a_acc) * Q <= Pd);
@@ -993,6 +996,16 @@ sonic_dense_finish_kernel(const KParams P, const int tiles) {
     }
     const int req = (P.op == OP_VERIFY) ? row / (P.K + 1) : row;
     const unsigned long long seed = P.seed ? P.seed[req] : 0ull, off = P.offset ? P.offset[req] : 0ull;
+    // verification: the position's draft token and its draft probability (inputs)
+    int draft = -1;
+    float q_draft = 0.0f;
+    if (P.op == OP_VERIFY) {
+        const int l = row - req * (P.K + 1);
+        if (l < P.K) {
+            const int d = P.draft_tokens[(size_t)req * P.K + l];
+            if (d >= 0 && d < P.V) { draft = d; q_draft = __ldg(P.draft_probs + ((size_t)req * P.K + l) * (size_t)P.V + d); }
+        }
+    }
     pdl_wait_primary();
     KERNEL_T0(8);
     {
@@ -1007,7 +1020,7 @@ sonic_dense_finish_kernel(const KParams P, const int tiles) {
             const unsigned long long pos = off + (unsigned long long)c.l;
             philox4x32_10((uint32_t)pos, (uint32_t)(pos >> 32), (uint32_t)c.b, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), r4);
             const uint2 cells = make_uint2(r4[0] >> 8, r4[1] >> 8);
-            const bool ok = dense_finish(P, c, row, tiles, sm, dyn, tid, par.Mkey, par.klo <= par.khi, par.target, par.tk, cells);
+            const bool ok = dense_finish(P, c, row, tiles, sm, dyn, tid, par.Mkey, par.klo <= par.khi, par.target, par.tk, cells, draft, q_draft);
             if (!ok && tid == 0) { P.rs[row].status = ST_FAILED; atomicAdd(&P.error[WS_FAILED_ROWS], 1u); }
         }
     }
