@@ -17,7 +17,7 @@
  *   0x040 greedy selection      0x080 top-k                0x100 top-p
  *   0x200 min-p                 0x400 top-k log-probabilities (reserved, ignored)
  * A parameter array may be NULL when no request sets the bit that reads it.
- * Parameter domains: tau > 0 finite; k >= 0; p, theta in (0, 1]; rep_penalty alpha > 0 finite (the paper states
+ * Parameter domains: tau > 0 finite; k >= 0 (0: no top-k); p, theta in (0, 1] (p = 1: no top-p truncation); rep_penalty alpha > 0 finite (the paper states
  * alpha >= 1), freq_penalty and pres_penalty finite (the paper states >= 0); a set bit with a parameter outside
  * its domain gives SONIC_FLAG_BADPARAM for that row (greedy rows too, for tau and the penalty coefficients).
  * Bias values and logits must not be NaN or +inf (a precondition, not checked; -inf logits are masked entries).

@@ -219,7 +219,10 @@ static trunc_t truncate_row(const item_t *items, int V, uint32_t z, int k, float
     }
     double Z = C[n - 1];
     int n_keep = n;
-    if (z & ORACLE_TOP_P) {
+    /* TopP (Appendix "Probability Truncation"): the smallest ranking prefix whose mass reaches p * Z.  At p = 1 that is
+     * the whole set (every weight is positive); taken literally the comparison C_j >= 1 * Z would be decided by the
+     * rounding of the running sum, so p = 1 is read as "no truncation". */
+    if ((z & ORACLE_TOP_P) && p < 1.0f) {
         double target = (double)p * Z;
         int np_ = n;
         for (int j = 0; j < n; ++j) {

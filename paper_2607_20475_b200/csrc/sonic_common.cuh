@@ -312,6 +312,9 @@ __device__ __forceinline__ RowCfg resolve_cfg(const KParams &P, int row, const C
         if ((z & M_MIN_P) && !(c.theta > 0.0f && c.theta <= 1.0f)) c.bad = true;
     }
     if (c.k < 0) c.k = 0;
+    // TopP with p = 1 keeps every survivor of the other filters (the whole mass is reached by the whole set only; in
+    // floating point the comparison would be decided by rounding): the bit is dropped
+    if ((z & M_TOP_P) && c.p >= 1.0f) { z &= ~M_TOP_P; c.z = z; c.p = 1.0f; }
     c.div_all = false;
     c.G = 0;
     c.tile_min = false;

@@ -135,6 +135,24 @@ def test_edge_rows(sonic, oracle):
     assert got["token"][3] == 7 and got["token"][9] == 0 and got["token"][2] == 12345
 
 
+def test_top_p_one_keeps_every_survivor(sonic, oracle):
+    # p = 1 with the bit set is "no truncation" on peaked rows whose tail no longer moves a floating-point sum:
+    # with top-k off (histogram path), with top-k (merge), with min-p, in a verification-free sampling call
+    V = 30000
+    rng = np.random.default_rng(13)
+    x = (rng.standard_normal((6, V)) * 3).astype(np.float32)
+    x[:, 17] += 60.0                                      # one token holds all but 1e-20 of the mass
+    mode = [wl.TOP_P, wl.TOP_P | wl.TEMPERATURE, wl.TOP_P | wl.TOP_K, wl.TOP_P | wl.MIN_P, wl.TOP_P | wl.TOP_K | wl.TEMPERATURE,
+            wl.TOP_P]
+    w = make_sample(x, mode, temperature=[1, 0.3, 1, 1, 0.5, 1], top_p=[1, 1, 1, 1, 1, np.float32(1 - 2.0 ** -16)],
+                    top_k=[0, 0, 700, 0, 50, 0], min_p=[0, 0, 0, 1e-30, 0, 0], seed=np.arange(6) + 70)
+    got, ref, n = run_sample(sonic, oracle, w)
+    assert n == 0
+    assert ref["support"].tolist()[:3] == [V, V, 700] and ref["support"][4] == 50 and ref["support"][5] == 1
+    assert got["support"].tolist() == ref["support"].tolist()
+    assert np.all(got["token"] == 17)
+
+
 def test_penalty_coefficients_outside_their_domain(sonic, oracle):
     # Appendix "Repetition Penalties": alpha >= 1, beta >= 0, gamma >= 0.  A divisor that is not positive and finite, or a
     # coefficient that is not finite, is a bad parameter (greedy rows too); a clear bit hides any value

@@ -283,6 +283,21 @@ def test_no_token_and_bad_parameters():
     assert out["flags"].tolist() == [1, 0, 2]
 
 
+def test_top_p_one_keeps_every_survivor():
+    # Appendix "Probability Truncation": the nucleus of mass >= p * Z.  At p = 1 only the whole set reaches the whole
+    # mass; in floating point the running sum of a peaked row stops growing long before the last token (here after
+    # the first: 1 + e^-50 == 1 in fp64), so the literal comparison would keep one token.  p = 1 means no truncation.
+    x = np.array([[0.0, -50.0, -60.0, -np.inf, -55.0, -70.0]], dtype=np.float32).repeat(3, 0)
+    w = make_sample(x, [wl.TOP_P, wl.TOP_P | wl.TOP_K, wl.TOP_P | wl.MIN_P], top_p=[1.0, 1.0, 1.0], top_k=[0, 3, 0],
+                    min_p=[0.0, 0.0, 1e-25])
+    out = oracle.sample(w)
+    assert out["support"].tolist() == [5, 3, 3]          # every finite token; the 3 best; those above ln(1e-25) = -57.6
+    assert out["token"].tolist() == [0, 0, 0] and np.all(out["margin"] > 1e-3)
+    # just below 1 the nucleus is decided by the masses again
+    out = oracle.sample(make_sample(x[:1], [wl.TOP_P], top_p=[np.float32(1.0 - 2.0 ** -20)]))
+    assert out["support"].tolist() == [1]
+
+
 def test_penalty_coefficients_outside_their_domain_are_bad_parameters():
     # Appendix "Repetition Penalties" states alpha >= 1, beta >= 0, gamma >= 0; a coefficient that would make a logit NaN
     # or infinite (divisor not positive and finite, coefficient not finite) is reported like any bad parameter,
