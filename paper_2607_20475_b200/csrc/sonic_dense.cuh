@@ -542,6 +542,17 @@ __device__ __forceinline__ int dense_warp_draw(const KParams &P, int row, int ti
     return token;
 }
 
+// 64-bit add to a shared-memory word as two native 32-bit atomics (low word first: the value it returns tells whether
+// the sum carried).  A 64-bit shared-memory atomic is a compare-and-swap loop, which crawls when many lanes add to a
+// handful of words (the per-tile masses of a row: 16 words, hundreds of listed elements).
+__device__ __forceinline__ void smem_add_u64(unsigned long long *p, unsigned long long w) {
+    unsigned int *q = reinterpret_cast<unsigned int *>(p);
+    const unsigned int lo = (unsigned int)w, hi = (unsigned int)(w >> 32);
+    unsigned int carry = 0u;
+    if (lo) { const unsigned int old = atomicAdd(q, lo); carry = (old + lo < old) ? 1u : 0u; }
+    if (hi + carry) atomicAdd(q + 1, hi + carry);
+}
+
 // Last arriver of pass C: the exact cut, the support's size and mass, then the draw or the accept test.
 // dyn: DENSE_DYN_SMEM bytes; cells: the row's two Philox cells.  Returns false if the row must go to the cluster kernel.
 __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int tiles, DenseShared &sm, unsigned long long *dyn, int tid,
@@ -704,7 +715,7 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
                 if (subbin(key) > xb && m >= cutc) {
                     const unsigned long long w = qweight(key, Mf);
                     const uint32_t idx = ~(uint32_t)m;
-                    if (w) { atomicAdd(&sm.tile_mass[idx / CTA_TILE], w); atomicAdd(&sm.chunk[idx / DENSE_CHUNK], w); }
+                    if (w) { smem_add_u64(&sm.tile_mass[idx / CTA_TILE], w); smem_add_u64(&sm.chunk[idx / DENSE_CHUNK], w); }
                 }
             }
             __syncthreads();
@@ -740,8 +751,8 @@ __device__ bool dense_finish(const KParams &P, const RowCfg &c, int row, int til
             const bool inc = have && mine_c >= cutc;
             if (inc && mine_w) {
                 const uint32_t idx = ~(uint32_t)mine_c;
-                atomicAdd(&sm.tile_mass[idx / CTA_TILE], mine_w);
-                atomicAdd(&sm.chunk[idx / DENSE_CHUNK], mine_w);
+                smem_add_u64(&sm.tile_mass[idx / CTA_TILE], mine_w);
+                smem_add_u64(&sm.chunk[idx / DENSE_CHUNK], mine_w);
             }
             n_in = (unsigned int)__syncthreads_count(inc ? 1 : 0);
             if (have && (unsigned int)tid + 1u == n_in) sm.bc64[1] = pre + mine_w;
