@@ -163,10 +163,14 @@ __device__ __forceinline__ int dense_pick_sub(int rows_in_pass, int tiles, int c
     while (sub < 4 && rows_in_pass * tiles * sub * 2 <= ctas) sub *= 2;
     return sub;
 }
-__device__ __forceinline__ DenseItem dense_item(const int *list, int item, int tiles, int sub) {
+// `head`: the lane's entry of the list's first 32 (requested together with the list's length, so that a CTA's first row
+// is known after one round trip instead of two); every thread of the CTA calls this at the same point.
+__device__ __forceinline__ DenseItem dense_item(const int *list, int head, int item, int tiles, int sub) {
     DenseItem it;
     const int per_row = tiles * sub;
-    it.row = __ldcg(&list[item / per_row]);
+    const int slot = item / per_row;
+    const int from_head = __shfl_sync(0xFFFFFFFFu, head, slot & 31);
+    it.row = (slot < 32) ? from_head : __ldcg(&list[slot]);
     const int rem = item % per_row;
     it.tile = rem / sub; it.part = rem % sub; it.sub = sub;
     return it;
@@ -938,6 +942,7 @@ __device__ __forceinline__ DenseRowPar dense_row_par(const KParams &P, int row, 
 // for another: the rows are finished in the kernel that follows (sonic_dense_finish_kernel).
 __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta, int ncta, unsigned long long *dyn, DenseShared &sm, const int stage) {
     const int tid = threadIdx.x;
+    const int head = __ldcg(&P.dlist[tid & 31]);          // (the list's region holds 64 entries at least)
     const int nd = (int)__ldcg(&P.error[WS_NDENSE]);
     const int sub = dense_pick_sub(nd, tiles, ncta);
     const int per_row = tiles * sub;
@@ -946,7 +951,7 @@ __device__ __forceinline__ void dense_items(const KParams &P, int tiles, int cta
     DenseRowPar par;
     par.kind = 0;
     for (int item = rg.lo; item < rg.hi; ++item) {
-        const DenseItem it = dense_item(P.dlist, item, tiles, sub);
+        const DenseItem it = dense_item(P.dlist, head, item, tiles, sub);
         uint4 kv[DENSE_NV];
         dense_load_keys(P, it, tid, kv);
         if (it.row != cur_row) {
@@ -1132,6 +1137,7 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
     pdl_launch_dependents();
     pdl_wait_primary();
     KERNEL_T0(4);
+    const int head = __ldcg(&P.rlist[tid & 31]);
     const int nr = (int)__ldcg(&P.error[WS_NRESID]);
     const DenseRange rg = dense_range(nr * tiles, (int)blockIdx.x, (int)gridDim.x);
     int cur_row = -1;
@@ -1140,7 +1146,7 @@ sonic_dense_resid_kernel(const KParams P, const int tiles) {
     double Md = 0.0, inv_Wt = 0.0;
     const float *q = nullptr;
     for (int item = rg.lo; item < rg.hi; ++item) {
-        const DenseItem it = dense_item(P.rlist, item, tiles, 1);
+        const DenseItem it = dense_item(P.rlist, head, item, tiles, 1);
         const int row = it.row, tile = it.tile;
         uint4 kv[DENSE_NV];
         dense_load_keys(P, it, tid, kv);
