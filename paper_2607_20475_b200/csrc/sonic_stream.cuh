@@ -99,6 +99,8 @@ struct MergeShared {
     unsigned int tkey;
     int n_p, n_m, pick;
     int found;
+    int wsum[THREADS / 32];                    // a block scan's warp totals
+    int bracket[4];                            // the counting bins' answer: bin, count above it, count with it
     alignas(16) double scratch[THREADS];      // also read as int4
 };
 
@@ -158,8 +160,24 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         return keep ? (((unsigned long long)yk << 32) | (uint32_t)cd) : 0ull;
     };
     unsigned long long floor_key = 1ull;           // keys below it are left out (1: every proven candidate)
+    // Large k: while the candidates are gathered they are also counted in 1024 bins of 8192 keys above the proven
+    // threshold (one binade of fp32 keys; whatever lies higher shares the top bin).  The bin in which the count from
+    // the top reaches k then brackets the k-th key without a pass of its own (GBINS ints in sh.scratch).
+    constexpr int GBINS = 2 * THREADS, GSHIFT = 13;
+    static_assert(GBINS * 4 <= THREADS * 8, "the counting bins live in the scratch words");
+    int *ghist = reinterpret_cast<int *>(sh.scratch);
+    const uint32_t gbase = c.temp ? tykey : tkey;
+    const bool use_bins = !complete && c.k > RANK_SORT_MAX / 2 && total > RANK_SORT_MAX;
+    auto gbin = [&](unsigned long long key) -> int {
+        const uint32_t d = ((uint32_t)(key >> 32) - gbase) >> GSHIFT;
+        return (int)min(d, (uint32_t)(GBINS - 1));
+    };
     for (int attempt = 0; attempt < 2; ++attempt) {
         unsigned long long kmax = 0ull;
+        if (use_bins) {
+            for (int i = tid; i < GBINS; i += THREADS) ghist[i] = 0;
+            csync();
+        }
         // tile-major: a warp takes tiles w and w + NW together, its lanes the slots' entries (no search for the
         // tile of an entry; the loads of both tiles are in flight at once)
         constexpr int NW = THREADS / 32, HB = GB / 2;
@@ -185,8 +203,8 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                 if (lane == 0 && nk) base = atomicAdd(&sh.count, nk);
                 base = __shfl_sync(0xFFFFFFFFu, base, 0);
                 const unsigned int below = (1u << lane) - 1u;
-                if (oa >= floor_key) { const int pos = base + __popc(ma & below); if (pos < MERGE_CAP) buf[pos] = oa; }
-                if (ob >= floor_key) { const int pos = base + __popc(ma) + __popc(mb & below); if (pos < MERGE_CAP) buf[pos] = ob; }
+                if (oa >= floor_key) { const int pos = base + __popc(ma & below); if (pos < MERGE_CAP) buf[pos] = oa; if (use_bins) atomicAdd(&ghist[gbin(oa)], 1); }
+                if (ob >= floor_key) { const int pos = base + __popc(ma) + __popc(mb & below); if (pos < MERGE_CAP) buf[pos] = ob; if (use_bins) atomicAdd(&ghist[gbin(ob)], 1); }
                 continue;
             }
             for (int j0 = 0; j0 < max(na, nb); j0 += (single ? 32 * GB : 32 * HB)) {
@@ -219,6 +237,7 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
                     if (out[u] >= floor_key) {
                         const int pos = base + __popc(km[u] & ((1u << lane) - 1u));
                         if (pos < MERGE_CAP) buf[pos] = out[u];
+                        if (use_bins) atomicAdd(&ghist[gbin(out[u])], 1);
                     }
                     base += __popc(km[u]);
                 }
@@ -397,7 +416,48 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         // such threshold keeps the n best), then sort only those
         unsigned long long lo = 0ull, hi = ~0ull;          // count(>= lo) >= n > count(>= hi)
         bool tight = false;
-        {
+        bool bracketed = false;
+        int cnt_lo = Pn, cnt_hi = 0;
+        if (use_bins) {
+            // the bins counted during the gather: thread t owns bins GBINS-1-2t and GBINS-2-2t (from the top)
+            constexpr int BPT = GBINS / THREADS;
+            const int lane = tid & 31, warp = tid >> 5;
+            int v[BPT], sum = 0;
+#pragma unroll
+            for (int j = 0; j < BPT; ++j) { v[j] = ghist[GBINS - 1 - (tid * BPT + j)]; sum += v[j]; }
+            int incl = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (lane == 31) sh.wsum[warp] = incl;
+            if (tid == 0) sh.bracket[0] = -1;
+            csync();
+            int pre = incl - sum;
+            for (int w = 0; w < warp; ++w) pre += sh.wsum[w];
+            if (pre < n && pre + sum >= n) {
+                int run = pre;
+#pragma unroll
+                for (int j = 0; j < BPT; ++j) {
+                    if (run < n && run + v[j] >= n) { sh.bracket[0] = GBINS - 1 - (tid * BPT + j); sh.bracket[1] = run; sh.bracket[2] = run + v[j]; }
+                    run += v[j];
+                }
+            }
+            csync();
+            const int b = sh.bracket[0];
+            if (b >= 0) {
+                // bin b holds the keys gbase + (b << GSHIFT) .. gbase + ((b + 1) << GSHIFT) - 1 (the top bin: and all above)
+                const unsigned long long klo = (unsigned long long)gbase + ((unsigned long long)b << GSHIFT);
+                lo = klo << 32;
+                hi = (b == GBINS - 1 || klo + (1ull << GSHIFT) > 0xFFFFFFFFull) ? ~0ull : ((klo + (1ull << GSHIFT)) << 32);
+                cnt_hi = sh.bracket[1];
+                cnt_lo = sh.bracket[2];
+                bracketed = true;
+            }
+            csync();
+        }
+        if (!bracketed) {
             // First bracket from the data itself: 31 of the keys, sorted, split the candidates into 32 buckets of
             // about equal population wherever the keys crowd; one counting pass then places n within one bucket.
             unsigned long long *sth = reinterpret_cast<unsigned long long *>(sh.scratch);          // [32] ascending, last = sentinel
@@ -448,9 +508,11 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
             }
             csync();
             lo = res[0]; hi = res[1];
-            const int cnt_lo = (int)res[2], cnt_hi = (int)res[3];
-            tight = cnt_lo <= want_hi;
+            cnt_lo = (int)res[2]; cnt_hi = (int)res[3];
             csync();
+        }
+        {
+            tight = cnt_lo <= want_hi;
             // The bucket [lo, hi) holds the boundary.  If it is small, its keys are collected and ranked, which gives
             // the threshold that keeps exactly n (no search over key space, whose passes multiply when equal values
             // differ only in their index bits).
