@@ -927,6 +927,88 @@ __device__ __forceinline__ void epilogue_tail(const KParams &P, const RowCfg &c,
 }
 
 
+// The draw of a sampling row with a large support (more survivors than the rank counting takes): the survivors are not
+// brought into index order at all.  Their weights, as 2^-40 fixed-point integers, are added up per tile, then per 256 ids
+// of the tile the target falls into, then per id of that range; each level is one pass over the survivors, a scan of
+// at most 256 bins and a barrier.  Integer sums: the same token in every replay; against the exact index-order CDF the
+// target moves by less than n * 2^-40 of the mass.
+template <int NT, typename Sync, typename SH>
+__device__ void epilogue_draw_large(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells) {
+    Sync csync;
+    static_assert(NT >= 256, "a thread per bin");
+    EpiView v(buf);
+    const double *w = v.w;
+    const double W = v.cs[n - 1];                              // ranking-order cumulative sums: the support's mass
+    unsigned int *blo = reinterpret_cast<unsigned int *>(v.ik), *bhi = blo + 256;      // (the index keys' place: unused on this path)
+    unsigned long long *red = reinterpret_cast<unsigned long long *>(sh.scratch);
+    const int lane = tid & 31, warp = tid >> 5;
+    auto fixed = [&](int j) -> unsigned long long { return (unsigned long long)(w[j] * 1099511627776.0); };
+    unsigned int range_lo = 0u;
+    unsigned long long rest = 0ull;
+    const int shifts[3] = {13, 8, 0};
+    const unsigned int spans[3] = {(unsigned int)MAX_TILES << 13, 8192u, 256u};
+#pragma unroll
+    for (int level = 0; level < 3; ++level) {
+        const int shift = shifts[level];
+        const unsigned int span = spans[level];
+        const int nb = (int)(span >> shift);                   // 32, 32, 256
+        if (tid < 256) { blo[tid] = 0u; bhi[tid] = 0u; }
+        csync();
+        for (int j = tid; j < n; j += NT) {
+            const unsigned int idx = ~(uint32_t)buf[j];
+            const unsigned int d = idx - range_lo;
+            const unsigned long long q = fixed(j);
+            if (d < span && q) {
+                const int b = (int)(d >> shift);
+                const unsigned int lo = (unsigned int)q, hi = (unsigned int)(q >> 32);
+                unsigned int carry = 0u;
+                if (lo) { const unsigned int old = atomicAdd(&blo[b], lo); carry = (old + lo < old) ? 1u : 0u; }
+                if (hi + carry) atomicAdd(&bhi[b], hi + carry);
+            }
+        }
+        csync();
+        // scan of the bins (a thread per bin, warps in order)
+        const unsigned long long mine = (tid < nb) ? (((unsigned long long)bhi[tid] << 32) + blo[tid]) : 0ull;
+        unsigned long long incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) red[warp] = incl;
+        if (tid == 0) sh.pick = -1;
+        csync();
+        unsigned long long before = 0ull, total = 0ull;
+        for (int wq = 0; wq < NT / 32; ++wq) { const unsigned long long t = red[wq]; before += (wq < warp) ? t : 0ull; total += t; }
+        if (level == 0) rest = draw_target(total, cells.y);     // the support's mass in fixed point, and the draw's target in it
+        const unsigned long long excl = before + incl - mine;
+        if (mine > 0ull && excl <= rest && rest < excl + mine) { sh.pick = tid; red[32] = excl; }
+        csync();
+        int b = sh.pick;
+        if (b < 0) {                                           // (rest < total always; kept for safety: the last bin with mass)
+            if (mine > 0ull) atomicMax(&sh.pick, tid);
+            csync();
+            b = sh.pick;
+            if (tid == b) red[32] = excl;
+            csync();
+        }
+        const unsigned long long excl_b = red[32];
+        rest = (rest > excl_b) ? rest - excl_b : 0ull;
+        range_lo += (unsigned int)b << shift;
+        csync();
+    }
+    // the survivor with that id
+    if (tid == 0) sh.pick = 0;
+    csync();
+    for (int j = tid; j < n; j += NT)
+        if (~(uint32_t)buf[j] == range_lo) sh.pick = j;
+    csync();
+    if (tid == 0) {
+        const int j = sh.pick;
+        emit_row(P, c, row, (int)(~(uint32_t)buf[j]), (float)(w[j] / W), 0u, n, 0.0f);
+    }
+}
+
 template <int NT, typename Sync, typename SH>
 __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n, unsigned long long *buf, SH &sh, int tid, uint2 cells) {
     Sync csync;
@@ -934,6 +1016,10 @@ __device__ void merge_epilogue(const KParams &P, const RowCfg &c, int row, int n
     if (tid == 0) { sh.n_p = n; sh.n_m = n; sh.found = 0; sh.pick = -1; }
     csync();
     n = epilogue_truncate<NT, Sync>(c, n, buf, sh, tid);
+    if (P.op == OP_SAMPLE && n > RANK_SORT_MAX) {
+        epilogue_draw_large<NT, Sync>(P, c, row, n, buf, sh, tid, cells);
+        return;
+    }
     epilogue_index_order<NT, Sync>(n, buf, tid);
     epilogue_tail<NT, Sync>(P, c, row, n, buf, sh, tid, cells);
 }
