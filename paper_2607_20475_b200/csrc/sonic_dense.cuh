@@ -253,18 +253,25 @@ __device__ __forceinline__ void dense_hist_item(const KParams &P, const DenseIte
 
 // Row step of pass H: the crossing bin of top-p against the min-p threshold, as the key interval pass C works with
 // (in every thread: klo, khi, tk, target).  Every CTA of pass C that meets the row computes it for itself from the
-// row's histogram (16 KB, one round of loads); `store` (the CTA of the row's first item) leaves it for the row's finish.
+// row's histogram (16 KB, four bins per thread); `store` (the CTA of the row's first item) leaves it for the row's finish.
 struct DenseCut { uint32_t tk, klo, khi; unsigned long long target; };
-__device__ __forceinline__ DenseCut dense_hist_finish(const KParams &P, const RowCfg &c, int row, DenseShared &sm,
-                                                      unsigned long long *h, int tid, uint32_t Mkey, float scale, bool store) {
+// A thread's bins of the row's histogram: thread t owns bins DBINS-1-4t .. DBINS-4-4t (from the top).  Requested by the
+// caller before the row's other loads are waited for.
+constexpr int DENSE_BPT = DBINS / DENSE_THREADS;
+struct DenseBins { unsigned long long v[DENSE_BPT]; };
+__device__ __forceinline__ DenseBins dense_load_bins(const KParams &P, int row, int tid) {
     const unsigned long long *hist = P.hist + (size_t)row * DBINS;
-    for (int i = tid; i < DBINS; i += DENSE_THREADS) h[i] = hist[i];
-    __syncthreads();
-    // thread t owns bins DBINS-1-4t .. DBINS-4-4t (from the top)
-    constexpr int BPT = DBINS / DENSE_THREADS;
+    DenseBins b;
+#pragma unroll
+    for (int j = 0; j < DENSE_BPT; ++j) b.v[j] = __ldcg(&hist[DBINS - 1 - (tid * DENSE_BPT + j)]);
+    return b;
+}
+__device__ __forceinline__ DenseCut dense_hist_finish(const KParams &P, const RowCfg &c, int row, DenseShared &sm,
+                                                      const DenseBins &bins, int tid, uint32_t Mkey, float scale, bool store) {
+    constexpr int BPT = DENSE_BPT;
     unsigned long long mine = 0;
 #pragma unroll
-    for (int j = 0; j < BPT; ++j) mine += h[DBINS - 1 - (tid * BPT + j)];
+    for (int j = 0; j < BPT; ++j) mine += bins.v[j];
     unsigned long long Z;
     const unsigned long long pre = dense_block_scan<unsigned long long>(mine, sm.red64, tid, Z);
     unsigned long long target = (unsigned long long)ceil((double)c.p * (double)Z);
@@ -278,7 +285,7 @@ __device__ __forceinline__ DenseCut dense_hist_finish(const KParams &P, const Ro
 #pragma unroll
         for (int j = 0; j < BPT; ++j) {
             const int b = DBINS - 1 - (tid * BPT + j);
-            cum += h[b];
+            cum += bins.v[j];
             if (found < 0 && cum >= target) found = b;
         }
         sm.digit = found;
@@ -908,6 +915,8 @@ __device__ __forceinline__ DenseRowPar dense_row_par(const KParams &P, int row, 
     const DenseRow *dr = P.drow + row;
     uint32_t s_tk = 0u, s_klo = 0u, s_khi = 0u, s_state = 0u;
     unsigned long long s_target = 0ull;
+    DenseBins bins;
+    if (stage == 3) bins = dense_load_bins(P, row, tid);          // (only top-p rows use them; asked for before anything is waited for)
     if (stage == 4) { s_state = __ldcg(&dr->state); s_tk = __ldcg(&dr->tk); s_klo = __ldcg(&dr->klo); s_khi = __ldcg(&dr->khi); s_target = __ldcg(&dr->target); }
     dense_row_stats(P, row, tiles, sm, tid);
     __syncthreads();
@@ -924,7 +933,7 @@ __device__ __forceinline__ DenseRowPar dense_row_par(const KParams &P, int row, 
         if (stage == 2) {
             r.kind = 1; r.scale = dense_scale(r.Mkey, mkey, Nf);
         } else if (stage == 3) {
-            const DenseCut cut = dense_hist_finish(P, c, row, sm, dyn, tid, r.Mkey, dense_scale(r.Mkey, mkey, Nf), first);
+            const DenseCut cut = dense_hist_finish(P, c, row, sm, bins, tid, r.Mkey, dense_scale(r.Mkey, mkey, Nf), first);
             r.kind = 2; r.tk = cut.tk; r.klo = cut.klo; r.khi = cut.khi; r.target = cut.target;
         } else if (s_state == 1u) {
             r.kind = 2; r.tk = s_tk; r.klo = s_klo; r.khi = s_khi; r.target = s_target;
