@@ -172,6 +172,37 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         const uint32_t d = ((uint32_t)(key >> 32) - gbase) >> GSHIFT;
         return (int)min(d, (uint32_t)(GBINS - 1));
     };
+    // the bin in which the count from the top reaches `need`, the count above it and the count with it (bin < 0: the
+    // bins hold fewer than `need`); thread t owns bins GBINS-1-2t and GBINS-2-2t.  Two barriers.
+    auto bins_find = [&](int need, int &bin, int &above, int &with) {
+        constexpr int BPT = GBINS / THREADS;
+        const int lane_ = tid & 31, warp_ = tid >> 5;
+        int v[BPT], sum = 0;
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) { v[j] = ghist[GBINS - 1 - (tid * BPT + j)]; sum += v[j]; }
+        int incl = sum;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane_ >= off) incl += o;
+        }
+        if (lane_ == 31) sh.wsum[warp_] = incl;
+        if (tid == 0) sh.bracket[0] = -1;
+        csync();
+        int pre = incl - sum;
+        for (int w = 0; w < warp_; ++w) pre += sh.wsum[w];
+        if (pre < need && pre + sum >= need) {
+            int run = pre;
+#pragma unroll
+            for (int j = 0; j < BPT; ++j) {
+                if (run < need && run + v[j] >= need) { sh.bracket[0] = GBINS - 1 - (tid * BPT + j); sh.bracket[1] = run; sh.bracket[2] = run + v[j]; }
+                run += v[j];
+            }
+        }
+        csync();
+        bin = sh.bracket[0]; above = sh.bracket[1]; with = sh.bracket[2];
+        csync();
+    };
     for (int attempt = 0; attempt < 2; ++attempt) {
         unsigned long long kmax = 0ull;
         if (use_bins) {
@@ -245,8 +276,19 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         }
         csync();
         if (attempt == 1 || sh.count <= MERGE_CAP || sh.count < c.k) break;
-        // More proven candidates than the buffer holds (large k): find a key floor that keeps between k and
-        // MERGE_CAP of them by an eight-way search over the candidates in global memory, then pack again.
+        // More proven candidates than the buffer holds (large k): a key floor that keeps between k and MERGE_CAP of
+        // them, then pack again.  The bins counted during the pass usually give it at once ...
+        if (use_bins) {
+            int b, above, with;
+            bins_find(c.k, b, above, with);
+            if (b >= 0 && with <= MERGE_CAP) {
+                floor_key = max(1ull, ((unsigned long long)gbase + ((unsigned long long)b << GSHIFT)) << 32);
+                if (tid == 0) sh.count = 0;
+                csync();
+                continue;
+            }
+        }
+        // ... otherwise a counting pass over the candidates in global memory, and an eight-way search if that leaves too many.
         unsigned long long *red = reinterpret_cast<unsigned long long *>(sh.scratch);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, off));
@@ -419,43 +461,17 @@ __device__ bool merge_topk_row(const KParams &P, const RowCfg &c, int row, int t
         bool bracketed = false;
         int cnt_lo = Pn, cnt_hi = 0;
         if (use_bins) {
-            // the bins counted during the gather: thread t owns bins GBINS-1-2t and GBINS-2-2t (from the top)
-            constexpr int BPT = GBINS / THREADS;
-            const int lane = tid & 31, warp = tid >> 5;
-            int v[BPT], sum = 0;
-#pragma unroll
-            for (int j = 0; j < BPT; ++j) { v[j] = ghist[GBINS - 1 - (tid * BPT + j)]; sum += v[j]; }
-            int incl = sum;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                if (lane >= off) incl += o;
-            }
-            if (lane == 31) sh.wsum[warp] = incl;
-            if (tid == 0) sh.bracket[0] = -1;
-            csync();
-            int pre = incl - sum;
-            for (int w = 0; w < warp; ++w) pre += sh.wsum[w];
-            if (pre < n && pre + sum >= n) {
-                int run = pre;
-#pragma unroll
-                for (int j = 0; j < BPT; ++j) {
-                    if (run < n && run + v[j] >= n) { sh.bracket[0] = GBINS - 1 - (tid * BPT + j); sh.bracket[1] = run; sh.bracket[2] = run + v[j]; }
-                    run += v[j];
-                }
-            }
-            csync();
-            const int b = sh.bracket[0];
+            int b, above, with;
+            bins_find(n, b, above, with);
             if (b >= 0) {
                 // bin b holds the keys gbase + (b << GSHIFT) .. gbase + ((b + 1) << GSHIFT) - 1 (the top bin: and all above)
                 const unsigned long long klo = (unsigned long long)gbase + ((unsigned long long)b << GSHIFT);
                 lo = klo << 32;
                 hi = (b == GBINS - 1 || klo + (1ull << GSHIFT) > 0xFFFFFFFFull) ? ~0ull : ((klo + (1ull << GSHIFT)) << 32);
-                cnt_hi = sh.bracket[1];
-                cnt_lo = sh.bracket[2];
+                cnt_hi = above;
+                cnt_lo = with;
                 bracketed = true;
             }
-            csync();
         }
         if (!bracketed) {
             // First bracket from the data itself: 31 of the keys, sorted, split the candidates into 32 buckets of
